@@ -1,0 +1,308 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent
+of the oracle's own code paths (brute force, closed forms, invariants, library
+routines).  CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import brute, hsa_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rnd(shape, seed, scale=1.0):
+    return np.random.default_rng(seed).standard_normal(shape) * scale
+
+
+def all_blocks(H, N, groups=1):
+    return [[np.arange(O.n_blocks(N), dtype=np.int32) for _ in range(groups)] for _ in range(H)]
+
+
+# ---------------------------------------------------------------- sizes the paper prints
+def test_golden_active_kv_tokens():
+    rows = [l.split() for l in open(os.path.join(GOLD, "hkv_active_kv_tokens.txt")) if l[0] != "#"]
+    kp, frames, tpf, total = map(int, rows[0])
+    assert kp * frames * tpf == total == 49920
+    assert O.n_blocks(total) == 780          # blocks of 64
+    assert O.block_count(779, total) == 64 and O.block_count(780, total) == 0
+
+
+def test_golden_block_sizes():
+    for l in open(os.path.join(GOLD, "hsa_block_sizes.txt")):
+        if l[0] == "#":
+            continue
+        name, B, ct, ch, cw = l.split()
+        assert int(B) == int(ct) * int(ch) * int(cw)
+        if name == "intra":
+            assert int(B) == O.BLOCK
+
+
+def test_block_counts_of_configs():
+    # one continuous token stream; a single partial tail block
+    for N, nb, tail in [(46800, 732, 16), (280800, 4388, 32), (140400, 2194, 48), (2048, 32, 64)]:
+        assert O.n_blocks(N) == nb
+        assert O.block_count(nb - 1, N) == tail
+
+
+# ---------------------------------------------------------------- dense equivalence
+@pytest.mark.parametrize("causal,q_pos0,N", [(False, 150, 150), (True, 150 - 24, 150), (True, 10, 150)])
+def test_all_selected_no_linear_equals_dense_brute(causal, q_pos0, N):
+    H, d, Lq = 2, 8, 24
+    q, K, V = rnd((Lq, H, d), 1), rnd((N, H, d), 2), rnd((N, H, d), 3)
+    r = O.hsa_forward(q, K, V, q_pos0, causal, all_blocks(H, N), no_linear=True)
+    keysets = [[list(range(N)) for _ in range(Lq)] for _ in range(H)]
+    ref = np.array(brute.attention_rows(q, K, V, N, H, d, Lq, q_pos0, causal, keysets))
+    assert np.abs(r["out"] - ref).max() < 1e-12
+    assert np.abs(r["out"] - O.dense_attention(q, K, V, q_pos0, causal)).max() < 1e-12
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_all_selected_equals_torch_sdpa(causal):
+    H, d, Lq, N = 3, 16, 40, 200
+    q, K, V = rnd((Lq, H, d), 4), rnd((N, H, d), 5), rnd((N, H, d), 6)
+    q_pos0 = N - Lq if causal else N
+    r = O.hsa_forward(q, K, V, q_pos0, causal, all_blocks(H, N), no_linear=True)
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(K).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(V).permute(1, 0, 2)[None]
+    mask = None
+    if causal:
+        mask = (torch.arange(N)[None, :] <= (q_pos0 + torch.arange(Lq))[:, None])
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=mask)
+    ref = ref[0].permute(1, 0, 2).numpy()
+    assert np.abs(r["out"] - ref).max() < 1e-12
+
+
+# ---------------------------------------------------------------- linear branch identities
+@pytest.mark.parametrize("causal,q_pos0", [(False, 300), (True, 300 - 37), (True, 5)])
+def test_linear_recurrent_equals_parallel(causal, q_pos0):
+    H, d, Lq, N = 2, 16, 37, 300
+    q, K, V = rnd((Lq, H, d), 7), rnd((N, H, d), 8), rnd((N, H, d), 9)
+    a = O.linear_parallel(q, K, V, q_pos0, causal)
+    b = O.linear_recurrent(q, K, V, q_pos0, causal)
+    assert np.abs(a - b).max() <= 1e-10 * max(1.0, np.abs(a).max())
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_linear_chunked_equals_parallel(causal):
+    H, d, Lq, N = 2, 16, 50, 260
+    q, K, V = rnd((Lq, H, d), 10), rnd((N, H, d), 11), rnd((N, H, d), 12)
+    q_pos0 = N - Lq if causal else N
+    a = O.linear_parallel(q, K, V, q_pos0, causal)
+    c = O.linear_chunked(q, K, V, q_pos0, causal, boundary=N - Lq)
+    assert np.abs(a - c).max() <= 1e-10
+    if not causal:
+        S, z = O.linear_state(K, V)
+        s = O.linear_from_state(q, S, z)
+        assert np.abs(a - s).max() <= 1e-10
+
+
+def test_linear_brute_force():
+    H, d, Lq, N = 2, 4, 6, 70
+    q, K, V = rnd((Lq, H, d), 13), rnd((N, H, d), 14), rnd((N, H, d), 15)
+    for causal, q_pos0 in [(False, N), (True, N - Lq), (True, 3)]:
+        a = O.linear_parallel(q, K, V, q_pos0, causal)
+        b = np.array(brute.linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal))
+        assert np.abs(a - b).max() < 1e-12
+
+
+def test_phi_is_elu_plus_one():
+    x = np.array([-30.0, -1.0, -1e-9, 0.0, 1e-9, 2.5])
+    ref = torch.nn.functional.elu(torch.from_numpy(x)).numpy() + 1.0
+    assert np.allclose(O.phi(x), ref, rtol=0, atol=1e-15)
+    assert (O.phi(x) > 0).all()
+
+
+def test_single_token_history():
+    H, d, Lq = 2, 8, 5
+    q, K, V = rnd((Lq, H, d), 16), rnd((1, H, d), 17), rnd((1, H, d), 18)
+    r = O.hsa_forward(q, K, V, 1, False, all_blocks(H, 1))
+    for i in range(Lq):
+        assert np.allclose(r["O_sp"][i], V[0], atol=1e-14)
+        assert np.allclose(r["O_lin"][i], V[0], atol=1e-14)
+        assert np.allclose(r["out"][i], 2 * V[0], atol=1e-14)
+
+
+# ---------------------------------------------------------------- sparse branch vs brute force
+@pytest.mark.parametrize("seed", range(6))
+def test_sparse_brute_force_tiny(seed):
+    rng = np.random.default_rng(100 + seed)
+    H = int(rng.integers(1, 3))
+    d = int(rng.choice([2, 4, 8]))
+    N = int(rng.integers(1, 193))
+    Lq = int(rng.integers(1, 17))
+    causal = bool(rng.integers(0, 2))
+    q_pos0 = int(rng.integers(0, N + 1)) if causal else N
+    q, K, V = rnd((Lq, H, d), seed), rnd((N, H, d), seed + 50), rnd((N, H, d), seed + 99)
+    budgets = [int(rng.choice([0, 1, 2, -1])) for _ in range(H)]
+    sel, s = O.select_blocks(q, K, q_pos0, causal, budgets)
+    # selection against the pure-Python scorer + selector
+    bs = brute.block_scores(q, K, N, H, d, Lq)
+    nb = O.n_blocks(N)
+    for h in range(H):
+        assert np.allclose(s[h, 0], bs[h], atol=1e-13)
+        cand = [(64 * b < N) and (not causal or 64 * b <= q_pos0 + Lq - 1) for b in range(nb)]
+        assert list(sel[h][0]) == brute.topk_blocks(bs[h], cand, budgets[h])
+    # sparse output against the pure-Python attention over the selected blocks' keys
+    keysets = [[[j for b in sel[h][0] for j in range(64 * b, min(N, 64 * b + 64))]
+                for _ in range(Lq)] for h in range(H)]
+    ref = np.array(brute.attention_rows(q, K, V, N, H, d, Lq, q_pos0, causal, keysets))
+    out = O.sparse_branch(q, K, V, sel, q_pos0, causal)
+    assert np.abs(out - ref).max() < 1e-12
+
+
+def test_partition_of_unity():
+    H, d, Lq, N = 2, 8, 20, 200
+    q, K = rnd((Lq, H, d), 20), rnd((N, H, d), 21)
+    V = np.ones((N, H, d))
+    sel, _ = O.select_blocks(q, K, N, False, [2, 1])
+    r = O.hsa_forward(q, K, V, N, False, sel)
+    assert np.allclose(r["O_sp"], 1.0, atol=1e-14)
+    assert np.allclose(r["O_lin"], 1.0, atol=1e-14)
+    assert np.allclose(r["out"], 2.0, atol=1e-13)
+
+
+def test_identical_keys_give_mean_of_values():
+    H, d, Lq, N = 1, 8, 7, 64 * 3
+    q, V = rnd((Lq, H, d), 22), rnd((N, H, d), 23)
+    K = rnd((N, H, d), 24)
+    K[64:128] = K[64]                       # block 1: identical keys
+    out = O.sparse_branch(q, K, V, [[np.array([1])]], N, False)
+    assert np.allclose(out[:, 0], V[64:128, 0].mean(axis=0)[None], atol=1e-13)
+    # causal, query in the middle of the block sees only the prefix
+    out = O.sparse_branch(q[:1], K, V, [[np.array([1])]], 64 + 9, True)
+    assert np.allclose(out[0, 0], V[64:64 + 10, 0].mean(axis=0), atol=1e-13)
+
+
+def test_zero_budget_gives_linear_only_and_empty_rows_zero():
+    H, d, Lq, N = 2, 8, 9, 130
+    q, K, V = rnd((Lq, H, d), 25), rnd((N, H, d), 26), rnd((N, H, d), 27)
+    sel, _ = O.select_blocks(q, K, N, False, [0, 0])
+    r = O.hsa_forward(q, K, V, N, False, sel)
+    assert np.array_equal(r["O_sp"], np.zeros_like(r["O_sp"]))
+    assert np.array_equal(r["out"], r["O_lin"])
+    # causal: a selected block lying wholly after a query contributes nothing to that row
+    out = O.sparse_branch(q, K, V, [[np.array([1])], [np.array([1])]], 0, True)
+    assert np.array_equal(out, np.zeros_like(out))      # positions 0..8 < 64
+    lin = O.linear_parallel(q, K, V, -5, True)
+    assert np.array_equal(lin[:5], np.zeros_like(lin[:5]))   # positions < 0 see nothing
+
+
+# ---------------------------------------------------------------- selection
+def test_selection_properties_and_planted_block():
+    H, d, Lq, N = 3, 16, 32, 64 * 20 + 13
+    q, K = rnd((Lq, H, d), 30), rnd((N, H, d), 31, 0.2)
+    qbar = q.mean(axis=0)
+    for h in range(H):
+        K[64 * 7:64 * 8, h] += 3.0 * qbar[h] / np.linalg.norm(qbar[h])   # planted block 7
+    budgets = [1, 5, 40]
+    sel, s = O.select_blocks(q, K, N, False, budgets)
+    nb = O.n_blocks(N)
+    assert nb == 21
+    for h in range(H):
+        ids = sel[h][0]
+        assert len(ids) == min(budgets[h], nb)
+        assert list(ids) == sorted(ids)
+        assert 7 in ids
+        assert int(np.argmax(s[h, 0])) == 7
+        rest = np.setdiff1d(np.arange(nb), ids)
+        if len(rest) and len(ids):
+            assert s[h, 0, ids].min() >= s[h, 0, rest].max()
+        # full fp64 sort done independently
+        ref = sorted(sorted(range(nb), key=lambda b: (-s[h, 0, b], b))[:budgets[h]])
+        assert list(ids) == ref
+
+
+def test_selection_ties_and_budget_edge_cases():
+    sc = np.array([1.0, 3.0, 3.0, 3.0, 0.5, 3.0])
+    cand = np.ones(6, bool)
+    assert list(O.select_topk(sc, cand, 2)) == [1, 2]          # lower index wins
+    assert list(O.select_topk(sc, cand, 4)) == [1, 2, 3, 5]
+    assert list(O.select_topk(sc, cand, 0)) == []
+    assert list(O.select_topk(sc, cand, -1)) == [0, 1, 2, 3, 4, 5]
+    assert list(O.select_topk(sc, cand, 99)) == [0, 1, 2, 3, 4, 5]
+    cand[1] = False
+    assert list(O.select_topk(sc, cand, 2)) == [2, 3]
+
+
+def test_candidates_under_causal_mask():
+    N = 64 * 5 + 3
+    assert O.candidate_mask(N, N, 10, False).sum() == 6
+    # last query position 130 -> blocks starting at 0, 64, 128
+    assert list(np.nonzero(O.candidate_mask(N, 100, 31, True))[0]) == [0, 1, 2]
+
+
+def test_scores_use_means_of_partial_block():
+    H, d, Lq, N = 1, 4, 3, 64 + 5
+    q, K = rnd((Lq, H, d), 32), rnd((N, H, d), 33)
+    s = O.block_scores(q, K)
+    ref = q.mean(axis=0)[0] @ K[64:, 0].mean(axis=0) / math.sqrt(d)
+    assert abs(s[0, 0, 1] - ref) < 1e-14
+
+
+def test_per_group_selection_layout():
+    H, d, Lq, N = 1, 8, 40, 64 * 6
+    q, K = rnd((Lq, H, d), 34), rnd((N, H, d), 35)
+    sel, s = O.select_blocks(q, K, N, False, [2], group_tokens=16)
+    assert s.shape == (1, 3, 6) and len(sel[0]) == 3
+    s0 = O.block_scores(q[16:32], K)
+    assert np.allclose(s[0, 1], s0[0, 0], atol=1e-14)
+
+
+# ---------------------------------------------------------------- merge
+def test_merge_linear_in_gates_and_single_branch_modes():
+    H, d, Lq = 2, 4, 6
+    a, b = rnd((Lq, H, d), 40), rnd((Lq, H, d), 41)
+    one, zero = np.ones((Lq, H)), np.zeros((Lq, H))
+    assert np.array_equal(O.merge(a, b, one, zero), a)
+    assert np.array_equal(O.merge(a, b, zero, one), b)
+    assert np.array_equal(O.merge(a, b), a + b)
+    g1, g2 = rnd((Lq, H), 42), rnd((Lq, H, d), 43)
+    assert np.allclose(O.merge(a, b, 2 * g1, g2), 2 * g1[..., None] * a + g2 * b)
+    sg = 1 / (1 + np.exp(-g1))
+    assert np.allclose(O.merge(a, b, g1, None, gate_act=1), sg[..., None] * a + b)
+
+
+# ---------------------------------------------------------------- Linformer form
+def test_linformer_identity_projection_is_dense_attention():
+    H, d, Lq, L_seg = 2, 8, 10, 32
+    N = 3 * L_seg
+    q, K, V = rnd((Lq, H, d), 50), rnd((N, H, d), 51), rnd((N, H, d), 52)
+    E = np.broadcast_to(np.eye(L_seg), (H, L_seg, L_seg))
+    Kt, Vt = O.linformer_compress(K, V, E, E, L_seg)
+    assert np.array_equal(Kt, K) and np.array_equal(Vt, V)
+    out = O.linformer_branch(q, Kt, Vt)
+    keysets = [[list(range(N)) for _ in range(Lq)] for _ in range(H)]
+    ref = np.array(brute.attention_rows(q, K, V, N, H, d, Lq, N, False, keysets))
+    assert np.abs(out - ref).max() < 1e-12
+
+
+def test_linformer_mean_projection_and_incremental():
+    H, d, L_seg, r = 2, 4, 16, 3
+    N = 2 * L_seg + 5                        # trailing incomplete segment is ignored
+    K, V = rnd((N, H, d), 53), rnd((N, H, d), 54)
+    E = np.full((H, L_seg, r), 1.0 / L_seg)
+    Kt, Vt = O.linformer_compress(K, V, E, E, L_seg)
+    assert Kt.shape == (2 * r, H, d)
+    assert np.allclose(Kt[0], K[:L_seg].mean(axis=0)) and np.allclose(Vt[r], V[L_seg:2 * L_seg].mean(axis=0))
+    E2 = rnd((H, L_seg, r), 55)
+    a, _ = O.linformer_compress(K, V, E2, E2, L_seg)
+    b, _ = O.linformer_compress(K[:L_seg], V[:L_seg], E2, E2, L_seg)
+    assert np.array_equal(a[:r], b)
+
+
+# ---------------------------------------------------------------- float32 carriers are widened
+def test_float32_inputs_are_computed_in_float64():
+    H, d, Lq, N = 2, 8, 12, 150
+    q = torch.randn(Lq, H, d).bfloat16().float().numpy()
+    K = torch.randn(N, H, d).bfloat16().float().numpy()
+    V = torch.randn(N, H, d).bfloat16().float().numpy()
+    sel32, s32 = O.select_blocks(q, K, N, False, [1, 2])
+    sel64, s64 = O.select_blocks(q.astype(np.float64), K.astype(np.float64), N, False, [1, 2])
+    assert np.array_equal(s32, s64)
+    a = O.hsa_forward(q, K, V, N, False, sel32)["out"]
+    b = O.hsa_forward(q.astype(np.float64), K.astype(np.float64), V.astype(np.float64), N, False, sel64)["out"]
+    assert a.dtype == np.float64 and np.array_equal(a, b)
