@@ -1,0 +1,173 @@
+/*
+ * hsa.h -- C ABI of the B200-native Hybrid Sparse Attention (HSA) forward path.
+ *
+ * One context (hsa_ctx) is one attention layer of one sequence (batch 1): a
+ * paged KV pool resident in HBM (the device tier of the Hierarchical KV Cache,
+ * Section 3.2), the per-block key sums used for block scoring, and the running
+ * state of the linear branch.  Per query chunk the caller does
+ *
+ *     hsa_append_kv      (new K/V of the chunk -> pool pages, key sums, state)
+ *     hsa_select_blocks  (pooled scores + per-head top-k, indices stay on device)
+ *     hsa_forward        (block-sparse softmax branch + linear branch + gated merge)
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA device addresses owned by the caller (allocated
+ *     with any allocator, e.g. torch); "host" pointers are ordinary host memory.
+ *     The library never allocates or frees device memory; a context owns only
+ *     host-side bookkeeping.  The caller frees its buffers after hsa_destroy.
+ *   - q / k / v / out are bf16 tensors indexed [token][head][dim] with explicit
+ *     token and head strides given in ELEMENTS; the dim stride is 1.  Base
+ *     addresses and byte strides must be multiples of 16.
+ *   - Every call only enqueues work on the given CUDA stream (a cudaStream_t
+ *     passed as void*; NULL = default stream) and returns; nothing synchronises
+ *     except hsa_device_status.  A context is not thread-safe.
+ *   - Return value: HSA_OK (0) or a negative hsa_status.  Device-side problems
+ *     (a bounded wait that ran out, an out-of-range block index) never trap:
+ *     the kernel records a code in a status word that hsa_device_status reads.
+ *   - History tokens form one continuous stream; block b holds tokens
+ *     [64 b, 64 b + 64); only the last block may be partial.  Query i of a chunk
+ *     sits at absolute position q_pos0 + i.  With causal != 0 key j is visible
+ *     to query i iff j <= q_pos0 + i (mask M of the attention definition,
+ *     Appendix A.1, Eq. 6).
+ */
+#ifndef HSA_H_
+#define HSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HSA_PAGE_TOKENS 64
+
+typedef enum {
+  HSA_OK = 0,
+  HSA_ERR_INVALID_ARG = -1,    /* null / misaligned pointer, size out of the configured range   */
+  HSA_ERR_OUT_OF_PAGES = -2,   /* append would exceed max_pages                                 */
+  HSA_ERR_UNSUPPORTED = -3,    /* valid request this build does not implement                   */
+  HSA_ERR_CUDA = -4,           /* a CUDA runtime / driver call failed (see hsa_last_cuda_error)  */
+  HSA_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired (status word)              */
+  HSA_ERR_DEVICE_BOUNDS = -6   /* a device-side index was out of range and was skipped          */
+} hsa_status;
+
+/* lin_mode */
+#define HSA_LIN_NONE 0
+#define HSA_LIN_STATE 1      /* running state S = sum phi(k)^T v, z = sum phi(k); phi = elu + 1 */
+#define HSA_LIN_LINFORMER 2  /* Section 3.3 "Linear branch" (Eq. 3); reserved, not built yet    */
+
+/* hsa_config.flags: reserve workspace for causal forwards with the linear branch on */
+#define HSA_CFG_CAUSAL 1u
+
+/* hsa_forward flags: the paper's "linear only" / "sparse only" ablation modes (Table 4) */
+#define HSA_FWD_NO_LINEAR 1u
+#define HSA_FWD_NO_SPARSE 2u
+
+typedef struct hsa_ctx hsa_ctx;
+
+typedef struct {
+  int32_t num_heads;      /* H >= 1                                                            */
+  int32_t head_dim;       /* 64 or 128                                                         */
+  int32_t page_tokens;    /* must be HSA_PAGE_TOKENS                                           */
+  int32_t max_pages;      /* pool capacity in pages (= KV blocks)                              */
+  int32_t max_q_tokens;   /* largest query chunk / appended chunk                              */
+  int32_t max_topk;       /* row capacity of sel_idx (blocks per head and query group)         */
+  int32_t lin_mode;       /* HSA_LIN_*                                                         */
+  int32_t gate_act;       /* 0: gates used as given; 1: sigmoid(gate) (Section 3.3, Eq. 5)     */
+  float softmax_scale;    /* 0 -> 1/sqrt(head_dim)                                             */
+  uint32_t flags;         /* HSA_CFG_* bits                                                    */
+} hsa_config;
+
+typedef struct {
+  size_t k_pool;     /* bytes: [max_pages][H][64][d] bf16                                      */
+  size_t v_pool;     /* same                                                                   */
+  size_t state;      /* linear-branch state + per-block key sums                               */
+  size_t workspace;  /* page table copy, partial sums, status word                             */
+} hsa_sizes;
+
+typedef struct {
+  void* k_pool;     /* device, 256-byte aligned                                                */
+  void* v_pool;     /* device, 256-byte aligned                                                */
+  void* state;      /* device, 256-byte aligned; zero-filled by hsa_create (synchronously)     */
+  void* workspace;  /* device, 256-byte aligned                                                */
+} hsa_buffers;
+
+/* Bytes the caller must allocate for a configuration.  Host only, no CUDA call. */
+int hsa_query_sizes(const hsa_config* cfg, hsa_sizes* out);
+
+/* Creates a context over caller-owned device buffers of at least hsa_query_sizes bytes.
+ * page_alloc_order_host: host int32[max_pages], a permutation of 0..max_pages-1 giving the
+ * physical page assigned to the b-th block of the history (NULL = identity).  The page table
+ * is copied to the workspace and the state is cleared, synchronously. */
+int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
+               const int32_t* page_alloc_order_host);
+
+/* Appends n_tokens (1..max_q_tokens) new history tokens:
+ * writes K/V rows into pool pages through the page table (continuing a partial tail
+ * page), updates the per-(head, block) key sums used by the pooled block scores
+ * (Section 3.3 "Sparse branch"; Section 3.2 Stage 2 "average key"), and the linear state
+ * S[h] += sum_j phi(k_j)^T v_j, z[h] += sum_j phi(k_j) (fp32), keeping the previous state
+ * for causal forwards.   k, v: device bf16 [n_tokens][H][d] with the given strides. */
+int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens,
+                  int64_t tok_stride, int64_t head_stride, void* stream);
+
+/* Pooled block scores s[h,g,b] = mean_q(group g) . mean_k(block b) * scale
+ * (Section 3.2 Stage 2 score form) and, per (head, group), the min(budget, candidates)
+ * highest-scoring candidate blocks; exact ties go to the lower block index.
+ *   budgets_dev      device int32[H]; < 0 or >= candidates selects every candidate.
+ *   q_group_tokens   0 = one selection for the whole chunk; otherwise a multiple of 128.
+ *   sel_idx_dev      device int32[H][n_groups][max_topk], ascending block ids (output).
+ *   sel_cnt_dev      device int32[H][n_groups] (output).
+ * Candidates: blocks with at least one token and, if causal, first token <= last query
+ * position of the group.  Counts are clamped to max_topk (flagged in the status word). */
+int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
+                      int64_t head_stride, int64_t q_pos0, int32_t causal,
+                      const int32_t* budgets_dev, int32_t q_group_tokens,
+                      int32_t* sel_idx_dev, int32_t* sel_cnt_dev, void* stream);
+
+/* out[i,h,:] = w(g_lin) * O_lin + w(g_sp) * O_sp  (Section 3.3, Eq. 5), where
+ *   O_sp  = softmax attention of query i over the visible keys of the selected blocks
+ *           (Eq. 4 with the block mask; Appendix A.1),
+ *   O_lin = phi(q_i) S / (phi(q_i) z) over all visible history (running-state form),
+ *   w(g)  = 1 if the gate pointer is NULL, else g or sigmoid(g) per gate_act.
+ * A branch with nothing visible contributes 0.  sel_idx_dev / sel_cnt_dev may come from
+ * hsa_select_blocks or from the caller (same layout).  Gates: device bf16 with element
+ * strides (token, head, dim); dim stride 0 broadcasts one gate per (token, head).
+ * causal != 0 with the linear branch on requires HSA_CFG_CAUSAL and the query chunk to be the
+ * most recently appended chunk (q_pos0 + n_q == tokens appended so far, n_q == size of the
+ * last append), otherwise HSA_ERR_UNSUPPORTED; the sparse branch alone takes any q_pos0.  out: device bf16 [n_q][H][d], strides as q. */
+int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                int64_t q_pos0, int32_t causal, const int32_t* sel_idx_dev,
+                const int32_t* sel_cnt_dev, int32_t q_group_tokens, const void* g_lin,
+                const void* g_sp, int64_t gate_tok_stride, int64_t gate_head_stride,
+                int64_t gate_dim_stride, void* out, int64_t out_tok_stride,
+                int64_t out_head_stride, uint32_t flags, void* stream);
+
+/* Host-tracked length of the history. */
+int hsa_get_info(hsa_ctx* ctx, int64_t* n_tokens, int32_t* n_blocks);
+
+/* Sets the history length back to n_tokens (<= current).  The pool keeps its pages, but the
+ * key sums of the new tail block and the linear state are NOT recomputed: the caller must
+ * restore the state buffer to the contents it had at that length (used by benchmarks that
+ * replay the same append). */
+int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens);
+
+/* Byte offsets inside the state buffer, for tests and snapshots:
+ * S fp32 [H][d][d], z fp32 [H][d], key sums fp32 [H][max_pages][d]. */
+int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksum);
+
+/* Synchronises the device, reads and clears the status word: HSA_OK or a DEVICE_* code. */
+int hsa_device_status(hsa_ctx* ctx, int32_t* status_out);
+
+/* Last CUDA error code recorded by a failing call on this context (0 if none). */
+int hsa_last_cuda_error(hsa_ctx* ctx);
+
+int hsa_destroy(hsa_ctx* ctx);
+
+const char* hsa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HSA_H_ */

@@ -1,0 +1,437 @@
+// C-ABI layer: context bookkeeping, argument validation, tensor maps and kernel launches.
+// The library owns no device memory; every device buffer comes from the caller.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "hsa_internal.h"
+
+using namespace hsa;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  // state
+  size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
+  // workspace
+  size_t status, page_table, qpart, spart, lin_num, lin_den, ws_total;
+};
+
+bool config_ok(const hsa_config* c) {
+  if (!c) return false;
+  if (c->num_heads < 1 || c->num_heads > 1024) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->page_tokens != HSA_PAGE_TOKENS) return false;
+  if (c->max_pages < 1 || c->max_q_tokens < 1 || c->max_topk < 1) return false;
+  if (static_cast<int64_t>(c->max_pages) * c->num_heads * kBlock >= (1ll << 31)) return false;
+  if (c->lin_mode != HSA_LIN_NONE && c->lin_mode != HSA_LIN_STATE) return false;
+  if (c->gate_act != 0 && c->gate_act != 1) return false;
+  if (!(c->softmax_scale >= 0.f)) return false;
+  return true;
+}
+
+Layout make_layout(const hsa_config* c) {
+  Layout L{};
+  const size_t H = c->num_heads, D = c->head_dim, P = c->max_pages;
+  size_t o = 0;
+  L.S = o;      o = align_up(o + H * D * D * 4, 1024);
+  L.z = o;      o = align_up(o + H * D * 4, 1024);
+  L.S_prev = o; o = align_up(o + H * D * D * 4, 1024);
+  L.z_prev = o; o = align_up(o + H * D * 4, 1024);
+  L.hilo = o;   o = align_up(o + H * 4 * D * D * 2, 1024);
+  L.ksum = o;   o = align_up(o + H * P * D * 4, 1024);
+  L.state_total = o;
+  const size_t tiles = (static_cast<size_t>(c->max_q_tokens) + kTileM - 1) / kTileM;
+  o = 0;
+  L.status = o;     o = align_up(o + 16, 256);
+  L.page_table = o; o = align_up(o + P * 4, 256);
+  L.qpart = o;      o = align_up(o + tiles * H * D * 4, 256);
+  L.spart = o;      o = align_up(o + H * kStateSplitMax * (D * D + D) * 4, 256);
+  if (c->flags & HSA_CFG_CAUSAL) {
+    L.lin_num = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 4, 256);
+    L.lin_den = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * 4, 256);
+  }
+  L.ws_total = o;
+  return L;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+struct hsa_ctx {
+  hsa_config cfg;
+  hsa_buffers buf;
+  Layout lay;
+  float scale;
+  int64_t n_tokens;
+  int32_t last_append;  // tokens of the most recent append (0 after a rewind)
+  int nsm;
+  CUtensorMap tm_k, tm_v, tm_state;
+  int last_cuda_error;
+};
+
+namespace {
+
+int cuda_fail(hsa_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda_error = static_cast<int>(e);
+  return HSA_ERR_CUDA;
+}
+
+int encode_2d_rows(CUtensorMap* tm, void* base, uint64_t rows, int D) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return HSA_ERR_CUDA;
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(D), rows};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(D) * 2};
+  cuuint32_t box[2] = {64, 64};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HSA_OK : HSA_ERR_CUDA;
+}
+
+int encode_q(CUtensorMap* tm, const void* q, int n_q, int H, int D, int64_t ts, int64_t hs) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return HSA_ERR_CUDA;
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(H),
+                        static_cast<cuuint64_t>(n_q)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(hs) * 2, static_cast<cuuint64_t>(ts) * 2};
+  cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(kTileM)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HSA_OK : HSA_ERR_CUDA;
+}
+
+bool tensor_args_ok(const hsa_ctx* ctx, const void* p, int64_t ts, int64_t hs) {
+  const int D = ctx->cfg.head_dim, H = ctx->cfg.num_heads;
+  if (!p || !aligned(p, 16)) return false;
+  if (ts <= 0 || hs <= 0 || (ts % 8) != 0 || (hs % 8) != 0) return false;
+  if (hs < D || ts < D) return false;
+  (void)H;
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hsa_query_sizes(const hsa_config* cfg, hsa_sizes* out) {
+  if (!config_ok(cfg) || !out) return HSA_ERR_INVALID_ARG;
+  const Layout L = make_layout(cfg);
+  const size_t pool = static_cast<size_t>(cfg->max_pages) * cfg->num_heads * kBlock * cfg->head_dim * 2;
+  out->k_pool = pool;
+  out->v_pool = pool;
+  out->state = L.state_total;
+  out->workspace = L.ws_total;
+  return HSA_OK;
+}
+
+int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
+               const int32_t* page_alloc_order_host) {
+  if (!out) return HSA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg) || !bufs) return HSA_ERR_INVALID_ARG;
+  if (!bufs->k_pool || !bufs->v_pool || !bufs->state || !bufs->workspace) return HSA_ERR_INVALID_ARG;
+  if (!aligned(bufs->k_pool, 256) || !aligned(bufs->v_pool, 256) || !aligned(bufs->state, 256) ||
+      !aligned(bufs->workspace, 256))
+    return HSA_ERR_INVALID_ARG;
+  std::vector<int32_t> pt(cfg->max_pages);
+  if (page_alloc_order_host) {
+    std::vector<char> seen(cfg->max_pages, 0);
+    for (int i = 0; i < cfg->max_pages; ++i) {
+      const int32_t v = page_alloc_order_host[i];
+      if (v < 0 || v >= cfg->max_pages || seen[v]) return HSA_ERR_INVALID_ARG;  // not a permutation
+      seen[v] = 1;
+      pt[i] = v;
+    }
+  } else {
+    for (int i = 0; i < cfg->max_pages; ++i) pt[i] = i;
+  }
+  hsa_ctx* ctx = new (std::nothrow) hsa_ctx();
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  ctx->cfg = *cfg;
+  ctx->buf = *bufs;
+  ctx->lay = make_layout(cfg);
+  ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale
+                                        : 1.0f / std::sqrt(static_cast<float>(cfg->head_dim));
+  ctx->n_tokens = 0;
+  ctx->last_append = 0;
+  ctx->last_cuda_error = 0;
+
+  cudaError_t e;
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) { delete ctx; return HSA_ERR_CUDA; }
+  int cc_major = 0;
+  cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+  cudaDeviceGetAttribute(&ctx->nsm, cudaDevAttrMultiProcessorCount, dev);
+  if (cc_major != 10) { delete ctx; return HSA_ERR_UNSUPPORTED; }  // sm_100a only, no fallback
+  uint8_t* ws = static_cast<uint8_t*>(bufs->workspace);
+  e = cudaMemcpy(ws + ctx->lay.page_table, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(ws + ctx->lay.status, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(bufs->state, 0, ctx->lay.state_total);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = forward_init();
+  if (e != cudaSuccess) { delete ctx; return HSA_ERR_CUDA; }
+  const int D = cfg->head_dim;
+  const uint64_t pool_rows = static_cast<uint64_t>(cfg->max_pages) * cfg->num_heads * kBlock;
+  int r = encode_2d_rows(&ctx->tm_k, bufs->k_pool, pool_rows, D);
+  if (r == HSA_OK) r = encode_2d_rows(&ctx->tm_v, bufs->v_pool, pool_rows, D);
+  if (r == HSA_OK)
+    r = encode_2d_rows(&ctx->tm_state, static_cast<uint8_t*>(bufs->state) + ctx->lay.hilo,
+                       static_cast<uint64_t>(cfg->num_heads) * 4 * D, D);
+  if (r != HSA_OK) { delete ctx; return r; }
+  *out = ctx;
+  return HSA_OK;
+}
+
+int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, int64_t tok_stride,
+                  int64_t head_stride, void* stream) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (n_tokens < 1 || n_tokens > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, k, tok_stride, head_stride) || !tensor_args_ok(ctx, v, tok_stride, head_stride))
+    return HSA_ERR_INVALID_ARG;
+  const int64_t n1 = ctx->n_tokens + n_tokens;
+  if ((n1 + kBlock - 1) / kBlock > ctx->cfg.max_pages) return HSA_ERR_OUT_OF_PAGES;
+  uint8_t* stt = static_cast<uint8_t*>(ctx->buf.state);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  AppendArgs a{};
+  a.k = static_cast<const __nv_bfloat16*>(k);
+  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.n_new = n_tokens;
+  a.tok_stride = tok_stride;
+  a.head_stride = head_stride;
+  a.n0 = ctx->n_tokens;
+  a.H = ctx->cfg.num_heads;
+  a.D = ctx->cfg.head_dim;
+  a.max_pages = ctx->cfg.max_pages;
+  a.page_table = reinterpret_cast<const int32_t*>(ws + ctx->lay.page_table);
+  a.k_pool = static_cast<__nv_bfloat16*>(ctx->buf.k_pool);
+  a.v_pool = static_cast<__nv_bfloat16*>(ctx->buf.v_pool);
+  a.ksum = reinterpret_cast<float*>(stt + ctx->lay.ksum);
+  a.S = reinterpret_cast<float*>(stt + ctx->lay.S);
+  a.z = reinterpret_cast<float*>(stt + ctx->lay.z);
+  a.S_prev = reinterpret_cast<float*>(stt + ctx->lay.S_prev);
+  a.z_prev = reinterpret_cast<float*>(stt + ctx->lay.z_prev);
+  a.hilo = reinterpret_cast<__nv_bfloat16*>(stt + ctx->lay.hilo);
+  a.spart = reinterpret_cast<float*>(ws + ctx->lay.spart);
+  int nsplit = ctx->nsm / a.H;
+  if (nsplit < 1) nsplit = 1;
+  if (nsplit > kStateSplitMax) nsplit = kStateSplitMax;
+  const int by_tokens = (n_tokens + 31) / 32;
+  if (nsplit > by_tokens) nsplit = by_tokens;
+  a.nsplit = nsplit;
+  a.lin_state = ctx->cfg.lin_mode == HSA_LIN_STATE;
+  cudaError_t e = launch_append(a, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  ctx->n_tokens = n1;
+  ctx->last_append = n_tokens;
+  return HSA_OK;
+}
+
+int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                      int64_t q_pos0, int32_t causal, const int32_t* budgets_dev,
+                      int32_t q_group_tokens, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
+                      void* stream) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (n_q < 1 || n_q > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, q, tok_stride, head_stride)) return HSA_ERR_INVALID_ARG;
+  if (!budgets_dev || !sel_idx_dev || !sel_cnt_dev) return HSA_ERR_INVALID_ARG;
+  if (q_group_tokens < 0 || (q_group_tokens % kTileM) != 0) return HSA_ERR_INVALID_ARG;
+  const int64_t nblk = (ctx->n_tokens + kBlock - 1) / kBlock;
+  if (nblk * 4 > 200 * 1024) return HSA_ERR_UNSUPPORTED;  // keys of one head must fit shared memory
+  uint8_t* stt = static_cast<uint8_t*>(ctx->buf.state);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  SelectArgs a{};
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.n_q = n_q;
+  a.tok_stride = tok_stride;
+  a.head_stride = head_stride;
+  a.q_pos0 = q_pos0;
+  a.causal = causal != 0;
+  a.n_tokens = ctx->n_tokens;
+  a.H = ctx->cfg.num_heads;
+  a.D = ctx->cfg.head_dim;
+  a.max_pages = ctx->cfg.max_pages;
+  a.ksum = reinterpret_cast<const float*>(stt + ctx->lay.ksum);
+  a.budgets = budgets_dev;
+  a.group_tokens = q_group_tokens;
+  a.n_groups = q_group_tokens > 0 ? (n_q + q_group_tokens - 1) / q_group_tokens : 1;
+  a.scale = ctx->scale;
+  a.qpart = reinterpret_cast<float*>(ws + ctx->lay.qpart);
+  a.sel_idx = sel_idx_dev;
+  a.sel_cnt = sel_cnt_dev;
+  a.kcap = ctx->cfg.max_topk;
+  a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  cudaError_t e = launch_select(a, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return HSA_OK;
+}
+
+int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                int64_t q_pos0, int32_t causal, const int32_t* sel_idx_dev, const int32_t* sel_cnt_dev,
+                int32_t q_group_tokens, const void* g_lin, const void* g_sp, int64_t gate_tok_stride,
+                int64_t gate_head_stride, int64_t gate_dim_stride, void* out, int64_t out_tok_stride,
+                int64_t out_head_stride, uint32_t flags, void* stream) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (n_q < 1 || n_q > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, q, tok_stride, head_stride)) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, out, out_tok_stride, out_head_stride)) return HSA_ERR_INVALID_ARG;
+  if (q_group_tokens < 0 || (q_group_tokens % kTileM) != 0) return HSA_ERR_INVALID_ARG;
+  if (flags & ~(HSA_FWD_NO_LINEAR | HSA_FWD_NO_SPARSE)) return HSA_ERR_INVALID_ARG;
+  const bool do_sparse = !(flags & HSA_FWD_NO_SPARSE);
+  const bool do_linear = !(flags & HSA_FWD_NO_LINEAR) && ctx->cfg.lin_mode == HSA_LIN_STATE;
+  if (do_sparse && (!sel_idx_dev || !sel_cnt_dev)) return HSA_ERR_INVALID_ARG;
+  if ((g_lin || g_sp) && (gate_tok_stride < 0 || gate_head_stride < 0 || gate_dim_stride < 0))
+    return HSA_ERR_INVALID_ARG;
+  const bool causal_lin = causal && do_linear;
+  if (causal_lin) {
+    if (!(ctx->cfg.flags & HSA_CFG_CAUSAL)) return HSA_ERR_UNSUPPORTED;
+    if (q_pos0 + n_q != ctx->n_tokens || n_q != ctx->last_append) return HSA_ERR_UNSUPPORTED;
+  }
+  const int D = ctx->cfg.head_dim, H = ctx->cfg.num_heads;
+  uint8_t* stt = static_cast<uint8_t*>(ctx->buf.state);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  CUtensorMap tm_q;
+  int r = encode_q(&tm_q, q, n_q, H, D, tok_stride, head_stride);
+  if (r != HSA_OK) return r;
+
+  FwdParams p{};
+  p.n_q = n_q;
+  p.H = H;
+  p.n_tokens = ctx->n_tokens;
+  p.q_pos0 = q_pos0;
+  p.causal = causal != 0;
+  p.sel_idx = sel_idx_dev;
+  p.sel_cnt = sel_cnt_dev;
+  p.kcap = ctx->cfg.max_topk;
+  p.group_tokens = q_group_tokens;
+  p.n_groups = q_group_tokens > 0 ? (n_q + q_group_tokens - 1) / q_group_tokens : 1;
+  p.page_table = reinterpret_cast<const int32_t*>(ws + ctx->lay.page_table);
+  p.n_blocks = static_cast<int>((ctx->n_tokens + kBlock - 1) / kBlock);
+  p.use_prev = causal_lin ? 1 : 0;
+  p.z = reinterpret_cast<const float*>(stt + (causal_lin ? ctx->lay.z_prev : ctx->lay.z));
+  p.g_lin = static_cast<const __nv_bfloat16*>(g_lin);
+  p.g_sp = static_cast<const __nv_bfloat16*>(g_sp);
+  p.g_ts = gate_tok_stride;
+  p.g_hs = gate_head_stride;
+  p.g_ds = gate_dim_stride;
+  p.gate_act = ctx->cfg.gate_act;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.o_ts = out_tok_stride;
+  p.o_hs = out_head_stride;
+  p.scale_log2 = ctx->scale * 1.4426950408889634f;
+  p.flags = flags;
+  p.do_linear = do_linear;
+  p.do_sparse = do_sparse;
+  p.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  if (causal_lin) {
+    CausalLinArgs c{};
+    c.q = static_cast<const __nv_bfloat16*>(q);
+    c.n_q = n_q;
+    c.q_ts = tok_stride;
+    c.q_hs = head_stride;
+    c.k_pool = static_cast<const __nv_bfloat16*>(ctx->buf.k_pool);
+    c.v_pool = static_cast<const __nv_bfloat16*>(ctx->buf.v_pool);
+    c.page_table = p.page_table;
+    c.q_pos0 = q_pos0;
+    c.n_tokens = ctx->n_tokens;
+    c.H = H;
+    c.D = D;
+    c.lin_num = reinterpret_cast<float*>(ws + ctx->lay.lin_num);
+    c.lin_den = reinterpret_cast<float*>(ws + ctx->lay.lin_den);
+    cudaError_t e = launch_causal_linear(c, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    p.lin_num = c.lin_num;
+    p.lin_den = c.lin_den;
+  }
+  cudaError_t e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return HSA_OK;
+}
+
+int hsa_get_info(hsa_ctx* ctx, int64_t* n_tokens, int32_t* n_blocks) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (n_tokens) *n_tokens = ctx->n_tokens;
+  if (n_blocks) *n_blocks = static_cast<int32_t>((ctx->n_tokens + kBlock - 1) / kBlock);
+  return HSA_OK;
+}
+
+int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens) {
+  if (!ctx || n_tokens < 0 || n_tokens > ctx->n_tokens) return HSA_ERR_INVALID_ARG;
+  ctx->n_tokens = n_tokens;
+  ctx->last_append = 0;
+  return HSA_OK;
+}
+
+int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksum) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (off_S) *off_S = ctx->lay.S;
+  if (off_z) *off_z = ctx->lay.z;
+  if (off_ksum) *off_ksum = ctx->lay.ksum;
+  return HSA_OK;
+}
+
+int hsa_device_status(hsa_ctx* ctx, int32_t* status_out) {
+  if (!ctx || !status_out) return HSA_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  int32_t v = 0;
+  e = cudaMemcpy(&v, ws + ctx->lay.status, 4, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && v != 0) e = cudaMemset(ws + ctx->lay.status, 0, 4);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  *status_out = v;
+  return HSA_OK;
+}
+
+int hsa_last_cuda_error(hsa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int hsa_destroy(hsa_ctx* ctx) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  delete ctx;
+  return HSA_OK;
+}
+
+const char* hsa_status_string(int s) {
+  switch (s) {
+    case HSA_OK: return "ok";
+    case HSA_ERR_INVALID_ARG: return "invalid argument";
+    case HSA_ERR_OUT_OF_PAGES: return "out of pages";
+    case HSA_ERR_UNSUPPORTED: return "unsupported";
+    case HSA_ERR_CUDA: return "CUDA error";
+    case HSA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case HSA_ERR_DEVICE_BOUNDS: return "device-side index out of range";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

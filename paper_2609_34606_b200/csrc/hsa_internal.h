@@ -1,0 +1,111 @@
+// Internal declarations shared by the C-ABI layer and the kernel launchers.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/hsa.h"
+
+namespace hsa {
+
+constexpr int kBlock = HSA_PAGE_TOKENS;  // tokens per KV block = tokens per page
+constexpr int kTileM = 128;              // query rows per work item of the forward kernel
+constexpr int kStateSplitMax = 16;       // token-axis splits of the state update (per head)
+
+__host__ __device__ inline int64_t min64(int64_t a, int64_t b) { return a < b ? a : b; }
+__host__ __device__ inline int64_t max64(int64_t a, int64_t b) { return a > b ? a : b; }
+
+// device status word values (match hsa_status)
+constexpr int kDevTimeout = HSA_ERR_DEVICE_TIMEOUT;
+constexpr int kDevBounds = HSA_ERR_DEVICE_BOUNDS;
+
+struct AppendArgs {
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  int n_new;
+  int64_t tok_stride, head_stride;
+  int64_t n0;  // tokens already in the history
+  int H, D, max_pages;
+  const int32_t* page_table;
+  __nv_bfloat16* k_pool;
+  __nv_bfloat16* v_pool;
+  float* ksum;      // [H][max_pages][D]
+  float* S;         // [H][D][D]
+  float* z;         // [H][D]
+  float* S_prev;    // state before this append
+  float* z_prev;
+  __nv_bfloat16* hilo;  // [H][2 cur/prev][2 hi/lo][D][D]
+  float* spart;         // [H][nsplit][D*D + D] scratch
+  int nsplit;
+  int lin_state;  // update the linear state?
+};
+
+struct SelectArgs {
+  const __nv_bfloat16* q;
+  int n_q;
+  int64_t tok_stride, head_stride;
+  int64_t q_pos0;
+  int causal;
+  int64_t n_tokens;
+  int H, D, max_pages;
+  const float* ksum;
+  const int32_t* budgets;
+  int group_tokens, n_groups;
+  float scale;
+  float* qpart;  // [n_tiles][H][D] scratch
+  int32_t* sel_idx;
+  int32_t* sel_cnt;
+  int kcap;
+  int32_t* status;
+};
+
+struct FwdParams {
+  int n_q, H;
+  int64_t n_tokens;
+  int64_t q_pos0;
+  int causal;
+  const int32_t* sel_idx;
+  const int32_t* sel_cnt;
+  int kcap, n_groups, group_tokens;
+  const int32_t* page_table;
+  int n_blocks;
+  const float* z;       // [H][D] state the linear branch applies
+  int state_row0_mul;   // row of the hi/lo state tensor map = ((h*2 + use_prev)*2 + hl)*D
+  int use_prev;
+  const __nv_bfloat16* g_lin;
+  const __nv_bfloat16* g_sp;
+  int64_t g_ts, g_hs, g_ds;
+  int gate_act;
+  __nv_bfloat16* out;
+  int64_t o_ts, o_hs;
+  float scale_log2;  // softmax scale * log2(e)
+  uint32_t flags;
+  int do_linear, do_sparse;
+  const float* lin_num;  // causal intra-chunk partials [n_q][H][D] (or null)
+  const float* lin_den;  // [n_q][H]
+  int32_t* status;
+};
+
+struct CausalLinArgs {
+  const __nv_bfloat16* q;
+  int n_q;
+  int64_t q_ts, q_hs;
+  const __nv_bfloat16* k_pool;
+  const __nv_bfloat16* v_pool;
+  const int32_t* page_table;
+  int64_t q_pos0;   // first query position == first token of the intra-chunk part
+  int64_t n_tokens;
+  int H, D;
+  float* lin_num;
+  float* lin_den;
+};
+
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
+                           const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                           const CUtensorMap& tm_state, cudaStream_t st);
+cudaError_t launch_causal_linear(const CausalLinArgs& a, cudaStream_t st);
+cudaError_t forward_init();  // opt in to the shared-memory size the forward kernel needs
+
+}  // namespace hsa

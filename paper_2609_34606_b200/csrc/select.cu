@@ -1,0 +1,236 @@
+// hsa_select_blocks kernels: mean query per group, pooled block scores
+//   s[h,g,b] = mean_q(g) . (Ksum[h,b] / cnt_b) * scale
+// and an exact per-(head, group) top-k by radix select, all on the device.
+#include <cuda_bf16.h>
+
+#include "hsa_internal.h"
+
+namespace hsa {
+
+// ---------------------------------------------------------------------------------------
+// Stage 1: column sums of q over one 128-token tile and one head -> qpart[tile][h][D].
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
+  constexpr int CH = D / 8;
+  constexpr int RP = 256 / CH;
+  __shared__ float red[RP][D];
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int c8 = threadIdx.x % CH, rg = threadIdx.x / CH;
+  const int t_hi = min(a.n_q, tile * kTileM + kTileM);
+  float acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+  for (int t = tile * kTileM + rg; t < t_hi; t += RP) {
+    const size_t src =
+        static_cast<size_t>(t) * a.tok_stride + static_cast<size_t>(h) * a.head_stride + c8 * 8;
+    const uint4 qq = *reinterpret_cast<const uint4*>(a.q + src);
+    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qq);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(q2[i]);
+      acc[2 * i] += f.x;
+      acc[2 * i + 1] += f.y;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) red[rg][c8 * 8 + i] = acc[i];
+  __syncthreads();
+  if (threadIdx.x < D) {
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < RP; ++r) s += red[r][threadIdx.x];
+    a.qpart[(static_cast<size_t>(tile) * a.H + h) * D + threadIdx.x] = s;
+  }
+}
+
+__device__ __forceinline__ uint32_t order_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // ascending with the float order
+}
+
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+  // 256 threads; returns the exclusive prefix of v over threadIdx.x and the block total
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  __syncthreads();
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) {
+    const int s = warp_sums[w];
+    if (w < warp) base += s;
+    tot += s;
+  }
+  *total = tot;
+  return base + incl - v;
+}
+
+// ---------------------------------------------------------------------------------------
+// Stage 2: one CTA per (group, head): scores for every block, k-th largest by a 4-pass
+// 8-bit radix select on order-preserving keys, then an index-ordered compaction.
+// Exact ties at the threshold go to the lower block index.
+// dynamic smem: uint32 keys[nblk]
+// ---------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) score_select_kernel(SelectArgs a) {
+  extern __shared__ uint32_t keys[];
+  __shared__ double qs[D];
+  __shared__ int hist[256];
+  __shared__ int warp_sums[8];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_krem;
+
+  const int g = blockIdx.x, h = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
+  const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
+  const int64_t p_last = a.q_pos0 + q_hi - 1;
+  // candidate blocks are a prefix [0, ncand)
+  int64_t ncand64 = nblk;
+  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
+  const int ncand = static_cast<int>(ncand64);
+
+  // mean query of the group (fp64 over the tile partials, fixed order), pre-scaled
+  if (threadIdx.x < D) {
+    double s = 0.0;
+    const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
+    for (int t = tile_lo; t < tile_hi; ++t)
+      s += static_cast<double>(a.qpart[(static_cast<size_t>(t) * a.H + h) * D + threadIdx.x]);
+    qs[threadIdx.x] = s / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
+  }
+  __syncthreads();
+
+  // scores
+  constexpr int PER = D / 32;
+  for (int b = warp; b < ncand; b += 8) {
+    const float* ks = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER;
+    double dot = 0.0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) dot += qs[lane * PER + i] * static_cast<double>(ks[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (lane == 0) {
+      const int64_t cnt = min64(kBlock, a.n_tokens - static_cast<int64_t>(b) * kBlock);
+      keys[b] = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
+    }
+  }
+  __syncthreads();
+
+  int budget = a.budgets[h];
+  if (budget < 0 || budget > ncand) budget = ncand;
+  const bool take_all = (budget >= ncand);
+  uint32_t thr = 0;
+  int need_ties = 0;
+  if (!take_all && budget > 0) {
+    if (threadIdx.x == 0) {
+      sh_prefix = 0;
+      sh_krem = budget;
+    }
+    uint32_t mask = 0;
+    for (int pass = 3; pass >= 0; --pass) {
+      const int shift = pass * 8;
+      hist[threadIdx.x] = 0;
+      __syncthreads();
+      const uint32_t prefix = sh_prefix;
+      for (int b = threadIdx.x; b < ncand; b += 256) {
+        const uint32_t k = keys[b];
+        if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        int krem = sh_krem, cum = 0, bin = 255;
+        for (; bin > 0; --bin) {
+          if (cum + hist[bin] >= krem) break;
+          cum += hist[bin];
+        }
+        sh_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+        sh_krem = krem - cum;  // still to take among keys matching the longer prefix
+      }
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+    thr = sh_prefix;
+    need_ties = sh_krem;
+  }
+
+  // index-ordered compaction: thread t owns the contiguous range [t*per, t*per+per)
+  const int per = (ncand + 255) / 256;
+  const int lo = min(ncand, static_cast<int>(threadIdx.x) * per), hi = min(ncand, lo + per);
+  int ties_before = 0, dummy;
+  if (!take_all && budget > 0) {
+    int my_ties = 0;
+    for (int b = lo; b < hi; ++b) my_ties += (keys[b] == thr);
+    ties_before = block_exclusive_scan(my_ties, warp_sums, &dummy);
+  }
+  int my_sel = 0;
+  if (take_all) {
+    my_sel = hi - lo;
+  } else if (budget > 0) {
+    int t = ties_before;
+    for (int b = lo; b < hi; ++b) {
+      const uint32_t k = keys[b];
+      if (k > thr) ++my_sel;
+      else if (k == thr) { if (t < need_ties) ++my_sel; ++t; }
+    }
+  }
+  int total = 0;
+  int pos = block_exclusive_scan(my_sel, warp_sums, &total);
+  int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
+  {
+    int t = ties_before;
+    for (int b = lo; b < hi; ++b) {
+      bool sel;
+      if (take_all) sel = true;
+      else if (budget == 0) sel = false;
+      else {
+        const uint32_t k = keys[b];
+        sel = (k > thr);
+        if (k == thr) { sel = (t < need_ties); ++t; }
+      }
+      if (sel) {
+        if (pos < a.kcap) out[pos] = b;
+        ++pos;
+      }
+    }
+  }
+  if (threadIdx.x == 0) {
+    a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
+    if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
+  }
+}
+
+cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  dim3 g1(n_tiles, a.H);
+  if (a.D == 128)
+    qsum_partial_kernel<128><<<g1, 256, 0, st>>>(a);
+  else
+    qsum_partial_kernel<64><<<g1, 256, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const size_t smem = static_cast<size_t>(nblk > 0 ? nblk : 1) * sizeof(uint32_t);
+  dim3 g2(a.n_groups, a.H);
+  if (a.D == 128) {
+    if (smem > 40 * 1024)
+      cudaFuncSetAttribute(score_select_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(smem));
+    score_select_kernel<128><<<g2, 256, smem, st>>>(a);
+  } else {
+    if (smem > 40 * 1024)
+      cudaFuncSetAttribute(score_select_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(smem));
+    score_select_kernel<64><<<g2, 256, smem, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace hsa

@@ -1,0 +1,298 @@
+"""Thin Python binding over the HSA C-ABI library (libhsa.so).
+
+Argument marshalling only: every step of the path (pool write, key sums, state
+update, block scoring, top-k, both attention branches, the merge) runs in the
+library's CUDA kernels.  torch is used for device memory and streams.  There is
+no fallback: if libhsa.so is missing or fails to load, importing this module
+raises.
+
+The module-level functions carry the C names (hsa_create, hsa_append_kv,
+hsa_select_blocks, hsa_forward, ...) and take torch tensors where the C ABI
+takes device pointers; `HSAContext` bundles buffer allocation with them.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libhsa.so")
+
+HSA_OK = 0
+HSA_ERR_INVALID_ARG = -1
+HSA_ERR_OUT_OF_PAGES = -2
+HSA_ERR_UNSUPPORTED = -3
+HSA_ERR_CUDA = -4
+HSA_ERR_DEVICE_TIMEOUT = -5
+HSA_ERR_DEVICE_BOUNDS = -6
+HSA_LIN_NONE, HSA_LIN_STATE = 0, 1
+HSA_CFG_CAUSAL = 1
+HSA_FWD_NO_LINEAR, HSA_FWD_NO_SPARSE = 1, 2
+PAGE_TOKENS = 64
+TILE_M = 128
+
+EXPORTS = [
+    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_forward",
+    "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_last_cuda_error",
+    "hsa_destroy", "hsa_status_string",
+]
+
+
+class hsa_config(C.Structure):
+    _fields_ = [("num_heads", C.c_int32), ("head_dim", C.c_int32), ("page_tokens", C.c_int32),
+                ("max_pages", C.c_int32), ("max_q_tokens", C.c_int32), ("max_topk", C.c_int32),
+                ("lin_mode", C.c_int32), ("gate_act", C.c_int32), ("softmax_scale", C.c_float),
+                ("flags", C.c_uint32)]
+
+
+class hsa_sizes(C.Structure):
+    _fields_ = [("k_pool", C.c_size_t), ("v_pool", C.c_size_t), ("state", C.c_size_t),
+                ("workspace", C.c_size_t)]
+
+
+class hsa_buffers(C.Structure):
+    _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("state", C.c_void_p),
+                ("workspace", C.c_void_p)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2609_34606_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32
+    lib.hsa_query_sizes.argtypes = [C.POINTER(hsa_config), C.POINTER(hsa_sizes)]
+    lib.hsa_create.argtypes = [C.POINTER(vp), C.POINTER(hsa_config), C.POINTER(hsa_buffers), vp]
+    lib.hsa_append_kv.argtypes = [vp, vp, vp, i32, i64, i64, vp]
+    lib.hsa_select_blocks.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp, vp]
+    lib.hsa_forward.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, vp, i32, vp, vp, i64, i64, i64,
+                                vp, i64, i64, u32, vp]
+    lib.hsa_get_info.argtypes = [vp, C.POINTER(i64), C.POINTER(i32)]
+    lib.hsa_rewind.argtypes = [vp, i64]
+    lib.hsa_state_layout.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t),
+                                     C.POINTER(C.c_size_t)]
+    lib.hsa_device_status.argtypes = [vp, C.POINTER(i32)]
+    lib.hsa_last_cuda_error.argtypes = [vp]
+    lib.hsa_destroy.argtypes = [vp]
+    lib.hsa_status_string.argtypes = [C.c_int]
+    lib.hsa_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "hsa_status_string":
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+_lib = _load()
+
+
+class HSAError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {hsa_status_string(code)} ({code})")
+
+
+def hsa_status_string(code: int) -> str:
+    return _lib.hsa_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != HSA_OK:
+        raise HSAError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _thd(t: torch.Tensor, name: str) -> Tuple[int, int]:
+    """(token stride, head stride) in elements of a bf16 [tokens, H, d] tensor, dim stride 1."""
+    if t.dtype != torch.bfloat16 or t.dim() != 3 or not t.is_cuda or t.stride(2) != 1:
+        raise ValueError(f"{name}: expected a CUDA bf16 [tokens, H, d] tensor with unit dim stride")
+    return t.stride(0), t.stride(1)
+
+
+# ------------------------------------------------------------------ C-named functions
+def hsa_query_sizes(cfg: hsa_config) -> hsa_sizes:
+    out = hsa_sizes()
+    _check(_lib.hsa_query_sizes(C.byref(cfg), C.byref(out)), "hsa_query_sizes")
+    return out
+
+
+def hsa_create(cfg: hsa_config, bufs: hsa_buffers, page_alloc_order: Optional[torch.Tensor]) -> int:
+    handle = C.c_void_p()
+    order_ptr = None
+    if page_alloc_order is not None:
+        order = page_alloc_order.to(device="cpu", dtype=torch.int32).contiguous()
+        order_ptr = order.data_ptr()
+    _check(_lib.hsa_create(C.byref(handle), C.byref(cfg), C.byref(bufs), order_ptr), "hsa_create")
+    return handle.value
+
+
+def hsa_append_kv(ctx: int, k: torch.Tensor, v: torch.Tensor) -> None:
+    ts, hs = _thd(k, "k")
+    if _thd(v, "v") != (ts, hs) or v.shape != k.shape:
+        raise ValueError("k and v must share shape and strides")
+    _check(_lib.hsa_append_kv(ctx, k.data_ptr(), v.data_ptr(), k.shape[0], ts, hs, _stream()),
+           "hsa_append_kv")
+
+
+def hsa_select_blocks(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budgets: torch.Tensor,
+                      q_group_tokens: int, sel_idx: torch.Tensor, sel_cnt: torch.Tensor) -> None:
+    ts, hs = _thd(q, "q")
+    _check(_lib.hsa_select_blocks(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
+                                  budgets.data_ptr(), int(q_group_tokens), sel_idx.data_ptr(),
+                                  sel_cnt.data_ptr(), _stream()), "hsa_select_blocks")
+
+
+def hsa_forward(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, sel_idx: Optional[torch.Tensor],
+                sel_cnt: Optional[torch.Tensor], q_group_tokens: int, g_lin: Optional[torch.Tensor],
+                g_sp: Optional[torch.Tensor], out: torch.Tensor, flags: int = 0) -> None:
+    ts, hs = _thd(q, "q")
+    ots, ohs = _thd(out, "out")
+    gts = ghs = gds = 0
+    for g in (g_lin, g_sp):
+        if g is not None:
+            if g.dtype != torch.bfloat16 or not g.is_cuda or g.dim() not in (2, 3):
+                raise ValueError("gates: expected CUDA bf16 [tokens, H] or [tokens, H, d]")
+            s = (g.stride(0), g.stride(1), g.stride(2) if g.dim() == 3 else 0)
+            if (gts, ghs, gds) != (0, 0, 0) and (gts, ghs, gds) != s:
+                raise ValueError("g_lin and g_sp must share strides")
+            gts, ghs, gds = s
+    _check(_lib.hsa_forward(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
+                            _ptr(sel_idx), _ptr(sel_cnt), int(q_group_tokens), _ptr(g_lin), _ptr(g_sp),
+                            gts, ghs, gds, out.data_ptr(), ots, ohs, int(flags), _stream()),
+           "hsa_forward")
+
+
+def hsa_get_info(ctx: int) -> Tuple[int, int]:
+    n, b = C.c_int64(), C.c_int32()
+    _check(_lib.hsa_get_info(ctx, C.byref(n), C.byref(b)), "hsa_get_info")
+    return n.value, b.value
+
+
+def hsa_rewind(ctx: int, n_tokens: int) -> None:
+    _check(_lib.hsa_rewind(ctx, int(n_tokens)), "hsa_rewind")
+
+
+def hsa_state_layout(ctx: int) -> Tuple[int, int, int]:
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(_lib.hsa_state_layout(ctx, C.byref(a), C.byref(b), C.byref(c)), "hsa_state_layout")
+    return a.value, b.value, c.value
+
+
+def hsa_device_status(ctx: int) -> int:
+    s = C.c_int32()
+    _check(_lib.hsa_device_status(ctx, C.byref(s)), "hsa_device_status")
+    return s.value
+
+
+def hsa_last_cuda_error(ctx: int) -> int:
+    return _lib.hsa_last_cuda_error(ctx)
+
+
+def hsa_destroy(ctx: int) -> None:
+    _check(_lib.hsa_destroy(ctx), "hsa_destroy")
+
+
+# ------------------------------------------------------------------ convenience wrapper
+class HSAContext:
+    """One attention layer of one sequence: allocates the caller-owned buffers with torch and
+    forwards every operation to the C ABI."""
+
+    def __init__(self, H: int, d: int, max_pages: int, max_q_tokens: int, max_topk: int,
+                 lin_mode: int = HSA_LIN_STATE, gate_act: int = 0, softmax_scale: float = 0.0,
+                 causal: bool = False, page_order: Optional[torch.Tensor] = None,
+                 device: str | torch.device = "cuda:0"):
+        self.device = torch.device(device)
+        self.H, self.d = H, d
+        self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
+        self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
+                              softmax_scale, HSA_CFG_CAUSAL if causal else 0)
+        self.sizes = hsa_query_sizes(self.cfg)
+        with torch.cuda.device(self.device):
+            mk = lambda n: torch.empty(max(n, 16), dtype=torch.uint8, device=self.device)
+            self.k_pool, self.v_pool = mk(self.sizes.k_pool), mk(self.sizes.v_pool)
+            self.state, self.workspace = mk(self.sizes.state), mk(self.sizes.workspace)
+            bufs = hsa_buffers(self.k_pool.data_ptr(), self.v_pool.data_ptr(), self.state.data_ptr(),
+                               self.workspace.data_ptr())
+            self.ctx = hsa_create(self.cfg, bufs, page_order)
+        self._off_S, self._off_z, self._off_ksum = hsa_state_layout(self.ctx)
+
+    # -- state views (fp32) for tests and snapshots
+    def _view(self, off: int, shape) -> torch.Tensor:
+        n = 1
+        for s in shape:
+            n *= s
+        return self.state[off:off + 4 * n].view(torch.float32).view(*shape)
+
+    @property
+    def S(self) -> torch.Tensor:
+        return self._view(self._off_S, (self.H, self.d, self.d))
+
+    @property
+    def z(self) -> torch.Tensor:
+        return self._view(self._off_z, (self.H, self.d))
+
+    @property
+    def ksum(self) -> torch.Tensor:
+        return self._view(self._off_ksum, (self.H, self.max_pages, self.d))
+
+    @property
+    def n_tokens(self) -> int:
+        return hsa_get_info(self.ctx)[0]
+
+    @property
+    def n_blocks(self) -> int:
+        return hsa_get_info(self.ctx)[1]
+
+    def n_groups(self, n_q: int, group_tokens: int) -> int:
+        return (n_q + group_tokens - 1) // group_tokens if group_tokens > 0 else 1
+
+    def append_kv(self, k: torch.Tensor, v: torch.Tensor) -> None:
+        hsa_append_kv(self.ctx, k, v)
+
+    def alloc_selection(self, n_q: int, group_tokens: int = 0):
+        g = self.n_groups(n_q, group_tokens)
+        return (torch.zeros(self.H, g, self.max_topk, dtype=torch.int32, device=self.device),
+                torch.zeros(self.H, g, dtype=torch.int32, device=self.device))
+
+    def select_blocks(self, q: torch.Tensor, budgets: torch.Tensor, q_pos0: Optional[int] = None,
+                      causal: bool = False, group_tokens: int = 0, sel=None):
+        q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
+        sel_idx, sel_cnt = sel if sel is not None else self.alloc_selection(q.shape[0], group_tokens)
+        hsa_select_blocks(self.ctx, q, q_pos0, causal, budgets, group_tokens, sel_idx, sel_cnt)
+        return sel_idx, sel_cnt
+
+    def forward(self, q: torch.Tensor, sel_idx, sel_cnt, q_pos0: Optional[int] = None,
+                causal: bool = False, group_tokens: int = 0, g_lin=None, g_sp=None, flags: int = 0,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.bfloat16, device=self.device)
+        hsa_forward(self.ctx, q, q_pos0, causal, sel_idx, sel_cnt, group_tokens, g_lin, g_sp, out, flags)
+        return out
+
+    def rewind(self, n_tokens: int) -> None:
+        hsa_rewind(self.ctx, n_tokens)
+
+    def device_status(self) -> int:
+        return hsa_device_status(self.ctx)
+
+    def destroy(self) -> None:
+        if getattr(self, "ctx", None):
+            hsa_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
