@@ -49,6 +49,13 @@ __global__ void __launch_bounds__(256) append_pool_ksum_kernel(AppendArgs a) {
       acc[2 * i + 1] += f.y;
     }
   }
+  // Rows of a partial tail page past the last token are zero-filled: the forward kernel masks
+  // their scores, but 0 * (uninitialised V) must not be able to produce a NaN.
+  for (int64_t t = t_hi + rg; t < b * kBlock + kBlock; t += RP) {
+    const size_t dst = (row_base + (t - b * kBlock)) * D + c8 * 8;
+    *reinterpret_cast<uint4*>(a.k_pool + dst) = make_uint4(0, 0, 0, 0);
+    *reinterpret_cast<uint4*>(a.v_pool + dst) = make_uint4(0, 0, 0, 0);
+  }
 #pragma unroll
   for (int i = 0; i < 8; ++i) red[rg][c8 * 8 + i] = acc[i];
   __syncthreads();

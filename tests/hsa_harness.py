@@ -32,6 +32,9 @@ def build_context(w: W.Workload, device, max_topk=None, causal=None, extra_pages
                          max_topk=max_topk or max(w.n_blocks, 1), lin_mode=lin_mode,
                          gate_act=gate_act, causal=w.causal if causal is None else causal,
                          page_order=order, device=device)
+    # poison the pools (0xFFFF is a bf16 NaN): anything read but never written shows up
+    ctx.k_pool.fill_(0xFF)
+    ctx.v_pool.fill_(0xFF)
     return ctx
 
 
