@@ -169,3 +169,8 @@ def sample_rows(w: Workload, n_random: int = 512, tile: int = 128) -> torch.Tens
     last = torch.arange(last_start, w.Lq)
     rnd = torch.randperm(w.Lq, generator=_gen(_tensor_seed(w, 9, 0)))[:n_random]
     return torch.unique(torch.cat([first, last, rnd])).to(torch.int64)
+
+
+def random_rows(w: Workload, n: int) -> torch.Tensor:
+    """n distinct seeded query rows (all rows if n >= Lq)."""
+    return torch.randperm(w.Lq, generator=_gen(_tensor_seed(w, 10, 0)))[:min(n, w.Lq)].to(torch.int64)
