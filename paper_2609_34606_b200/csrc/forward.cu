@@ -1,14 +1,19 @@
 // hsa_forward kernel for sm_100a.
 //
-// One CTA per (128-row query tile, head).  Warp roles:
-//   warp 0      TMA producer: Q tile, then the selected K/V pages gathered through the page
-//               table (two 64-token pages = 128 keys per step), then the hi/lo halves of the
-//               linear state; also owns the TMEM allocation
-//   warp 1      tcgen05.mma issuer: S = Q K^T into a double-buffered TMEM accumulator,
-//               O += P V with P read from TMEM, then the linear numerator phi(Q) S
-//   warps 2..5  one query row per thread: online softmax on S (tcgen05.ld), P written back to
-//               TMEM as bf16, lazy rescale of O, and the epilogue that normalises the sparse
-//               branch, applies the linear branch and the gates and stores bf16 once
+// One CTA per (128-row query tile, head), 384 threads in three warpgroups:
+//   warp 0       TMA producer: Q tile, then the selected K/V pages gathered through the page
+//                table (two 64-token pages = 128 keys per step) into a 3-stage ring, then the
+//                hi/lo halves of the linear state; also owns the TMEM allocation
+//   warp 1       tcgen05.mma issuer: S = Q K^T, O += P V with P read from TMEM, then the linear
+//                numerator phi(Q) S
+//   warps 4..7   softmax group A: the even KV steps     } one query row per thread; each group
+//   warps 8..11  softmax group B: the odd KV steps      } keeps its own running max / sum and
+//                                                         its own O accumulator in TMEM
+// The two groups never talk during the loop: while one exponentiates step j the tensor cores run
+// Q K^T of a later step and P V of the other group's step.  The two partial results of a row
+// are merged (log-sum-exp) in the epilogue, which also applies the linear branch and the gates
+// and stores bf16 once.  TMEM: S_A | S_B | O_A | O_B (128 fp32 columns each); P overwrites the
+// first 64 columns of its S buffer as packed bf16.
 // Every barrier wait is bounded; when one gives up the kernel records a timeout in the status
 // word and all roles drain to the common exit.
 #include <cuda_bf16.h>
@@ -20,30 +25,32 @@ namespace hsa {
 
 namespace {
 
-constexpr int kThreads = 192;
-constexpr int kStepKeys = 128;
-constexpr int kStages = 2;
+constexpr int kThreads = 384;
+constexpr int kStages = 3;
 constexpr uint32_t kTmemCols = 512;
-// TMEM column map
-constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256, kColP = 384, kColLin = 0;
+constexpr uint32_t kColS = 0;      // + 128 * group
+constexpr uint32_t kColO = 256;    // + 128 * group
+constexpr uint32_t kColLin = 0;    // linear numerator accumulator (after the loop)
+constexpr uint32_t kColPhi = 128;  // phi(Q) as a bf16 A operand (after the loop)
 
 template <int D>
 struct Smem {
-  static constexpr int kHalf = 128 * 128;               // bytes of one [128 rows x 128 B] slab
-  static constexpr int kTile = 128 * D * 2;             // Q tile, K stage, V stage
+  static constexpr int kHalf = 128 * 128;    // bytes of one [128 rows x 128 B] slab
+  static constexpr int kTile = 128 * D * 2;  // Q tile, K stage, V stage
   static constexpr int kQ = 0;
   static constexpr int kK = kTile;
   static constexpr int kV = kTile + kStages * kTile;
+  static constexpr int kStats = kK;  // float[2][128][4], reuses K stage 0 once the loop is over
   static constexpr int kBars = kTile + 2 * kStages * kTile;
-  static constexpr int kTotal = kBars + 256 + 1024;     // + alignment slack
+  static constexpr int kTotal = kBars + 256 + 1024;  // + alignment slack
 };
 
 struct Bars {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2];
-  uint64_t p_full;
-  uint64_t pv_done;
+  uint64_t p_full[2];
+  uint64_t o_done;
   uint64_t lin_a_full;
   uint64_t lin_done;
   uint32_t tmem_base;
@@ -79,6 +86,27 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float m;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+  return m;
+}
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+// (a0, a1) * s2 + t2 on the packed fp32 pipe
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, uint64_t s2,
+                                      uint64_t t2) {
+  uint64_t d;
+  const uint64_t a = pack2(a0, a1);
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(s2), "l"(t2));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 
 }  // namespace
 
@@ -93,6 +121,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   Bars* bars = reinterpret_cast<Bars*>(smem + L::kBars);
+  float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][m, l, den, -]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, h = blockIdx.y;
@@ -111,11 +140,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(&bars->v_full[s], 1);
       mbar_init(&bars->v_empty[s], 1);
     }
-    mbar_init(&bars->s_full[0], 1);
-    mbar_init(&bars->s_full[1], 1);
-    mbar_init(&bars->p_full, 128);
-    mbar_init(&bars->pv_done, 1);
-    mbar_init(&bars->lin_a_full, 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->s_full[i], 1);
+      mbar_init(&bars->p_full[i], 128);
+    }
+    mbar_init(&bars->o_done, 1);
+    mbar_init(&bars->lin_a_full, 256);
     mbar_init(&bars->lin_done, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -129,249 +159,263 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
-  if (warp == 0) {
-    // ================================================================= TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_q);
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(&bars->q_full, L::kTile);
-      for (int dh = 0; dh < DH; ++dh)
-        tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, h, row0);
-      bool ok = true;
-      int armed_k = 0, armed_v = 0;  // loads issued per ring, for the drain on abort
-      for (int j = 0; j < nsteps && ok; ++j) {
-        const int s = j % kStages;
-        const uint32_t ph = (j / kStages) & 1;
-        const int npg = min(2, cnt - 2 * j);
-        int32_t ycoord[2];
-        for (int pg = 0; pg < npg; ++pg) {
-          int blk = sel[2 * j + pg];
-          if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
-            atomicCAS(p.status, 0, kDevBounds);
-            blk = 0;
-          }
-          ycoord[pg] = (p.page_table[blk] * p.H + h) * kBlock;
-        }
-        ok = wait_bar(&bars->k_empty[s], ph ^ 1, bars, p.status);
-        if (!ok) break;
-        mbar_expect_tx(&bars->k_full[s], npg * kBlock * D * 2);
-        for (int pg = 0; pg < npg; ++pg)
-          for (int dh = 0; dh < DH; ++dh)
-            tma_load_2d(smem + L::kK + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_k,
-                        &bars->k_full[s], dh * 64, ycoord[pg]);
-        ++armed_k;
-        ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
-        if (!ok) break;
-        mbar_expect_tx(&bars->v_full[s], npg * kBlock * D * 2);
-        for (int pg = 0; pg < npg; ++pg)
-          for (int dh = 0; dh < DH; ++dh)
-            tma_load_2d(smem + L::kV + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_v,
-                        &bars->v_full[s], dh * 64, ycoord[pg]);
-        ++armed_v;
-      }
-      if (ok && p.do_linear) {
-        // hi and lo halves of the D x D state ride the V ring as two more "steps"
-        for (int hl = 0; hl < 2 && ok; ++hl) {
-          const int j = nsteps + hl;
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 0) {
+      // ================================================================= TMA producer
+      if (lane == 0) {
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        mbar_expect_tx(&bars->q_full, L::kTile);
+        for (int dh = 0; dh < DH; ++dh)
+          tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, h, row0);
+        bool ok = true;
+        int armed_k = 0, armed_v = 0;  // loads issued per ring, for the drain on abort
+        for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
           const uint32_t ph = (j / kStages) & 1;
+          const int npg = min(2, cnt - 2 * j);
+          int32_t ycoord[2];
+          for (int pg = 0; pg < npg; ++pg) {
+            int blk = sel[2 * j + pg];
+            if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
+              atomicCAS(p.status, 0, kDevBounds);
+              blk = 0;
+            }
+            ycoord[pg] = (p.page_table[blk] * p.H + h) * kBlock;
+          }
+          ok = wait_bar(&bars->k_empty[s], ph ^ 1, bars, p.status);
+          if (!ok) break;
+          mbar_expect_tx(&bars->k_full[s], npg * kBlock * D * 2);
+          for (int pg = 0; pg < npg; ++pg)
+            for (int dh = 0; dh < DH; ++dh)
+              tma_load_2d(smem + L::kK + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_k,
+                          &bars->k_full[s], dh * 64, ycoord[pg]);
+          ++armed_k;
           ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
           if (!ok) break;
-          const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
-          mbar_expect_tx(&bars->v_full[s], D * D * 2);
-          for (int kb = 0; kb < DH; ++kb)
+          mbar_expect_tx(&bars->v_full[s], npg * kBlock * D * 2);
+          for (int pg = 0; pg < npg; ++pg)
             for (int dh = 0; dh < DH; ++dh)
-              tma_load_2d(smem + L::kV + s * L::kTile + dh * L::kHalf + kb * (kBlock * 128),
-                          &tm_state, &bars->v_full[s], dh * 64, rbase + kb * 64);
+              tma_load_2d(smem + L::kV + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_v,
+                          &bars->v_full[s], dh * 64, ycoord[pg]);
           ++armed_v;
         }
-      }
-      if (!ok) {
-        // drain: let every copy already issued land before the CTA's shared memory goes away
-        for (int s = 0; s < kStages; ++s) {
-          for (int i = 0; i < 2; ++i) {
-            const int arms = i == 0 ? armed_k : armed_v;
-            uint64_t* bar = i == 0 ? &bars->k_full[s] : &bars->v_full[s];
-            const int last = ((arms - 1 - s) / kStages) * kStages + s;  // last step armed on s
-            if (arms > s) mbar_wait(bar, (last / kStages) & 1, 1u << 16);
+        if (ok && p.do_linear) {
+          // hi and lo halves of the D x D state ride the V ring as two more "steps"
+          for (int hl = 0; hl < 2 && ok; ++hl) {
+            const int j = nsteps + hl;
+            const int s = j % kStages;
+            const uint32_t ph = (j / kStages) & 1;
+            ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
+            if (!ok) break;
+            const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
+            mbar_expect_tx(&bars->v_full[s], D * D * 2);
+            for (int kb = 0; kb < DH; ++kb)
+              for (int dh = 0; dh < DH; ++dh)
+                tma_load_2d(smem + L::kV + s * L::kTile + dh * L::kHalf + kb * (kBlock * 128),
+                            &tm_state, &bars->v_full[s], dh * 64, rbase + kb * 64);
+            ++armed_v;
+          }
+        }
+        if (!ok) {
+          // drain: let every copy already issued land before the CTA's shared memory goes away
+          for (int s = 0; s < kStages; ++s) {
+            for (int i = 0; i < 2; ++i) {
+              const int arms = i == 0 ? armed_k : armed_v;
+              uint64_t* bar = i == 0 ? &bars->k_full[s] : &bars->v_full[s];
+              const int last = ((arms - 1 - s) / kStages) * kStages + s;  // last step armed on s
+              if (arms > s) mbar_wait(bar, (last / kStages) & 1, 1u << 16);
+            }
           }
         }
       }
-    }
-  } else if (warp == 1) {
-    // ================================================================= MMA issuer
-    if (lane == 0) {
-      const uint32_t q_addr = smem_u32(smem + L::kQ);
-      bool ok = wait_bar(&bars->q_full, 0, bars, p.status);
-      tc_fence_after();
-      auto issue_qk = [&](int j) -> bool {
-        const int s = j % kStages;
-        if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
+    } else if (warp == 1) {
+      // ================================================================= MMA issuer
+      if (lane == 0) {
+        const uint32_t q_addr = smem_u32(smem + L::kQ);
+        bool ok = wait_bar(&bars->q_full, 0, bars, p.status);
         tc_fence_after();
-        const int n = min(2, cnt - 2 * j) * kBlock;
-        const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
-        const uint32_t k_addr = smem_u32(smem + L::kK + s * L::kTile);
-        const uint32_t d_tmem = tmem + ((j & 1) ? kColS1 : kColS0);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * L::kHalf + (kk % 4) * 32;
-          tc_mma_ss(d_tmem, smem_desc_sw128(q_addr + off, 16, 1024),
-                    smem_desc_sw128(k_addr + off, 16, 1024), idesc, kk > 0);
-        }
-        tc_commit(&bars->k_empty[s]);
-        tc_commit(&bars->s_full[j & 1]);
-        return true;
-      };
-      if (ok && nsteps > 0) ok = issue_qk(0);
-      for (int j = 0; j < nsteps && ok; ++j) {
-        if (j + 1 < nsteps) {
-          ok = issue_qk(j + 1);
-          if (!ok) break;
-        }
-        const int s = j % kStages;
-        ok = wait_bar(&bars->p_full, j & 1, bars, p.status);
-        if (!ok) break;
-        ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const int n = min(2, cnt - 2 * j) * kBlock;
-        const uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
-        const uint32_t v_addr = smem_u32(smem + L::kV + s * L::kTile);
-        for (int kk = 0; kk < n / 16; ++kk)
-          tc_mma_ts(tmem + kColO, tmem + kColP + kk * 8,
-                    smem_desc_sw128(v_addr + kk * 2048, L::kHalf, 1024), idesc, (j > 0) || (kk > 0));
-        tc_commit(&bars->v_empty[s]);
-        tc_commit(&bars->pv_done);
-      }
-      if (ok && p.do_linear) {
-        ok = wait_bar(&bars->lin_a_full, 0, bars, p.status);
-        for (int hl = 0; hl < 2 && ok; ++hl) {
-          const int j = nsteps + hl;
+        auto issue_qk = [&](int j) -> bool {
           const int s = j % kStages;
+          if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
+          tc_fence_after();
+          const int n = min(2, cnt - 2 * j) * kBlock;
+          const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
+          const uint32_t k_addr = smem_u32(smem + L::kK + s * L::kTile);
+          const uint32_t d_tmem = tmem + kColS + 128 * (j & 1);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk / 4) * L::kHalf + (kk % 4) * 32;
+            tc_mma_ss(d_tmem, smem_desc_sw128(q_addr + off, 16, 1024),
+                      smem_desc_sw128(k_addr + off, 16, 1024), idesc, kk > 0);
+          }
+          tc_commit(&bars->k_empty[s]);
+          tc_commit(&bars->s_full[j & 1]);
+          return true;
+        };
+        if (ok && nsteps > 0) ok = issue_qk(0);
+        if (ok && nsteps > 1) ok = issue_qk(1);
+        for (int j = 0; j < nsteps && ok; ++j) {
+          const int s = j % kStages;
+          ok = wait_bar(&bars->p_full[j & 1], (j >> 1) & 1, bars, p.status);
+          if (!ok) break;
           ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
           if (!ok) break;
           tc_fence_after();
+          const int n = min(2, cnt - 2 * j) * kBlock;
           const uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
-          const uint32_t b_addr = smem_u32(smem + L::kV + s * L::kTile);
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk)
-            tc_mma_ts(tmem + kColLin, tmem + kColP + kk * 8,
-                      smem_desc_sw128(b_addr + kk * 2048, L::kHalf, 1024), idesc,
-                      (hl > 0) || (kk > 0));
+          const uint32_t v_addr = smem_u32(smem + L::kV + s * L::kTile);
+          const uint32_t o_acc = tmem + kColO + 128 * (j & 1);
+          const uint32_t p_op = tmem + kColS + 128 * (j & 1);
+          for (int kk = 0; kk < n / 16; ++kk)
+            tc_mma_ts(o_acc, p_op + kk * 8, smem_desc_sw128(v_addr + kk * 2048, L::kHalf, 1024),
+                      idesc, (j >= 2) || (kk > 0));
           tc_commit(&bars->v_empty[s]);
+          // the next scores of this group overwrite the P just consumed: issued after the P V
+          // above, the tensor pipe runs them in order
+          if (j + 2 < nsteps) ok = issue_qk(j + 2);
         }
-        if (ok) tc_commit(&bars->lin_done);
+        if (ok) tc_commit(&bars->o_done);
+        if (ok && p.do_linear) {
+          ok = wait_bar(&bars->lin_a_full, 0, bars, p.status);
+          for (int hl = 0; hl < 2 && ok; ++hl) {
+            const int j = nsteps + hl;
+            const int s = j % kStages;
+            ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
+            const uint32_t b_addr = smem_u32(smem + L::kV + s * L::kTile);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk)
+              tc_mma_ts(tmem + kColLin, tmem + kColPhi + kk * 8,
+                        smem_desc_sw128(b_addr + kk * 2048, L::kHalf, 1024), idesc,
+                        (hl > 0) || (kk > 0));
+            tc_commit(&bars->v_empty[s]);
+          }
+          if (ok) tc_commit(&bars->lin_done);
+        }
       }
     }
   } else {
-    // ================================================================= softmax + epilogue
+    // ================================================================= softmax groups + epilogue
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int grp = (warp - 4) >> 2;                 // 0: even steps, 1: odd steps
     const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
     const int r = quad * 32 + lane;                  // row inside the tile
     const int row = row0 + r;                        // query index inside the chunk
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+    const uint32_t s_tmem = tmem + lane_off + kColS + 128 * grp;
+    const uint32_t o_tmem = tmem + lane_off + kColO + 128 * grp;
     const int64_t qpos = p.q_pos0 + row;
     const int64_t vis_end = p.causal ? min64(p.n_tokens, qpos + 1) : p.n_tokens;
+    // the first row of the tile sees the fewest keys: a step whose pages all end at or before
+    // that row's limit needs no masking
+    const int64_t tile_vis_end = p.causal ? min64(p.n_tokens, p.q_pos0 + row0 + 1) : p.n_tokens;
     const float sl2 = p.scale_log2;
     float m_used = -INFINITY;  // reference maximum the stored exponents are relative to (raw)
     float l = 0.f;
     bool ok = true;
 
-    for (int j = 0; j < nsteps; ++j) {
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[j & 1], (j >> 1) & 1, bars, p.status));
+    for (int j = grp; j < nsteps; j += 2) {
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[grp], (j >> 1) & 1, bars, p.status));
       if (!ok) break;
       tc_fence_after();
       const int npg = min(2, cnt - 2 * j);
       const int n = npg * kBlock;
-      const uint32_t s_addr = tmem + lane_off + ((j & 1) ? kColS1 : kColS0);
       uint32_t sr[128];
-      tmem_ld32(s_addr + 0, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
-      tmem_ld32(s_addr + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
+      tmem_ld32(s_tmem + 0, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
+      tmem_ld32(s_tmem + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
       if (n == 128) {
-        tmem_ld32(s_addr + 64, reinterpret_cast<uint32_t(&)[32]>(sr[64]));
-        tmem_ld32(s_addr + 96, reinterpret_cast<uint32_t(&)[32]>(sr[96]));
+        tmem_ld32(s_tmem + 64, reinterpret_cast<uint32_t(&)[32]>(sr[64]));
+        tmem_ld32(s_tmem + 96, reinterpret_cast<uint32_t(&)[32]>(sr[96]));
       }
+      int blk0 = sel[2 * j], blk1 = npg > 1 ? sel[2 * j + 1] : 0;
+      if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
+      if (blk1 < 0 || blk1 >= p.n_blocks) blk1 = 0;
+      const int64_t last_blk = blk0 > blk1 ? blk0 : blk1;
+      const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > tile_vis_end);
       tc_wait_ld();
-      // visible keys per page: columns [0, lim) of the page's 64
-      int lim[2];
+      if (need_mask) {
+        // visible keys per page: columns [0, lim) of the page's 64
+        const int lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
+        const int lim1 =
+            npg > 1 ? static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk1) * kBlock))) : 0;
 #pragma unroll
-      for (int pg = 0; pg < 2; ++pg) {
-        int blk = pg < npg ? sel[2 * j + pg] : 0;
-        if (blk < 0 || blk >= p.n_blocks) blk = 0;
-        const int64_t v = vis_end - static_cast<int64_t>(blk) * kBlock;
-        lim[pg] = pg < npg ? static_cast<int>(max64(0, min64(kBlock, v))) : 0;
+        for (int c = 0; c < 128; ++c) {
+          const bool valid = (c & 63) < ((c >> 6) ? lim1 : lim0);
+          if (!valid) sr[c] = 0xff800000u;  // -inf
+        }
       }
-      float m_new = -INFINITY;
+      float m_new = fmaxf(__uint_as_float(sr[0]), __uint_as_float(sr[1]));
 #pragma unroll
-      for (int c = 0; c < 128; ++c) {
-        const bool valid = (c & 63) < lim[c >> 6];
-        float v = valid ? __uint_as_float(sr[c]) : -INFINITY;
-        sr[c] = __float_as_uint(v);
-        m_new = fmaxf(m_new, v);
-      }
+      for (int c = 2; c < 128; c += 2)
+        m_new = fmax3(m_new, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
       // lazy rescale: move the reference maximum only when it would grow by more than 2^8
       float factor = 1.f;
-      bool rescale = false;
       if (m_used == -INFINITY) {
         m_used = m_new;  // nothing accumulated so far (O and l are zero or not yet written)
       } else if ((m_new - m_used) * sl2 > 8.f) {
         factor = ex2((m_used - m_new) * sl2);
         l *= factor;
         m_used = m_new;
-        rescale = true;
       }
-      const float moff = (m_used == -INFINITY) ? 0.f : m_used * sl2;
-      uint32_t pr[64];
-      float lsum = 0.f;
+      // O of this group is quiescent here: its previous P V completed before this step's scores
+      // were committed, and its next P V waits for the P written below
+      if (j >= 2 && __any_sync(0xffffffffu, factor != 1.f)) {
 #pragma unroll
-      for (int c = 0; c < 128; c += 2) {
-        const float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -moff));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -moff));
-        lsum += p0 + p1;
-        pr[c >> 1] = pack_bf16(p0, p1);
-      }
-      l += lsum;
-      if (j > 0) {
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (j - 1) & 1, bars, p.status));
-        if (!ok) break;
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, rescale)) {
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld32(o_tmem + c0, o);
+          tc_wait_ld();
 #pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t o[32];
-            tmem_ld32(tmem + lane_off + kColO + c0, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-            tmem_st32(tmem + lane_off + kColO + c0, o);
-          }
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+          tmem_st32(o_tmem + c0, o);
         }
       }
-      tmem_st32(tmem + lane_off + kColP, reinterpret_cast<uint32_t(&)[32]>(pr[0]));
-      if (n == 128) tmem_st32(tmem + lane_off + kColP + 32, reinterpret_cast<uint32_t(&)[32]>(pr[32]));
+      const float moff = (m_used == -INFINITY) ? 0.f : m_used * sl2;
+      const uint64_t s2 = pack2(sl2, sl2), t2 = pack2(-moff, -moff);
+      float lsum0 = 0.f, lsum1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 128; c += 2) {
+        float x0, x1;
+        ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), s2, t2);
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        lsum0 += p0;
+        lsum1 += p1;
+        sr[c >> 1] = pack_bf16(p0, p1);
+      }
+      l += lsum0 + lsum1;
+      tmem_st32(s_tmem, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
+      if (n == 128) tmem_st32(s_tmem + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(&bars->p_full);
+      mbar_arrive(&bars->p_full[grp]);
     }
 
     // ---------------------------------------------------------------- epilogue
     if (ok && nsteps > 0) {
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (nsteps - 1) & 1, bars, p.status));
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
       tc_fence_after();
     }
-    float den = 0.f;
+    // this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D)
+    constexpr int HC = D / 2;
+    const int cbase = grp * HC;
+    float den_part = 0.f;
     if (ok && p.do_linear) {
-      // phi(q) of this thread's row -> bf16 A operand in TMEM; denominator phi(q) . z
+      // phi(q) of this thread's row for its half of the dims -> bf16 A operand in TMEM;
+      // partial denominator phi(q) . z over the same dims
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
       const uint8_t* qrow = smem + L::kQ + r * 128;
       const float* z = p.z + static_cast<size_t>(h) * D;
-      uint32_t fr[D / 2];
-      // Q landed through the async proxy; q_full was observed only by the MMA warp, so observe it
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
+      uint32_t fr[HC / 2];
 #pragma unroll
-      for (int c16 = 0; c16 < D / 8; ++c16) {
-        const int dh = c16 >> 3, ch = c16 & 7;
-        const uint4 raw =
-            *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
+      for (int c16 = 0; c16 < HC / 8; ++c16) {
+        const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
+        const int dh = cc >> 3, ch = cc & 7;
+        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
         const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -381,21 +425,42 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
           fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
           const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
-          den = fmaf(rr.x, z[c16 * 8 + 2 * i], den);
-          den = fmaf(rr.y, z[c16 * 8 + 2 * i + 1], den);
+          den_part = fmaf(rr.x, z[cbase + c16 * 8 + 2 * i], den_part);
+          den_part = fmaf(rr.y, z[cbase + c16 * 8 + 2 * i + 1], den_part);
         }
       }
-      tmem_st32(tmem + lane_off + kColP, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
-      if (D == 128) tmem_st32(tmem + lane_off + kColP + 32, reinterpret_cast<uint32_t(&)[32]>(fr[D / 2 - 32]));
+      if constexpr (D == 128) {
+        tmem_st32(tmem + lane_off + kColPhi + grp * 32, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
+      } else {
+        tmem_st16(tmem + lane_off + kColPhi + grp * 16, reinterpret_cast<uint32_t(&)[16]>(fr[0]));
+      }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->lin_a_full);
-      if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
+    }
+    // publish this group's row statistics, then read the other group's
+    stats[(grp * 128 + r) * 4 + 0] = m_used;
+    stats[(grp * 128 + r) * 4 + 1] = l;
+    stats[(grp * 128 + r) * 4 + 2] = den_part;
+    named_bar_sync(1, 256);
+    const float m_o = stats[((grp ^ 1) * 128 + r) * 4 + 0];
+    const float l_o = stats[((grp ^ 1) * 128 + r) * 4 + 1];
+    const float den = den_part + stats[((grp ^ 1) * 128 + r) * 4 + 2];
+    // log-sum-exp merge of the two partial softmax results of this row
+    const float mm = fmaxf(m_used, m_o);
+    const float c_me = (m_used == -INFINITY) ? 0.f : ex2((m_used - mm) * sl2);
+    const float c_ot = (m_o == -INFINITY) ? 0.f : ex2((m_o - mm) * sl2);
+    const float lsum = l * c_me + l_o * c_ot;
+    const float inv_l = lsum > 0.f ? 1.f / lsum : 0.f;
+    const float w_a = (grp == 0 ? c_me : c_ot) * inv_l;  // weight of accumulator A
+    const float w_b = (grp == 0 ? c_ot : c_me) * inv_l;  // weight of accumulator B
+    const bool has_a = nsteps > 0, has_b = nsteps > 1;
+    if (ok && p.do_linear) {
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
       tc_fence_after();
     }
     if (ok) {  // warp-uniform: the TMEM loads below are warp-collective
       const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
-      const float inv_l = (nsteps > 0 && l > 0.f) ? 1.f / l : 0.f;
       float lin_den = den;
       const float* lnum = nullptr;
       if (wr && p.do_linear && p.lin_num != nullptr) {
@@ -409,20 +474,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const __nv_bfloat16* gs =
           (wr && p.g_sp) ? p.g_sp + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
 #pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t o[32], ln[32];
-        if (nsteps > 0) {
-          tmem_ld32(tmem + lane_off + kColO + c0, o);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = 0u;
-        }
-        if (p.do_linear) {
-          tmem_ld32(tmem + lane_off + kColLin + c0, ln);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) ln[i] = 0u;
-        }
+      for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
+        uint32_t oa[32], ob[32], ln[32];
+        if (has_a) tmem_ld32(tmem + lane_off + kColO + c0, oa);
+        if (has_b) tmem_ld32(tmem + lane_off + kColO + 128 + c0, ob);
+        if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
         tc_wait_ld();
         uint32_t packed[16];
 #pragma unroll
@@ -431,10 +487,15 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int c = c0 + i + e;
-            const float osp = __uint_as_float(o[i + e]) * inv_l;
-            float num = __uint_as_float(ln[i + e]);
-            if (lnum) num += lnum[c];
-            const float olin = num * inv_den;
+            float osp = 0.f;
+            if (has_a) osp = __uint_as_float(oa[i + e]) * w_a;
+            if (has_b) osp = fmaf(__uint_as_float(ob[i + e]), w_b, osp);
+            float olin = 0.f;
+            if (p.do_linear) {
+              float num = __uint_as_float(ln[i + e]);
+              if (lnum) num += lnum[c];
+              olin = num * inv_den;
+            }
             float wl = 1.f, ws = 1.f;
             if (gl) {
               wl = __bfloat162float(gl[static_cast<size_t>(c) * p.g_ds]);
@@ -448,11 +509,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           packed[i >> 1] = pack_bf16(res[0], res[1]);
         }
-        if (wr)
+        if (wr) {
 #pragma unroll
-        for (int v4 = 0; v4 < 4; ++v4)
-          *reinterpret_cast<uint4*>(orow + c0 + v4 * 8) =
-              make_uint4(packed[v4 * 4], packed[v4 * 4 + 1], packed[v4 * 4 + 2], packed[v4 * 4 + 3]);
+          for (int v4 = 0; v4 < 4; ++v4)
+            *reinterpret_cast<uint4*>(orow + c0 + v4 * 8) =
+                make_uint4(packed[v4 * 4], packed[v4 * 4 + 1], packed[v4 * 4 + 2], packed[v4 * 4 + 3]);
+        }
       }
     }
   }

@@ -38,7 +38,7 @@ struct Layout {
   // state
   size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
   // workspace
-  size_t status, page_table, qpart, spart, lin_num, lin_den, ws_total;
+  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ws_total;
 };
 
 bool config_ok(const hsa_config* c) {
@@ -70,6 +70,7 @@ Layout make_layout(const hsa_config* c) {
   L.status = o;     o = align_up(o + 16, 256);
   L.page_table = o; o = align_up(o + P * 4, 256);
   L.qpart = o;      o = align_up(o + tiles * H * D * 4, 256);
+  L.keys = o;       o = align_up(o + H * tiles * P * 4, 256);
   L.spart = o;      o = align_up(o + H * kStateSplitMax * (D * D + D) * 4, 256);
   if (c->flags & HSA_CFG_CAUSAL) {
     L.lin_num = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 4, 256);
@@ -285,6 +286,7 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
   a.n_groups = q_group_tokens > 0 ? (n_q + q_group_tokens - 1) / q_group_tokens : 1;
   a.scale = ctx->scale;
   a.qpart = reinterpret_cast<float*>(ws + ctx->lay.qpart);
+  a.keys = reinterpret_cast<uint32_t*>(ws + ctx->lay.keys);
   a.sel_idx = sel_idx_dev;
   a.sel_cnt = sel_cnt_dev;
   a.kcap = ctx->cfg.max_topk;

@@ -53,6 +53,7 @@ struct SelectArgs {
   int group_tokens, n_groups;
   float scale;
   float* qpart;  // [n_tiles][H][D] scratch
+  uint32_t* keys;  // [H][n_groups][max_pages] scratch: order-preserving score keys
   int32_t* sel_idx;
   int32_t* sel_cnt;
   int kcap;

@@ -1,6 +1,7 @@
 // hsa_select_blocks kernels: mean query per group, pooled block scores
 //   s[h,g,b] = mean_q(g) . (Ksum[h,b] / cnt_b) * scale
-// and an exact per-(head, group) top-k by radix select, all on the device.
+// and an exact per-(head, group) top-k by radix select, all on the device:
+// query partial sums -> scores (many CTAs) -> top-k (one CTA per head and group).
 #include <cuda_bf16.h>
 
 #include "hsa_internal.h"
@@ -73,32 +74,20 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
 }
 
 // ---------------------------------------------------------------------------------------
-// Stage 2: one CTA per (group, head): scores for every block, k-th largest by a 4-pass
-// 8-bit radix select on order-preserving keys, then an index-ordered compaction.
-// Exact ties at the threshold go to the lower block index.
-// dynamic smem: uint32 keys[nblk]
+// Stage 2: pooled scores.  grid (ceil(nblk/32), n_groups, H); one warp per block, four blocks
+// per warp.  The mean query of the group is rebuilt from the tile partials in fp64 (fixed
+// order), the dot product runs in fp64 and is rounded once to the fp32 sort key.
 // ---------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(256) score_select_kernel(SelectArgs a) {
-  extern __shared__ uint32_t keys[];
-  __shared__ double qs[D];
-  __shared__ int hist[256];
-  __shared__ int warp_sums[8];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_krem;
+constexpr int kScoreBlocksPerCta = 32;
 
-  const int g = blockIdx.x, h = blockIdx.y;
+template <int D>
+__global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
+  __shared__ double qs[D];
+  const int g = blockIdx.y, h = blockIdx.z;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
-  const int64_t p_last = a.q_pos0 + q_hi - 1;
-  // candidate blocks are a prefix [0, ncand)
-  int64_t ncand64 = nblk;
-  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
-  const int ncand = static_cast<int>(ncand64);
-
-  // mean query of the group (fp64 over the tile partials, fixed order), pre-scaled
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   if (threadIdx.x < D) {
     double s = 0.0;
     const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
@@ -107,20 +96,51 @@ __global__ void __launch_bounds__(256) score_select_kernel(SelectArgs a) {
     qs[threadIdx.x] = s / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
   }
   __syncthreads();
-
-  // scores
   constexpr int PER = D / 32;
-  for (int b = warp; b < ncand; b += 8) {
+  uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+#pragma unroll
+  for (int i = 0; i < kScoreBlocksPerCta / 8; ++i) {
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * kScoreBlocksPerCta + i * 8 + warp;
+    if (b >= nblk) continue;  // warp-uniform
     const float* ks = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER;
     double dot = 0.0;
 #pragma unroll
-    for (int i = 0; i < PER; ++i) dot += qs[lane * PER + i] * static_cast<double>(ks[i]);
+    for (int e = 0; e < PER; ++e) dot += qs[lane * PER + e] * static_cast<double>(ks[e]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
     if (lane == 0) {
-      const int64_t cnt = min64(kBlock, a.n_tokens - static_cast<int64_t>(b) * kBlock);
+      const int64_t cnt = min64(kBlock, a.n_tokens - b * kBlock);
       keys[b] = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
     }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Stage 3: one CTA per (group, head): k-th largest key by a 4-pass 8-bit radix select, then an
+// index-ordered compaction.  Exact ties at the threshold go to the lower block index.
+// dynamic smem: uint32 keys[ncand]
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
+  extern __shared__ uint32_t keys[];
+  __shared__ int hist[256];
+  __shared__ int warp_sums[8];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_krem;
+
+  const int g = blockIdx.x, h = blockIdx.y;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
+  const int q_hi = min(a.n_q, g * gtok + gtok);
+  const int64_t p_last = a.q_pos0 + q_hi - 1;
+  // candidate blocks are a prefix [0, ncand)
+  int64_t ncand64 = nblk;
+  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
+  const int ncand = static_cast<int>(ncand64);
+  const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = gkeys[b];
+  if (threadIdx.x == 0) {
+    sh_prefix = 0;
+    sh_krem = 0;
   }
   __syncthreads();
 
@@ -130,35 +150,33 @@ __global__ void __launch_bounds__(256) score_select_kernel(SelectArgs a) {
   uint32_t thr = 0;
   int need_ties = 0;
   if (!take_all && budget > 0) {
-    if (threadIdx.x == 0) {
-      sh_prefix = 0;
-      sh_krem = budget;
-    }
-    uint32_t mask = 0;
+    uint32_t mask = 0, prefix = 0;
+    int krem = budget;
     for (int pass = 3; pass >= 0; --pass) {
       const int shift = pass * 8;
       hist[threadIdx.x] = 0;
       __syncthreads();
-      const uint32_t prefix = sh_prefix;
       for (int b = threadIdx.x; b < ncand; b += 256) {
         const uint32_t k = keys[b];
         if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        int krem = sh_krem, cum = 0, bin = 255;
-        for (; bin > 0; --bin) {
-          if (cum + hist[bin] >= krem) break;
-          cum += hist[bin];
-        }
+      // thread t owns bin 255 - t: an inclusive prefix over t is the count of keys in bins >= own
+      const int bin = 255 - static_cast<int>(threadIdx.x);
+      const int mine = hist[bin];
+      int tot;
+      const int above = block_exclusive_scan(mine, warp_sums, &tot);  // keys in strictly higher bins
+      if (above < krem && above + mine >= krem) {                     // exactly one thread
         sh_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
-        sh_krem = krem - cum;  // still to take among keys matching the longer prefix
+        sh_krem = krem - above;  // still to take among keys matching the longer prefix
       }
-      mask |= 255u << shift;
       __syncthreads();
+      prefix = sh_prefix;
+      krem = sh_krem;
+      mask |= 255u << shift;
     }
-    thr = sh_prefix;
-    need_ties = sh_krem;
+    thr = prefix;
+    need_ties = krem;
   }
 
   // index-ordered compaction: thread t owns the contiguous range [t*per, t*per+per)
@@ -217,19 +235,20 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  const size_t smem = static_cast<size_t>(nblk > 0 ? nblk : 1) * sizeof(uint32_t);
-  dim3 g2(a.n_groups, a.H);
-  if (a.D == 128) {
-    if (smem > 40 * 1024)
-      cudaFuncSetAttribute(score_select_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(smem));
-    score_select_kernel<128><<<g2, 256, smem, st>>>(a);
-  } else {
-    if (smem > 40 * 1024)
-      cudaFuncSetAttribute(score_select_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(smem));
-    score_select_kernel<64><<<g2, 256, smem, st>>>(a);
+  if (nblk > 0) {
+    dim3 g2(static_cast<unsigned>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta), a.n_groups, a.H);
+    if (a.D == 128)
+      block_scores_kernel<128><<<g2, 256, 0, st>>>(a);
+    else
+      block_scores_kernel<64><<<g2, 256, 0, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
   }
+  const size_t smem = static_cast<size_t>(nblk > 0 ? nblk : 1) * sizeof(uint32_t);
+  if (smem > 40 * 1024)
+    cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  dim3 g3(a.n_groups, a.H);
+  topk_kernel<<<g3, 256, smem, st>>>(a);
   return cudaGetLastError();
 }
 
