@@ -81,6 +81,17 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b
   }
 }
 
+#ifdef HSA_TIMING
+__device__ long long g_hsa_timing[4096];
+#define HSA_T(slot)                                                                  \
+  do {                                                                               \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (slot) < 4096)             \
+      g_hsa_timing[(slot)] = clock64();                                              \
+  } while (0)
+#else
+#define HSA_T(slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -104,6 +115,14 @@ __device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, 
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(s2), "l"(t2));
   asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
 }
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
@@ -124,6 +143,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][m, l, den, -]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp == 4) HSA_T(3000);
   const int tile = blockIdx.x, h = blockIdx.y;
   const int row0 = tile * kTileM;
   const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
@@ -158,12 +178,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
+  if (warp == 4) HSA_T(3001);
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (warp == 0) {
       // ================================================================= TMA producer
-      if (lane == 0) {
+      if (elect_one_sync()) {
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
@@ -172,6 +193,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, h, row0);
         bool ok = true;
         int armed_k = 0, armed_v = 0;  // loads issued per ring, for the drain on abort
+#pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
           const uint32_t ph = (j / kStages) & 1;
@@ -233,23 +255,32 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
     } else if (warp == 1) {
       // ================================================================= MMA issuer
-      if (lane == 0) {
-        const uint32_t q_addr = smem_u32(smem + L::kQ);
+      if (elect_one_sync()) {
+        constexpr uint32_t kHiSw = desc_hi_sw128(1024);
+        const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::kQ), 16);
         bool ok = wait_bar(&bars->q_full, 0, bars, p.status);
         tc_fence_after();
+        HSA_T(3011);
         auto issue_qk = [&](int j) -> bool {
           const int s = j % kStages;
           if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
           tc_fence_after();
-          const int n = min(2, cnt - 2 * j) * kBlock;
-          const uint32_t idesc = idesc_bf16_f32(128, n, 0, 0);
-          const uint32_t k_addr = smem_u32(smem + L::kK + s * L::kTile);
+          const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::kK + s * L::kTile), 16);
           const uint32_t d_tmem = tmem + kColS + 128 * (j & 1);
+          if (cnt - 2 * j >= 2) {
+            constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 0, 0);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk / 4) * L::kHalf + (kk % 4) * 32;
-            tc_mma_ss(d_tmem, smem_desc_sw128(q_addr + off, 16, 1024),
-                      smem_desc_sw128(k_addr + off, 16, 1024), idesc, kk > 0);
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t off = ((kk / 4) * L::kHalf + (kk % 4) * 32) >> 4;
+              tc_mma_ss_lo(d_tmem, q_lo + off, k_lo + off, kHiSw, idesc, kk > 0 ? 1u : 0u);
+            }
+          } else {
+            constexpr uint32_t idesc = idesc_bf16_f32(128, 64, 0, 0);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t off = ((kk / 4) * L::kHalf + (kk % 4) * 32) >> 4;
+              tc_mma_ss_lo(d_tmem, q_lo + off, k_lo + off, kHiSw, idesc, kk > 0 ? 1u : 0u);
+            }
           }
           tc_commit(&bars->k_empty[s]);
           tc_commit(&bars->s_full[j & 1]);
@@ -257,25 +288,36 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         };
         if (ok && nsteps > 0) ok = issue_qk(0);
         if (ok && nsteps > 1) ok = issue_qk(1);
+#pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
+          HSA_T(2048 + j * 8 + 0);
           ok = wait_bar(&bars->p_full[j & 1], (j >> 1) & 1, bars, p.status);
           if (!ok) break;
+          HSA_T(2048 + j * 8 + 1);
           ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
           if (!ok) break;
           tc_fence_after();
-          const int n = min(2, cnt - 2 * j) * kBlock;
-          const uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
-          const uint32_t v_addr = smem_u32(smem + L::kV + s * L::kTile);
+          HSA_T(2048 + j * 8 + 2);
+          constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
+          const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
           const uint32_t o_acc = tmem + kColO + 128 * (j & 1);
           const uint32_t p_op = tmem + kColS + 128 * (j & 1);
-          for (int kk = 0; kk < n / 16; ++kk)
-            tc_mma_ts(o_acc, p_op + kk * 8, smem_desc_sw128(v_addr + kk * 2048, L::kHalf, 1024),
-                      idesc, (j >= 2) || (kk > 0));
+          const uint32_t acc0 = j >= 2 ? 1u : 0u;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, kk > 0 ? 1u : acc0);
+          if (cnt - 2 * j >= 2) {
+#pragma unroll
+            for (int kk = 4; kk < 8; ++kk)
+              tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, 1u);
+          }
           tc_commit(&bars->v_empty[s]);
+          HSA_T(2048 + j * 8 + 3);
           // the next scores of this group overwrite the P just consumed: issued after the P V
           // above, the tensor pipe runs them in order
           if (j + 2 < nsteps) ok = issue_qk(j + 2);
+          HSA_T(2048 + j * 8 + 4);
         }
         if (ok) tc_commit(&bars->o_done);
         if (ok && p.do_linear) {
@@ -286,13 +328,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
-            const uint32_t b_addr = smem_u32(smem + L::kV + s * L::kTile);
+            constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
+            const uint32_t b_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk)
-              tc_mma_ts(tmem + kColLin, tmem + kColPhi + kk * 8,
-                        smem_desc_sw128(b_addr + kk * 2048, L::kHalf, 1024), idesc,
-                        (hl > 0) || (kk > 0));
+              tc_mma_ts_lo(tmem + kColLin, tmem + kColPhi + kk * 8, b_lo + kk * 128, kHiSw, idesc,
+                           (hl > 0 || kk > 0) ? 1u : 0u);
             tc_commit(&bars->v_empty[s]);
           }
           if (ok) tc_commit(&bars->lin_done);
@@ -319,10 +360,24 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     float l = 0.f;
     bool ok = true;
 
+    // block ids of this group's next step are fetched one step ahead, off the critical path
+    int nb0 = 0, nb1 = 0;
+    if (grp < nsteps) {
+      nb0 = sel[2 * grp];
+      nb1 = (2 * grp + 1 < cnt) ? sel[2 * grp + 1] : 0;
+    }
+#pragma unroll 1
     for (int j = grp; j < nsteps; j += 2) {
+      int blk0 = nb0, blk1 = nb1;
+      if (j + 2 < nsteps) {
+        nb0 = sel[2 * (j + 2)];
+        nb1 = (2 * (j + 2) + 1 < cnt) ? sel[2 * (j + 2) + 1] : 0;
+      }
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 0);
       ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[grp], (j >> 1) & 1, bars, p.status));
       if (!ok) break;
       tc_fence_after();
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 1);
       const int npg = min(2, cnt - 2 * j);
       const int n = npg * kBlock;
       uint32_t sr[128];
@@ -332,12 +387,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tmem_ld32(s_tmem + 64, reinterpret_cast<uint32_t(&)[32]>(sr[64]));
         tmem_ld32(s_tmem + 96, reinterpret_cast<uint32_t(&)[32]>(sr[96]));
       }
-      int blk0 = sel[2 * j], blk1 = npg > 1 ? sel[2 * j + 1] : 0;
       if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
       if (blk1 < 0 || blk1 >= p.n_blocks) blk1 = 0;
       const int64_t last_blk = blk0 > blk1 ? blk0 : blk1;
       const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > tile_vis_end);
       tc_wait_ld();
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 2);
       if (need_mask) {
         // visible keys per page: columns [0, lim) of the page's 64
         const int lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
@@ -349,10 +404,17 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (!valid) sr[c] = 0xff800000u;  // -inf
         }
       }
-      float m_new = fmaxf(__uint_as_float(sr[0]), __uint_as_float(sr[1]));
+      // row maximum: four independent chains
+      float mx[4];
 #pragma unroll
-      for (int c = 2; c < 128; c += 2)
-        m_new = fmax3(m_new, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+      for (int q = 0; q < 4; ++q) mx[q] = fmaxf(__uint_as_float(sr[32 * q]), __uint_as_float(sr[32 * q + 1]));
+#pragma unroll
+      for (int c = 2; c < 32; c += 2)
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          mx[q] = fmax3(mx[q], __uint_as_float(sr[32 * q + c]), __uint_as_float(sr[32 * q + c + 1]));
+      const float m_new = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 3);
       // lazy rescale: move the reference maximum only when it would grow by more than 2^8
       float factor = 1.f;
       if (m_used == -INFINITY) {
@@ -365,7 +427,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // O of this group is quiescent here: its previous P V completed before this step's scores
       // were committed, and its next P V waits for the P written below
       if (j >= 2 && __any_sync(0xffffffffu, factor != 1.f)) {
-#pragma unroll
+#pragma unroll 1
         for (int c0 = 0; c0 < D; c0 += 32) {
           uint32_t o[32];
           tmem_ld32(o_tmem + c0, o);
@@ -377,22 +439,31 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       const float moff = (m_used == -INFINITY) ? 0.f : m_used * sl2;
       const uint64_t s2 = pack2(sl2, sl2), t2 = pack2(-moff, -moff);
-      float lsum0 = 0.f, lsum1 = 0.f;
+      uint64_t acc0 = 0, acc1 = 0;  // two packed fp32 pairs of partial row sums
 #pragma unroll
-      for (int c = 0; c < 128; c += 2) {
-        float x0, x1;
+      for (int c = 0; c < 128; c += 4) {
+        float x0, x1, x2, x3;
         ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), s2, t2);
-        const float p0 = ex2(x0), p1 = ex2(x1);
-        lsum0 += p0;
-        lsum1 += p1;
+        ffma2(x2, x3, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]), s2, t2);
+        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+        acc0 = fadd2(acc0, pack2(p0, p1));
+        acc1 = fadd2(acc1, pack2(p2, p3));
         sr[c >> 1] = pack_bf16(p0, p1);
+        sr[(c >> 1) + 1] = pack_bf16(p2, p3);
       }
-      l += lsum0 + lsum1;
+      {
+        float a, b, c2, d2;
+        unpack2(acc0, a, b);
+        unpack2(acc1, c2, d2);
+        l += (a + b) + (c2 + d2);
+      }
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 4);
       tmem_st32(s_tmem, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
       if (n == 128) tmem_st32(s_tmem + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->p_full[grp]);
+      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 5);
     }
 
     // ---------------------------------------------------------------- epilogue
@@ -400,6 +471,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
       tc_fence_after();
     }
+    if (quad == 0) HSA_T(3002 + grp);
     // this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D)
     constexpr int HC = D / 2;
     const int cbase = grp * HC;
@@ -409,10 +481,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // partial denominator phi(q) . z over the same dims
       ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
       const uint8_t* qrow = smem + L::kQ + r * 128;
-      const float* z = p.z + static_cast<size_t>(h) * D;
+      const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
       uint32_t fr[HC / 2];
 #pragma unroll
       for (int c16 = 0; c16 < HC / 8; ++c16) {
+        const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
+        const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
         const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
         const int dh = cc >> 3, ch = cc & 7;
         const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
@@ -425,8 +499,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
           fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
           const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
-          den_part = fmaf(rr.x, z[cbase + c16 * 8 + 2 * i], den_part);
-          den_part = fmaf(rr.y, z[cbase + c16 * 8 + 2 * i + 1], den_part);
+          den_part = fmaf(rr.x, z[2 * i], den_part);
+          den_part = fmaf(rr.y, z[2 * i + 1], den_part);
         }
       }
       if constexpr (D == 128) {
@@ -442,6 +516,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     stats[(grp * 128 + r) * 4 + 0] = m_used;
     stats[(grp * 128 + r) * 4 + 1] = l;
     stats[(grp * 128 + r) * 4 + 2] = den_part;
+    if (quad == 0) HSA_T(3004 + grp);
     named_bar_sync(1, 256);
     const float m_o = stats[((grp ^ 1) * 128 + r) * 4 + 0];
     const float l_o = stats[((grp ^ 1) * 128 + r) * 4 + 1];
@@ -459,6 +534,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
       tc_fence_after();
     }
+    if (quad == 0) HSA_T(3006 + grp);
     if (ok) {  // warp-uniform: the TMEM loads below are warp-collective
       const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
       float lin_den = den;
@@ -473,60 +549,69 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
       const __nv_bfloat16* gs =
           (wr && p.g_sp) ? p.g_sp + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
+      const int g_ds = static_cast<int>(p.g_ds);
+      const bool sig = p.gate_act == 1;
+      // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
 #pragma unroll 1
-      for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
-        uint32_t oa[32], ob[32], ln[32];
-        if (has_a) tmem_ld32(tmem + lane_off + kColO + c0, oa);
-        if (has_b) tmem_ld32(tmem + lane_off + kColO + 128 + c0, ob);
-        if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
+      for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
+        uint32_t oa[16], ob[16], ln[16];
+        if (has_a) tmem_ld16(tmem + lane_off + kColO + c0, oa);
+        if (has_b) tmem_ld16(tmem + lane_off + kColO + 128 + c0, ob);
+        if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
         tc_wait_ld();
-        uint32_t packed[16];
+        uint32_t packed[8];
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
+        for (int i = 0; i < 16; i += 2) {
           float res[2];
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const int c = c0 + i + e;
             float osp = 0.f;
             if (has_a) osp = __uint_as_float(oa[i + e]) * w_a;
             if (has_b) osp = fmaf(__uint_as_float(ob[i + e]), w_b, osp);
             float olin = 0.f;
             if (p.do_linear) {
               float num = __uint_as_float(ln[i + e]);
-              if (lnum) num += lnum[c];
+              if (lnum) num += lnum[c0 + i + e];
               olin = num * inv_den;
             }
-            float wl = 1.f, ws = 1.f;
             if (gl) {
-              wl = __bfloat162float(gl[static_cast<size_t>(c) * p.g_ds]);
-              if (p.gate_act == 1) wl = 1.f / (1.f + __expf(-wl));
+              float wl = __bfloat162float(gl[(c0 + i + e) * g_ds]);
+              if (sig) wl = __fdividef(1.f, 1.f + __expf(-wl));
+              olin *= wl;
             }
             if (gs) {
-              ws = __bfloat162float(gs[static_cast<size_t>(c) * p.g_ds]);
-              if (p.gate_act == 1) ws = 1.f / (1.f + __expf(-ws));
+              float ws = __bfloat162float(gs[(c0 + i + e) * g_ds]);
+              if (sig) ws = __fdividef(1.f, 1.f + __expf(-ws));
+              osp *= ws;
             }
-            res[e] = wl * olin + ws * osp;
+            res[e] = olin + osp;
           }
           packed[i >> 1] = pack_bf16(res[0], res[1]);
         }
         if (wr) {
-#pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4)
-            *reinterpret_cast<uint4*>(orow + c0 + v4 * 8) =
-                make_uint4(packed[v4 * 4], packed[v4 * 4 + 1], packed[v4 * 4 + 2], packed[v4 * 4 + 3]);
+          *reinterpret_cast<uint4*>(orow + c0) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
         }
       }
     }
   }
 
+  if (warp == 4 || warp == 8) HSA_T(3008 + (warp == 8));
   // ------------------------------------------------------------------- common exit
   tc_fence_before();
   __syncthreads();
+  if (warp == 4) HSA_T(3010);
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
 }
+
+#ifdef HSA_TIMING
+extern "C" int hsa_debug_read_timing(long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_hsa_timing, sizeof(long long) * n));
+}
+#endif
 
 cudaError_t forward_init() {
   cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128>,
