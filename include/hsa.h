@@ -160,6 +160,13 @@ int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksu
 /* Synchronises the device, reads and clears the status word: HSA_OK or a DEVICE_* code. */
 int hsa_device_status(hsa_ctx* ctx, int32_t* status_out);
 
+/* Synchronises the device, reads and clears a counter: the number of (query tile, head) work
+ * items since the last read whose softmax had to be redone with a running maximum because a
+ * later key block outscored the first block of the tile by more than about 2^47 (the normal
+ * pass fixes the exponent reference once per tile; results are the same, the redo only costs
+ * time).  Informational. */
+int hsa_safe_pass_tiles(hsa_ctx* ctx, int64_t* count_out);
+
 /* Last CUDA error code recorded by a failing call on this context (0 if none). */
 int hsa_last_cuda_error(hsa_ctx* ctx);
 

@@ -2,18 +2,24 @@
 //
 // One CTA per (128-row query tile, head), 384 threads in three warpgroups:
 //   warp 0       TMA producer: Q tile, then the selected K/V pages gathered through the page
-//                table (two 64-token pages = 128 keys per step) into a 3-stage ring, then the
+//                table (two 64-token pages = 128 keys per step) into two 3-stage rings, then the
 //                hi/lo halves of the linear state; also owns the TMEM allocation
-//   warp 1       tcgen05.mma issuer: S = Q K^T, O += P V with P read from TMEM, then the linear
-//                numerator phi(Q) S
-//   warps 4..7   softmax group A: the even KV steps     } one query row per thread; each group
-//   warps 8..11  softmax group B: the odd KV steps      } keeps its own running max / sum and
-//                                                         its own O accumulator in TMEM
-// The two groups never talk during the loop: while one exponentiates step j the tensor cores run
-// Q K^T of a later step and P V of the other group's step.  The two partial results of a row
-// are merged (log-sum-exp) in the epilogue, which also applies the linear branch and the gates
-// and stores bf16 once.  TMEM: S_A | S_B | O_A | O_B (128 fp32 columns each); P overwrites the
-// first 64 columns of its S buffer as packed bf16.
+//   warp 1       tcgen05.mma issuer: S = Q K^T three steps ahead, O += P V with P read from
+//                TMEM, then the linear numerator phi(Q) S
+//   warps 4..11  two softmax groups of four warps: group g takes the KV steps j = g (mod 2);
+//                one query row per thread
+// TMEM: O (128 fp32 columns) | three S buffers (128 columns each); P overwrites the first 64
+// columns of its S buffer as packed bf16.  With three score buffers the tensor pipe never waits
+// for a softmax group: Q K^T of step j+3 is issued right after P V of step j.
+//
+// Both groups accumulate into ONE O.  That needs a common exponent reference per row, so in the
+// normal ("fast") pass the reference is fixed once: the row maximum of the first step plus a
+// headroom of 2^20.  Every later weight is exp2(s - ref) with no running maximum and no rescale.
+// fp32 / bf16 carry the same relative precision at any magnitude, so the result equals the
+// usual online softmax as long as no weight overflows; a step whose weights exceed 2^27 sets a
+// flag and the tile is redone in a "safe" pass: one group, classic online softmax with lazy
+// rescale.  The two groups' partial row sums are added in the epilogue, which also applies the
+// linear branch and the gates and stores bf16 once.
 // Every barrier wait is bounded; when one gives up the kernel records a timeout in the status
 // word and all roles drain to the common exit.
 #include <cuda_bf16.h>
@@ -25,13 +31,24 @@ namespace hsa {
 
 namespace {
 
-constexpr int kThreads = 384;
-constexpr int kStages = 3;
+#ifndef HSA_GROUPS
+#define HSA_GROUPS 2
+#endif
+#ifndef HSA_SMREGS
+#define HSA_SMREGS 224
+#endif
+constexpr int kGroups = HSA_GROUPS;  // softmax groups; group g takes the KV steps j = g (mod kGroups)
+constexpr bool kTokens = false;       // serialise the groups' exponential phases (2 groups only)
+constexpr int kThreads = 128 + 128 * kGroups;
+constexpr int kStages = 3;   // K ring and V ring depth
+constexpr int kSBufs = 3;    // score buffers in TMEM
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;      // + 128 * group
-constexpr uint32_t kColO = 256;    // + 128 * group
-constexpr uint32_t kColLin = 0;    // linear numerator accumulator (after the loop)
-constexpr uint32_t kColPhi = 128;  // phi(Q) as a bf16 A operand (after the loop)
+constexpr uint32_t kColO = 0;
+constexpr uint32_t kColS = 128;    // + 128 * buffer
+constexpr uint32_t kColPhi = 128;  // phi(Q) as a bf16 A operand (after the loop: buffer 0)
+constexpr uint32_t kColLin = 256;  // linear numerator accumulator (after the loop: buffer 1)
+constexpr float kHeadroom = 20.f;  // log2 units below 1 at which the first step's maximum sits
+constexpr float kRedoSum = 134217728.f;  // 2^27: a step's row sum above this forces the safe pass
 
 template <int D>
 struct Smem {
@@ -42,20 +59,39 @@ struct Smem {
   static constexpr int kV = kTile + kStages * kTile;
   static constexpr int kStats = kK;  // float[2][128][4], reuses K stage 0 once the loop is over
   static constexpr int kBars = kTile + 2 * kStages * kTile;
-  static constexpr int kTotal = kBars + 256 + 1024;  // + alignment slack
+  static constexpr int kTotal = kBars + 1024 + 1024;  // barriers + per-row reference, + slack
 };
 
 struct Bars {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2];
-  uint64_t p_full[2];
+  uint64_t s_full[kSBufs];
+  uint64_t p_full[kSBufs];
+  uint64_t pv_done;
   uint64_t o_done;
+  uint64_t mref_ready;
+  uint64_t tok[2];  // exponential-phase token: the two softmax groups take turns on the SFU
   uint64_t lin_a_full;
   uint64_t lin_done;
   uint32_t tmem_base;
   volatile int abort_flag;
+  volatile int redo;
+  float mref[128];  // per-row exponent reference (log2 domain) of the fast pass
 };
+static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory slot");
+
+#ifdef HSA_TIMING
+__device__ long long g_hsa_timing[4096];
+#define HSA_T(slot)                                                      \
+  do {                                                                   \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (slot) < 4096) \
+      g_hsa_timing[(slot)] = clock64();                                  \
+  } while (0)
+#else
+#define HSA_T(slot) \
+  do {              \
+  } while (0)
+#endif
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
@@ -81,17 +117,6 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b
   }
 }
 
-#ifdef HSA_TIMING
-__device__ long long g_hsa_timing[4096];
-#define HSA_T(slot)                                                                  \
-  do {                                                                               \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (slot) < 4096)             \
-      g_hsa_timing[(slot)] = clock64();                                              \
-  } while (0)
-#else
-#define HSA_T(slot) do { } while (0)
-#endif
-
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -107,24 +132,47 @@ __device__ __forceinline__ uint64_t pack2(float a, float b) {
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
   return r;
 }
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
 // (a0, a1) * s2 + t2 on the packed fp32 pipe
 __device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, uint64_t s2,
                                       uint64_t t2) {
   uint64_t d;
   const uint64_t a = pack2(a0, a1);
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(s2), "l"(t2));
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+  unpack2(d, d0, d1);
 }
 __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
   uint64_t d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ void init_barriers(Bars* bars) {
+  mbar_init(&bars->q_full, 1);
+  for (int s = 0; s < kStages; ++s) {
+    mbar_init(&bars->k_full[s], 1);
+    mbar_init(&bars->k_empty[s], 1);
+    mbar_init(&bars->v_full[s], 1);
+    mbar_init(&bars->v_empty[s], 1);
+  }
+  for (int i = 0; i < kSBufs; ++i) {
+    mbar_init(&bars->s_full[i], 1);
+    mbar_init(&bars->p_full[i], 128);
+  }
+  mbar_init(&bars->pv_done, 1);
+  mbar_init(&bars->o_done, 1);
+  mbar_init(&bars->mref_ready, 128);  // group 0 publishes the per-row reference
+  mbar_init(&bars->tok[0], 128);
+  mbar_init(&bars->tok[1], 128);
+  mbar_init(&bars->lin_a_full, 256);
+  mbar_init(&bars->lin_done, 1);
+  bars->redo = 0;
+  fence_mbar_init();
 }
 
 }  // namespace
@@ -140,7 +188,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   Bars* bars = reinterpret_cast<Bars*>(smem + L::kBars);
-  float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][m, l, den, -]
+  float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][l, den, -, -]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp == 4) HSA_T(3000);
@@ -153,22 +201,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int nsteps = (cnt + 1) / 2;
 
   if (threadIdx.x == 0) {
-    mbar_init(&bars->q_full, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&bars->k_full[s], 1);
-      mbar_init(&bars->k_empty[s], 1);
-      mbar_init(&bars->v_full[s], 1);
-      mbar_init(&bars->v_empty[s], 1);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars->s_full[i], 1);
-      mbar_init(&bars->p_full[i], 128);
-    }
-    mbar_init(&bars->o_done, 1);
-    mbar_init(&bars->lin_a_full, 256);
-    mbar_init(&bars->lin_done, 1);
     bars->abort_flag = 0;
-    fence_mbar_init();
+    init_barriers(bars);
   }
   if (warp == 0) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
@@ -180,8 +214,28 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const uint32_t tmem = bars->tmem_base;
   if (warp == 4) HSA_T(3001);
 
+  // attempt 0: fast pass (fixed exponent reference); attempt 1 only if a step overflowed: safe
+  // pass.  Both role branches run the same attempt loop and meet at the same CTA-wide barriers.
+  bool safe = false;
+  auto end_of_attempt = [&]() -> bool {  // true: run the safe pass next
+    tc_fence_before();
+    __syncthreads();
+    if (safe || bars->redo == 0 || bars->abort_flag) return false;
+    // a fast-pass step overflowed its fixed reference: every barrier starts over
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      init_barriers(bars);
+      atomicAdd(p.status + 1, 1);  // informational: tiles that needed the safe pass
+    }
+    __syncthreads();
+    tc_fence_after();
+    return true;
+  };
+
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+#pragma unroll 1
+    for (int attempt = 0; attempt < 2; ++attempt) {
     if (warp == 0) {
       // ================================================================= TMA producer
       if (elect_one_sync()) {
@@ -193,36 +247,41 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, h, row0);
         bool ok = true;
         int armed_k = 0, armed_v = 0;  // loads issued per ring, for the drain on abort
-#pragma unroll 1
-        for (int j = 0; j < nsteps && ok; ++j) {
+        auto page_row = [&](int idx) -> int32_t {
+          int blk = sel[idx];
+          if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
+            atomicCAS(p.status, 0, kDevBounds);
+            blk = 0;
+          }
+          return (p.page_table[blk] * p.H + h) * kBlock;
+        };
+        auto load_kv = [&](int j, bool is_k) -> bool {
           const int s = j % kStages;
           const uint32_t ph = (j / kStages) & 1;
           const int npg = min(2, cnt - 2 * j);
-          int32_t ycoord[2];
-          for (int pg = 0; pg < npg; ++pg) {
-            int blk = sel[2 * j + pg];
-            if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
-              atomicCAS(p.status, 0, kDevBounds);
-              blk = 0;
-            }
-            ycoord[pg] = (p.page_table[blk] * p.H + h) * kBlock;
-          }
-          ok = wait_bar(&bars->k_empty[s], ph ^ 1, bars, p.status);
-          if (!ok) break;
-          mbar_expect_tx(&bars->k_full[s], npg * kBlock * D * 2);
+          uint64_t* full = is_k ? &bars->k_full[s] : &bars->v_full[s];
+          uint64_t* empty = is_k ? &bars->k_empty[s] : &bars->v_empty[s];
+          uint8_t* dst = smem + (is_k ? L::kK : L::kV) + s * L::kTile;
+          const void* tm = is_k ? static_cast<const void*>(&tm_k) : static_cast<const void*>(&tm_v);
+          int32_t y[2] = {0, 0};
+          for (int pg = 0; pg < npg; ++pg) y[pg] = page_row(2 * j + pg);
+          if (!wait_bar(empty, ph ^ 1, bars, p.status)) return false;
+          mbar_expect_tx(full, npg * kBlock * D * 2);
           for (int pg = 0; pg < npg; ++pg)
             for (int dh = 0; dh < DH; ++dh)
-              tma_load_2d(smem + L::kK + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_k,
-                          &bars->k_full[s], dh * 64, ycoord[pg]);
-          ++armed_k;
-          ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
-          if (!ok) break;
-          mbar_expect_tx(&bars->v_full[s], npg * kBlock * D * 2);
-          for (int pg = 0; pg < npg; ++pg)
-            for (int dh = 0; dh < DH; ++dh)
-              tma_load_2d(smem + L::kV + s * L::kTile + dh * L::kHalf + pg * (kBlock * 128), &tm_v,
-                          &bars->v_full[s], dh * 64, ycoord[pg]);
-          ++armed_v;
+              tma_load_2d(dst + dh * L::kHalf + pg * (kBlock * 128), tm, full, dh * 64, y[pg]);
+          if (is_k)
+            ++armed_k;
+          else
+            ++armed_v;
+          return true;
+        };
+        // K runs three steps ahead of V: the scores of step j+3 are issued right after P V of j
+        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = load_kv(j, true);
+#pragma unroll 1
+        for (int j = 0; j < nsteps && ok; ++j) {
+          ok = load_kv(j, false);
+          if (ok && j + kSBufs < nsteps) ok = load_kv(j + kSBufs, true);
         }
         if (ok && p.do_linear) {
           // hi and lo halves of the D x D state ride the V ring as two more "steps"
@@ -266,7 +325,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
           tc_fence_after();
           const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::kK + s * L::kTile), 16);
-          const uint32_t d_tmem = tmem + kColS + 128 * (j & 1);
+          const uint32_t d_tmem = tmem + kColS + 128 * (j % kSBufs);
           if (cnt - 2 * j >= 2) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 0, 0);
 #pragma unroll
@@ -283,16 +342,16 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
           }
           tc_commit(&bars->k_empty[s]);
-          tc_commit(&bars->s_full[j & 1]);
+          tc_commit(&bars->s_full[j % kSBufs]);
           return true;
         };
-        if (ok && nsteps > 0) ok = issue_qk(0);
-        if (ok && nsteps > 1) ok = issue_qk(1);
+        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = issue_qk(j);
 #pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
+          const int b = j % kSBufs;
           HSA_T(2048 + j * 8 + 0);
-          ok = wait_bar(&bars->p_full[j & 1], (j >> 1) & 1, bars, p.status);
+          ok = wait_bar(&bars->p_full[b], (j / kSBufs) & 1, bars, p.status);
           if (!ok) break;
           HSA_T(2048 + j * 8 + 1);
           ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
@@ -301,9 +360,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           HSA_T(2048 + j * 8 + 2);
           constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
           const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
-          const uint32_t o_acc = tmem + kColO + 128 * (j & 1);
-          const uint32_t p_op = tmem + kColS + 128 * (j & 1);
-          const uint32_t acc0 = j >= 2 ? 1u : 0u;
+          const uint32_t o_acc = tmem + kColO;
+          const uint32_t p_op = tmem + kColS + 128 * b;
+          const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, kk > 0 ? 1u : acc0);
@@ -313,10 +372,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, 1u);
           }
           tc_commit(&bars->v_empty[s]);
+          tc_commit(&bars->pv_done);
           HSA_T(2048 + j * 8 + 3);
-          // the next scores of this group overwrite the P just consumed: issued after the P V
-          // above, the tensor pipe runs them in order
-          if (j + 2 < nsteps) ok = issue_qk(j + 2);
+          // the scores of step j+3 overwrite the P just consumed: issued after the P V above,
+          // the tensor pipe runs them in order
+          if (j + kSBufs < nsteps) ok = issue_qk(j + kSBufs);
           HSA_T(2048 + j * 8 + 4);
         }
         if (ok) tc_commit(&bars->o_done);
@@ -340,266 +400,325 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
       }
     }
+      if (!end_of_attempt()) break;
+      safe = true;
+    }
   } else {
-    // ================================================================= softmax groups + epilogue
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-    const int grp = (warp - 4) >> 2;                 // 0: even steps, 1: odd steps
-    const int quad = warp & 3;                       // TMEM lane quadrant this warp may access
-    const int r = quad * 32 + lane;                  // row inside the tile
-    const int row = row0 + r;                        // query index inside the chunk
-    const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
-    const uint32_t s_tmem = tmem + lane_off + kColS + 128 * grp;
-    const uint32_t o_tmem = tmem + lane_off + kColO + 128 * grp;
-    const int64_t qpos = p.q_pos0 + row;
-    const int64_t vis_end = p.causal ? min64(p.n_tokens, qpos + 1) : p.n_tokens;
-    // the first row of the tile sees the fewest keys: a step whose pages all end at or before
-    // that row's limit needs no masking
-    const int64_t tile_vis_end = p.causal ? min64(p.n_tokens, p.q_pos0 + row0 + 1) : p.n_tokens;
-    const float sl2 = p.scale_log2;
-    float m_used = -INFINITY;  // reference maximum the stored exponents are relative to (raw)
-    float l = 0.f;
-    bool ok = true;
-
-    // block ids of this group's next step are fetched one step ahead, off the critical path
-    int nb0 = 0, nb1 = 0;
-    if (grp < nsteps) {
-      nb0 = sel[2 * grp];
-      nb1 = (2 * grp + 1 < cnt) ? sel[2 * grp + 1] : 0;
-    }
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(HSA_SMREGS));
 #pragma unroll 1
-    for (int j = grp; j < nsteps; j += 2) {
-      int blk0 = nb0, blk1 = nb1;
-      if (j + 2 < nsteps) {
-        nb0 = sel[2 * (j + 2)];
-        nb1 = (2 * (j + 2) + 1 < cnt) ? sel[2 * (j + 2) + 1] : 0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      // ================================================================= softmax groups + epilogue
+      const int grp = (warp - 4) >> 2;  // group g takes the steps j = g (mod 3)
+      const int quad = warp & 3;        // TMEM lane quadrant this warp may access
+      const int r = quad * 32 + lane;   // row inside the tile
+      const int row = row0 + r;         // query index inside the chunk
+      const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+      const uint32_t o_tmem = tmem + lane_off + kColO;
+      const int64_t qpos = p.q_pos0 + row;
+      const int64_t vis_end = p.causal ? min64(p.n_tokens, qpos + 1) : p.n_tokens;
+      // the first row of the tile sees the fewest keys: a step whose pages all end at or before
+      // that row's limit needs no masking
+      const int64_t tile_vis_end = p.causal ? min64(p.n_tokens, p.q_pos0 + row0 + 1) : p.n_tokens;
+      const float sl2 = p.scale_log2;
+      // fast pass: t_ref is the fixed exponent reference (log2 domain) of the row;
+      // safe pass: m_used is the running reference maximum (raw score units) with lazy rescale
+      float t_ref = 0.f;
+      float m_used = -INFINITY;
+      float l = 0.f;
+      bool ok = true;
+      const int first = safe ? (grp == 0 ? 0 : nsteps) : grp;
+      const int stride = safe ? 1 : kGroups;
+
+      // block ids of the next step are fetched one step ahead, off the critical path
+      int nb0 = 0, nb1 = 0;
+      if (first < nsteps) {
+        nb0 = sel[2 * first];
+        nb1 = (2 * first + 1 < cnt) ? sel[2 * first + 1] : 0;
       }
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 0);
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[grp], (j >> 1) & 1, bars, p.status));
-      if (!ok) break;
-      tc_fence_after();
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 1);
-      const int npg = min(2, cnt - 2 * j);
-      const int n = npg * kBlock;
-      uint32_t sr[128];
-      tmem_ld32(s_tmem + 0, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
-      tmem_ld32(s_tmem + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
-      if (n == 128) {
-        tmem_ld32(s_tmem + 64, reinterpret_cast<uint32_t(&)[32]>(sr[64]));
-        tmem_ld32(s_tmem + 96, reinterpret_cast<uint32_t(&)[32]>(sr[96]));
-      }
-      if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
-      if (blk1 < 0 || blk1 >= p.n_blocks) blk1 = 0;
-      const int64_t last_blk = blk0 > blk1 ? blk0 : blk1;
-      const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > tile_vis_end);
-      tc_wait_ld();
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 2);
-      if (need_mask) {
+      // fast pass: the two groups alternate on the exponential phase.  Both are bound by the same
+      // SFU pipe there, so running the phases one after the other costs nothing and lets each
+      // group's loads, stores and barrier traffic hide under the other's exponentials.
+      if (kTokens && !safe && grp == 1) mbar_arrive(&bars->tok[0]);
+      int tok_i = 0;
+#pragma unroll 1
+      for (int j = first; j < nsteps; j += stride) {
+        int blk0 = nb0, blk1 = nb1;
+        if (j + stride < nsteps) {
+          nb0 = sel[2 * (j + stride)];
+          nb1 = (2 * (j + stride) + 1 < cnt) ? sel[2 * (j + stride) + 1] : 0;
+        }
+        const int b = j % kSBufs;
+        const uint32_t s_tmem = tmem + lane_off + kColS + 128 * b;
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 0);
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], (j / kSBufs) & 1, bars, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 1);
+        const int npg = min(2, cnt - 2 * j);
+        const int n = npg * kBlock;
+        if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
+        if (blk1 < 0 || blk1 >= p.n_blocks) blk1 = 0;
+        const int64_t last_blk = blk0 > blk1 ? blk0 : blk1;
+        const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > tile_vis_end);
         // visible keys per page: columns [0, lim) of the page's 64
-        const int lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
-        const int lim1 =
-            npg > 1 ? static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk1) * kBlock))) : 0;
-#pragma unroll
-        for (int c = 0; c < 128; ++c) {
-          const bool valid = (c & 63) < ((c >> 6) ? lim1 : lim0);
-          if (!valid) sr[c] = 0xff800000u;  // -inf
+        int lim0 = kBlock, lim1 = kBlock;
+        if (need_mask) {
+          lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
+          lim1 = npg > 1 ? static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk1) * kBlock))) : 0;
         }
-      }
-      // row maximum: four independent chains
-      float mx[4];
+        uint32_t cbuf[2][32];  // two 32-column chunks of the score row in flight
+        const int nchunks = n / 32;
+        if (safe || j == 0) {
+          // the reference needs the row maximum first: a pass over the score row in chunks
+          float mxa = -INFINITY, mxb = -INFINITY;
+          tmem_ld32(s_tmem, cbuf[0]);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) mx[q] = fmaxf(__uint_as_float(sr[32 * q]), __uint_as_float(sr[32 * q + 1]));
+          for (int c = 0; c < 4; ++c) {
+            if (c < nchunks) {
+              tc_wait_ld();
+              if (c + 1 < nchunks) tmem_ld32(s_tmem + 32 * (c + 1), cbuf[(c + 1) & 1]);
+              uint32_t(&x)[32] = cbuf[c & 1];
+              if (need_mask) {
+                const int lim = ((c >> 1) ? lim1 : lim0) - (c & 1) * 32;
 #pragma unroll
-      for (int c = 2; c < 32; c += 2)
+                for (int i = 0; i < 32; ++i)
+                  if (i >= lim) x[i] = 0xff800000u;  // -inf
+              }
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          mx[q] = fmax3(mx[q], __uint_as_float(sr[32 * q + c]), __uint_as_float(sr[32 * q + c + 1]));
-      const float m_new = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 3);
-      // lazy rescale: move the reference maximum only when it would grow by more than 2^8
-      float factor = 1.f;
-      if (m_used == -INFINITY) {
-        m_used = m_new;  // nothing accumulated so far (O and l are zero or not yet written)
-      } else if ((m_new - m_used) * sl2 > 8.f) {
-        factor = ex2((m_used - m_new) * sl2);
-        l *= factor;
-        m_used = m_new;
-      }
-      // O of this group is quiescent here: its previous P V completed before this step's scores
-      // were committed, and its next P V waits for the P written below
-      if (j >= 2 && __any_sync(0xffffffffu, factor != 1.f)) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < D; c0 += 32) {
-          uint32_t o[32];
-          tmem_ld32(o_tmem + c0, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-          tmem_st32(o_tmem + c0, o);
-        }
-      }
-      const float moff = (m_used == -INFINITY) ? 0.f : m_used * sl2;
-      const uint64_t s2 = pack2(sl2, sl2), t2 = pack2(-moff, -moff);
-      uint64_t acc0 = 0, acc1 = 0;  // two packed fp32 pairs of partial row sums
-#pragma unroll
-      for (int c = 0; c < 128; c += 4) {
-        float x0, x1, x2, x3;
-        ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), s2, t2);
-        ffma2(x2, x3, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]), s2, t2);
-        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-        acc0 = fadd2(acc0, pack2(p0, p1));
-        acc1 = fadd2(acc1, pack2(p2, p3));
-        sr[c >> 1] = pack_bf16(p0, p1);
-        sr[(c >> 1) + 1] = pack_bf16(p2, p3);
-      }
-      {
-        float a, b, c2, d2;
-        unpack2(acc0, a, b);
-        unpack2(acc1, c2, d2);
-        l += (a + b) + (c2 + d2);
-      }
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 4);
-      tmem_st32(s_tmem, reinterpret_cast<uint32_t(&)[32]>(sr[0]));
-      if (n == 128) tmem_st32(s_tmem + 32, reinterpret_cast<uint32_t(&)[32]>(sr[32]));
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bars->p_full[grp]);
-      if (quad == 0) HSA_T(grp * 1024 + (j >> 1) * 8 + 5);
-    }
-
-    // ---------------------------------------------------------------- epilogue
-    if (ok && nsteps > 0) {
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
-      tc_fence_after();
-    }
-    if (quad == 0) HSA_T(3002 + grp);
-    // this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D)
-    constexpr int HC = D / 2;
-    const int cbase = grp * HC;
-    float den_part = 0.f;
-    if (ok && p.do_linear) {
-      // phi(q) of this thread's row for its half of the dims -> bf16 A operand in TMEM;
-      // partial denominator phi(q) . z over the same dims
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
-      const uint8_t* qrow = smem + L::kQ + r * 128;
-      const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
-      uint32_t fr[HC / 2];
-#pragma unroll
-      for (int c16 = 0; c16 < HC / 8; ++c16) {
-        const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
-        const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
-        const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
-        const int dh = cc >> 3, ch = cc & 7;
-        const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
-        const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 f = __bfloat1622float2(q2[i]);
-          const float a0 = f.x > 0.f ? f.x + 1.f : __expf(f.x);
-          const float a1 = f.y > 0.f ? f.y + 1.f : __expf(f.y);
-          const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
-          fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
-          const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
-          den_part = fmaf(rr.x, z[2 * i], den_part);
-          den_part = fmaf(rr.y, z[2 * i + 1], den_part);
-        }
-      }
-      if constexpr (D == 128) {
-        tmem_st32(tmem + lane_off + kColPhi + grp * 32, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
-      } else {
-        tmem_st16(tmem + lane_off + kColPhi + grp * 16, reinterpret_cast<uint32_t(&)[16]>(fr[0]));
-      }
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bars->lin_a_full);
-    }
-    // publish this group's row statistics, then read the other group's
-    stats[(grp * 128 + r) * 4 + 0] = m_used;
-    stats[(grp * 128 + r) * 4 + 1] = l;
-    stats[(grp * 128 + r) * 4 + 2] = den_part;
-    if (quad == 0) HSA_T(3004 + grp);
-    named_bar_sync(1, 256);
-    const float m_o = stats[((grp ^ 1) * 128 + r) * 4 + 0];
-    const float l_o = stats[((grp ^ 1) * 128 + r) * 4 + 1];
-    const float den = den_part + stats[((grp ^ 1) * 128 + r) * 4 + 2];
-    // log-sum-exp merge of the two partial softmax results of this row
-    const float mm = fmaxf(m_used, m_o);
-    const float c_me = (m_used == -INFINITY) ? 0.f : ex2((m_used - mm) * sl2);
-    const float c_ot = (m_o == -INFINITY) ? 0.f : ex2((m_o - mm) * sl2);
-    const float lsum = l * c_me + l_o * c_ot;
-    const float inv_l = lsum > 0.f ? 1.f / lsum : 0.f;
-    const float w_a = (grp == 0 ? c_me : c_ot) * inv_l;  // weight of accumulator A
-    const float w_b = (grp == 0 ? c_ot : c_me) * inv_l;  // weight of accumulator B
-    const bool has_a = nsteps > 0, has_b = nsteps > 1;
-    if (ok && p.do_linear) {
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
-      tc_fence_after();
-    }
-    if (quad == 0) HSA_T(3006 + grp);
-    if (ok) {  // warp-uniform: the TMEM loads below are warp-collective
-      const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
-      float lin_den = den;
-      const float* lnum = nullptr;
-      if (wr && p.do_linear && p.lin_num != nullptr) {
-        lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D;
-        lin_den += p.lin_den[static_cast<size_t>(row) * p.H + h];
-      }
-      const float inv_den = (p.do_linear && lin_den > 0.f) ? 1.f / lin_den : 0.f;
-      __nv_bfloat16* orow = p.out + static_cast<size_t>(row) * p.o_ts + static_cast<size_t>(h) * p.o_hs;
-      const __nv_bfloat16* gl =
-          (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
-      const __nv_bfloat16* gs =
-          (wr && p.g_sp) ? p.g_sp + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
-      const int g_ds = static_cast<int>(p.g_ds);
-      const bool sig = p.gate_act == 1;
-      // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
-#pragma unroll 1
-      for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
-        uint32_t oa[16], ob[16], ln[16];
-        if (has_a) tmem_ld16(tmem + lane_off + kColO + c0, oa);
-        if (has_b) tmem_ld16(tmem + lane_off + kColO + 128 + c0, ob);
-        if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
-        tc_wait_ld();
-        uint32_t packed[8];
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-          float res[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            float osp = 0.f;
-            if (has_a) osp = __uint_as_float(oa[i + e]) * w_a;
-            if (has_b) osp = fmaf(__uint_as_float(ob[i + e]), w_b, osp);
-            float olin = 0.f;
-            if (p.do_linear) {
-              float num = __uint_as_float(ln[i + e]);
-              if (lnum) num += lnum[c0 + i + e];
-              olin = num * inv_den;
+              for (int i = 0; i < 32; i += 4) {
+                mxa = fmax3(mxa, __uint_as_float(x[i]), __uint_as_float(x[i + 1]));
+                mxb = fmax3(mxb, __uint_as_float(x[i + 2]), __uint_as_float(x[i + 3]));
+              }
             }
-            if (gl) {
-              float wl = __bfloat162float(gl[(c0 + i + e) * g_ds]);
-              if (sig) wl = __fdividef(1.f, 1.f + __expf(-wl));
-              olin *= wl;
-            }
-            if (gs) {
-              float ws = __bfloat162float(gs[(c0 + i + e) * g_ds]);
-              if (sig) ws = __fdividef(1.f, 1.f + __expf(-ws));
-              osp *= ws;
-            }
-            res[e] = olin + osp;
           }
-          packed[i >> 1] = pack_bf16(res[0], res[1]);
+          const float m_new = fmaxf(mxa, mxb);
+          if (!safe) {
+            // fix the row's reference for the whole tile and hand it to the other group
+            t_ref = (m_new == -INFINITY) ? 0.f : fmaf(m_new, sl2, kHeadroom);
+            bars->mref[r] = t_ref;
+            mbar_arrive(&bars->mref_ready);
+          } else {
+            // lazy rescale: move the reference only when it would grow by more than 2^8
+            float factor = 1.f;
+            if (m_used == -INFINITY) {
+              m_used = m_new;  // nothing accumulated so far
+            } else if ((m_new - m_used) * sl2 > 8.f) {
+              factor = ex2((m_used - m_new) * sl2);
+              l *= factor;
+              m_used = m_new;
+            }
+            if (j > 0) {
+              // O must be quiescent: the previous P V has to be complete before it is rescaled
+              ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (j - 1) & 1, bars, p.status));
+              if (!ok) break;
+              tc_fence_after();
+              if (__any_sync(0xffffffffu, factor != 1.f)) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                  uint32_t o[32];
+                  tmem_ld32(o_tmem + c0, o);
+                  tc_wait_ld();
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                  tmem_st32(o_tmem + c0, o);
+                }
+                tc_wait_st();
+              }
+            }
+            t_ref = (m_used == -INFINITY) ? 0.f : m_used * sl2;
+          }
+        } else if (j < kGroups) {
+          // first step of groups 1 and 2 in the fast pass: take the reference group 0 fixed
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready, 0, bars, p.status));
+          if (!ok) break;
+          t_ref = bars->mref[r];
         }
-        if (wr) {
-          *reinterpret_cast<uint4*>(orow + c0) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 2);
+        // exponentials in four chunks of 32 columns: the load of the next chunk and the store of
+        // the previous P chunk run under the arithmetic of the current one
+        const float nt = -t_ref;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
+        tmem_ld32(s_tmem, cbuf[0]);
+        if (kTokens && !safe) {
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->tok[grp], tok_i & 1, bars, p.status));
+          if (!ok) break;
+          ++tok_i;
+        }
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 3);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (c < nchunks) {
+            tc_wait_ld();
+            if (c + 1 < nchunks) tmem_ld32(s_tmem + 32 * (c + 1), cbuf[(c + 1) & 1]);
+            uint32_t(&x)[32] = cbuf[c & 1];
+            if (need_mask) {
+              const int lim = ((c >> 1) ? lim1 : lim0) - (c & 1) * 32;  // visible columns of this chunk
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i >= lim) x[i] = 0xff800000u;  // -inf
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const float p0 = ex2(fmaf(__uint_as_float(x[i]), sl2, nt));
+              const float p1 = ex2(fmaf(__uint_as_float(x[i + 1]), sl2, nt));
+              const float p2 = ex2(fmaf(__uint_as_float(x[i + 2]), sl2, nt));
+              const float p3 = ex2(fmaf(__uint_as_float(x[i + 3]), sl2, nt));
+              acc[0] += p0;
+              acc[1] += p1;
+              acc[2] += p2;
+              acc[3] += p3;
+              pk[i >> 1] = pack_bf16(p0, p1);
+              pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+            }
+            tmem_st16(s_tmem + 16 * c, pk);
+            if (quad == 0) HSA_T(3100 + grp * 256 + (j / kGroups) * 8 + c);
+          }
+        }
+        {
+          const float lstep = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          l += lstep;
+          // a weight far above the fixed reference: finite here, but the tile is redone safely
+          if (!safe && !(lstep <= kRedoSum)) bars->redo = 1;
+        }
+        if (kTokens && !safe) mbar_arrive(&bars->tok[grp ^ 1]);
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 4);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->p_full[b]);
+        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 5);
+      }
+
+      // ---------------------------------------------------------------- epilogue
+      // this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D)
+      // (groups 0 and 1 share the epilogue; group 2 only contributes its partial row sum)
+      constexpr int HC = D / 2;
+      const bool epi = grp < 2;
+      const int cbase = (grp & 1) * HC;
+      float den_part = 0.f;
+      uint32_t fr[HC / 2];
+      if (ok && p.do_linear && epi) {
+        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
+        // MMA) and the partial denominator phi(q) . z -- computed while the last P V drains
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
+        const uint8_t* qrow = smem + L::kQ + r * 128;
+        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
+#pragma unroll
+        for (int c16 = 0; c16 < HC / 8; ++c16) {
+          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
+          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
+          const int dh = cc >> 3, ch = cc & 7;
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
+          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(q2[i]);
+            const float a0 = f.x > 0.f ? f.x + 1.f : __expf(f.x);
+            const float a1 = f.y > 0.f ? f.y + 1.f : __expf(f.y);
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
+            fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
+            const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
+            den_part = fmaf(rr.x, z[2 * i], den_part);
+            den_part = fmaf(rr.y, z[2 * i + 1], den_part);
+          }
         }
       }
+      if (ok && nsteps > 0) {
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
+        tc_fence_after();
+      }
+      if (quad == 0) HSA_T(3002 + grp);
+      if (ok && p.do_linear && epi) {
+        if constexpr (D == 128) {
+          tmem_st32(tmem + lane_off + kColPhi + grp * 32, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
+        } else {
+          tmem_st16(tmem + lane_off + kColPhi + grp * 16, reinterpret_cast<uint32_t(&)[16]>(fr[0]));
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->lin_a_full);
+      }
+      // publish this group's partial row sum and denominator, then read the other group's
+      stats[(grp * 128 + r) * 4 + 0] = l;
+      stats[(grp * 128 + r) * 4 + 1] = den_part;
+      if (quad == 0) HSA_T(3004 + grp);
+      named_bar_sync(1, 128 * kGroups);
+      float lsum = 0.f, den = 0.f;
+#pragma unroll
+      for (int gg = 0; gg < kGroups; ++gg) {
+        lsum += stats[(gg * 128 + r) * 4 + 0];
+        den += stats[(gg * 128 + r) * 4 + 1];
+      }
+      const float inv_l = (nsteps > 0 && lsum > 0.f) ? 1.f / lsum : 0.f;
+      const bool has_o = nsteps > 0;
+      if (ok && p.do_linear && epi) {
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
+        tc_fence_after();
+      }
+      if (quad == 0) HSA_T(3006 + grp);
+      if (ok && epi) {  // warp-uniform: the TMEM loads below are warp-collective
+        const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
+        float lin_den = den;
+        const float* lnum = nullptr;
+        if (wr && p.do_linear && p.lin_num != nullptr) {
+          lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D;
+          lin_den += p.lin_den[static_cast<size_t>(row) * p.H + h];
+        }
+        const float inv_den = (p.do_linear && lin_den > 0.f) ? 1.f / lin_den : 0.f;
+        __nv_bfloat16* orow = p.out + static_cast<size_t>(row) * p.o_ts + static_cast<size_t>(h) * p.o_hs;
+        const __nv_bfloat16* gl =
+            (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
+        const __nv_bfloat16* gs =
+            (wr && p.g_sp) ? p.g_sp + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
+        const int g_ds = static_cast<int>(p.g_ds);
+        const bool sig = p.gate_act == 1;
+        // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
+#pragma unroll 1
+        for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
+          uint32_t oa[16], ln[16];
+          if (has_o) tmem_ld16(o_tmem + c0, oa);
+          if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
+          tc_wait_ld();
+          uint32_t packed[8];
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            float res[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float osp = has_o ? __uint_as_float(oa[i + e]) * inv_l : 0.f;
+              float olin = 0.f;
+              if (p.do_linear) {
+                float num = __uint_as_float(ln[i + e]);
+                if (lnum) num += lnum[c0 + i + e];
+                olin = num * inv_den;
+              }
+              if (gl) {
+                float wl = __bfloat162float(gl[(c0 + i + e) * g_ds]);
+                if (sig) wl = __fdividef(1.f, 1.f + __expf(-wl));
+                olin *= wl;
+              }
+              if (gs) {
+                float ws = __bfloat162float(gs[(c0 + i + e) * g_ds]);
+                if (sig) ws = __fdividef(1.f, 1.f + __expf(-ws));
+                osp *= ws;
+              }
+              res[e] = olin + osp;
+            }
+            packed[i >> 1] = pack_bf16(res[0], res[1]);
+          }
+          if (wr) {
+            *reinterpret_cast<uint4*>(orow + c0) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+          }
+        }
+      }
+      if (quad == 0) HSA_T(3008 + grp);
+      if (!end_of_attempt()) break;
+      safe = true;
     }
   }
 
-  if (warp == 4 || warp == 8) HSA_T(3008 + (warp == 8));
-  // ------------------------------------------------------------------- common exit
-  tc_fence_before();
-  __syncthreads();
   if (warp == 4) HSA_T(3010);
   if (warp == 0) {
     tc_fence_after();

@@ -415,6 +415,19 @@ int hsa_device_status(hsa_ctx* ctx, int32_t* status_out) {
   return HSA_OK;
 }
 
+int hsa_safe_pass_tiles(hsa_ctx* ctx, int64_t* count_out) {
+  if (!ctx || !count_out) return HSA_ERR_INVALID_ARG;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  int32_t v = 0;
+  e = cudaMemcpy(&v, ws + ctx->lay.status + 4, 4, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess && v != 0) e = cudaMemset(ws + ctx->lay.status + 4, 0, 4);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  *count_out = v;
+  return HSA_OK;
+}
+
 int hsa_last_cuda_error(hsa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 int hsa_destroy(hsa_ctx* ctx) {

@@ -36,7 +36,8 @@ TILE_M = 128
 
 EXPORTS = [
     "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_forward",
-    "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_last_cuda_error",
+    "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
+    "hsa_last_cuda_error",
     "hsa_destroy", "hsa_status_string",
 ]
 
@@ -76,6 +77,7 @@ def _load() -> C.CDLL:
     lib.hsa_state_layout.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t),
                                      C.POINTER(C.c_size_t)]
     lib.hsa_device_status.argtypes = [vp, C.POINTER(i32)]
+    lib.hsa_safe_pass_tiles.argtypes = [vp, C.POINTER(i64)]
     lib.hsa_last_cuda_error.argtypes = [vp]
     lib.hsa_destroy.argtypes = [vp]
     lib.hsa_status_string.argtypes = [C.c_int]
@@ -194,6 +196,12 @@ def hsa_device_status(ctx: int) -> int:
     return s.value
 
 
+def hsa_safe_pass_tiles(ctx: int) -> int:
+    n = C.c_int64()
+    _check(_lib.hsa_safe_pass_tiles(ctx, C.byref(n)), "hsa_safe_pass_tiles")
+    return n.value
+
+
 def hsa_last_cuda_error(ctx: int) -> int:
     return _lib.hsa_last_cuda_error(ctx)
 
@@ -285,6 +293,9 @@ class HSAContext:
 
     def device_status(self) -> int:
         return hsa_device_status(self.ctx)
+
+    def safe_pass_tiles(self) -> int:
+        return hsa_safe_pass_tiles(self.ctx)
 
     def destroy(self) -> None:
         if getattr(self, "ctx", None):
