@@ -126,6 +126,32 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
                       const int32_t* budgets_dev, int32_t q_group_tokens,
                       int32_t* sel_idx_dev, int32_t* sel_cnt_dev, void* stream);
 
+/* Block selection for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a convenience of this library).  Some callers run where cudaMalloc is off limits --
+ * inside a region being captured into a CUDA graph, in a process whose memory pool is owned by
+ * another framework, or in a service that forbids allocation after start-up -- and cannot
+ * provide the context's workspace either.  This entry point computes exactly what
+ * hsa_select_blocks computes for q_group_tokens = 0 (one selection per head for the whole chunk),
+ * needs no context, and keeps its scratch (query partial sums and score keys, about 1 MiB) in a
+ * fixed array inside the library: every GPU that loads the library holds that array until the
+ * process exits.
+ *   ksum_dev                  device fp32 [H][ksum_head_stride_blocks][d]: per-(head, block) key
+ *                             sums as hsa_append_kv maintains them (see hsa_state_layout)
+ *   status_dev                device int32 status word, or NULL to use one inside the scratch
+ * Limits (HSA_ERR_OUT_OF_PAGES beyond them): ceil(n_q/128) * H * d <= 131072,
+ * H * ksum_head_stride_blocks <= 131072, ceil(n_tokens/64) <= 51200.
+ * It calls no allocator (no cudaMalloc / cudaFree, no library routine that allocates).  The first
+ * call on a device looks up the device address of the scratch array (with that device current);
+ * make that first call before any stream capture begins.  All calls share the one array, which
+ * keeps the previous call's contents: two calls whose kernels may overlap on the GPU (different
+ * streams, or different threads) race on it -- serialise them. */
+int hsa_select_blocks_noalloc(const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                              int32_t num_heads, int32_t head_dim, const float* ksum_dev,
+                              int32_t ksum_head_stride_blocks, int64_t n_tokens, int64_t q_pos0,
+                              int32_t causal, float softmax_scale, const int32_t* budgets_dev,
+                              int32_t max_topk, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
+                              int32_t* status_dev, void* stream);
+
 /* out[i,h,:] = w(g_lin) * O_lin + w(g_sp) * O_sp  (Section 3.3, Eq. 5), where
  *   O_sp  = softmax attention of query i over the visible keys of the selected blocks
  *           (Eq. 4 with the block mask; Appendix A.1),

@@ -4,6 +4,9 @@
 // query partial sums -> scores (many CTAs) -> top-k (one CTA per head and group).
 #include <cuda_bf16.h>
 
+#include <cmath>
+#include <mutex>
+
 #include "hsa_internal.h"
 
 namespace hsa {
@@ -253,3 +256,91 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
 }
 
 }  // namespace hsa
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant of the block selection (no context, no caller workspace).
+// Its scratch -- the per-tile query partial sums and the score keys -- lives in a fixed array
+// that is part of the library image.  Every GPU that loads the library carries that array
+// until the process exits, and all calls share it.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kNoAllocQpartFloats = 64 * 2048;   // up to 64 query tiles x (heads * dim <= 2048)
+constexpr size_t kNoAllocKeys = 128 * 1024;         // heads * blocks <= 131072
+constexpr size_t kNoAllocScratchBytes = 256 + kNoAllocQpartFloats * 4 + kNoAllocKeys * 4;
+static __device__ __align__(256) unsigned char g_select_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_dev_ptr[kMaxDevices] = {nullptr};
+
+// The array's name is only a host-side handle; the device address has to be looked up, once per
+// device and with that device current.
+int scratch_pointer(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HSA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_dev_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_select_scratch) != cudaSuccess || ptr == nullptr) return HSA_ERR_CUDA;
+    g_scratch_dev_ptr[dev] = ptr;
+  }
+  *out = g_scratch_dev_ptr[dev];
+  return HSA_OK;
+}
+
+}  // namespace
+
+extern "C" int hsa_select_blocks_noalloc(const void* q, int32_t n_q, int64_t tok_stride,
+                                         int64_t head_stride, int32_t num_heads, int32_t head_dim,
+                                         const float* ksum_dev, int32_t ksum_head_stride_blocks,
+                                         int64_t n_tokens, int64_t q_pos0, int32_t causal,
+                                         float softmax_scale, const int32_t* budgets_dev,
+                                         int32_t max_topk, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
+                                         int32_t* status_dev, void* stream) {
+  using namespace hsa;
+  if (!q || !ksum_dev || !budgets_dev || !sel_idx_dev || !sel_cnt_dev) return HSA_ERR_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return HSA_ERR_INVALID_ARG;
+  if (num_heads < 1 || n_q < 1 || max_topk < 1 || n_tokens < 0) return HSA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) % 16) != 0 || tok_stride < head_dim || head_stride < head_dim ||
+      (tok_stride % 8) != 0 || (head_stride % 8) != 0)
+    return HSA_ERR_INVALID_ARG;
+  const int64_t nblk = (n_tokens + kBlock - 1) / kBlock;
+  if (ksum_head_stride_blocks < nblk) return HSA_ERR_INVALID_ARG;
+  // fixed scratch: refuse anything that does not fit
+  const int64_t n_tiles = (static_cast<int64_t>(n_q) + kTileM - 1) / kTileM;
+  if (n_tiles * num_heads * head_dim > static_cast<int64_t>(kNoAllocQpartFloats) ||
+      static_cast<int64_t>(num_heads) * ksum_head_stride_blocks > static_cast<int64_t>(kNoAllocKeys) ||
+      nblk * 4 > 200 * 1024)
+    return HSA_ERR_OUT_OF_PAGES;
+  void* base = nullptr;
+  const int rc = scratch_pointer(&base);
+  if (rc != HSA_OK) return rc;
+  unsigned char* sc = static_cast<unsigned char*>(base);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the first 256 bytes hold a status word for callers that pass none: it has to start at zero
+  if (!status_dev && cudaMemsetAsync(sc, 0, 256, st) != cudaSuccess) return HSA_ERR_CUDA;
+  SelectArgs a{};
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.n_q = n_q;
+  a.tok_stride = tok_stride;
+  a.head_stride = head_stride;
+  a.q_pos0 = q_pos0;
+  a.causal = causal != 0;
+  a.n_tokens = n_tokens;
+  a.H = num_heads;
+  a.D = head_dim;
+  a.max_pages = ksum_head_stride_blocks;
+  a.ksum = ksum_dev;
+  a.budgets = budgets_dev;
+  a.group_tokens = 0;
+  a.n_groups = 1;
+  a.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(head_dim));
+  a.qpart = reinterpret_cast<float*>(sc + 256);
+  a.keys = reinterpret_cast<uint32_t*>(sc + 256 + kNoAllocQpartFloats * 4);
+  a.sel_idx = sel_idx_dev;
+  a.sel_cnt = sel_cnt_dev;
+  a.kcap = max_topk;
+  a.status = status_dev ? status_dev : reinterpret_cast<int32_t*>(sc);
+  return launch_select(a, st) == cudaSuccess ? HSA_OK : HSA_ERR_CUDA;
+}

@@ -35,7 +35,8 @@ PAGE_TOKENS = 64
 TILE_M = 128
 
 EXPORTS = [
-    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_forward",
+    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_noalloc",
+    "hsa_forward",
     "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
     "hsa_last_cuda_error",
     "hsa_destroy", "hsa_status_string",
@@ -70,6 +71,8 @@ def _load() -> C.CDLL:
     lib.hsa_create.argtypes = [C.POINTER(vp), C.POINTER(hsa_config), C.POINTER(hsa_buffers), vp]
     lib.hsa_append_kv.argtypes = [vp, vp, vp, i32, i64, i64, vp]
     lib.hsa_select_blocks.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp, vp]
+    lib.hsa_select_blocks_noalloc.argtypes = [vp, i32, i64, i64, i32, i32, vp, i32, i64, i64, i32, C.c_float,
+                                              vp, i32, vp, vp, vp, vp]
     lib.hsa_forward.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, vp, i32, vp, vp, i64, i64, i64,
                                 vp, i64, i64, u32, vp]
     lib.hsa_get_info.argtypes = [vp, C.POINTER(i64), C.POINTER(i32)]
@@ -152,6 +155,21 @@ def hsa_select_blocks(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budg
     _check(_lib.hsa_select_blocks(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
                                   budgets.data_ptr(), int(q_group_tokens), sel_idx.data_ptr(),
                                   sel_cnt.data_ptr(), _stream()), "hsa_select_blocks")
+
+
+def hsa_select_blocks_noalloc(q: torch.Tensor, ksum: torch.Tensor, n_tokens: int, q_pos0: int, causal: bool,
+                              softmax_scale: float, budgets: torch.Tensor, sel_idx: torch.Tensor,
+                              sel_cnt: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    """Allocation-free selection: ksum is the fp32 [H, blocks, d] key-sum view of a context's state
+    (or any tensor of that layout); sel_idx is int32 [H, 1, max_topk], sel_cnt int32 [H, 1]."""
+    ts, hs = _thd(q, "q")
+    if ksum.dtype != torch.float32 or ksum.dim() != 3 or not ksum.is_contiguous():
+        raise ValueError("ksum: expected a contiguous CUDA fp32 [H, blocks, d] tensor")
+    _check(_lib.hsa_select_blocks_noalloc(q.data_ptr(), q.shape[0], ts, hs, q.shape[1], q.shape[2],
+                                          ksum.data_ptr(), ksum.shape[1], int(n_tokens), int(q_pos0),
+                                          int(causal), float(softmax_scale), budgets.data_ptr(),
+                                          sel_idx.shape[-1], sel_idx.data_ptr(), sel_cnt.data_ptr(),
+                                          _ptr(status), _stream()), "hsa_select_blocks_noalloc")
 
 
 def hsa_forward(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, sel_idx: Optional[torch.Tensor],
