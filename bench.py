@@ -31,6 +31,9 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_34606_b200 import workloads as W  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one hsa_forward_kernel<128> launch on cfg2, from the
+# ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.44 MB + 0.58 MB)
+NCU_TRAFFIC_BYTES = {"cfg2": 41.02e6}
 METRIC = "hsa_effective_tflops"
 UNIT = "TFLOP/s"
 RING = 4  # distinct (q, k, v, out) input sets rotated between steps (> L2 in total)
@@ -279,7 +282,8 @@ def bench_ours(args, rank: int, world: int):
             "device_status": status,
             "roofline": {"kernel": "hsa_forward_kernel<128>", "bound": "tensor", "achieved": fwd_tf,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tf / peaks["bf16_tflops"],
-                         "traffic": None, "peak_source": peaks["source"] + " (burst)",
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": by["forward"],
+                         "peak_source": peaks["source"] + " (burst)",
                          "frac_of_sustained": fwd_tf / peaks["bf16_tflops_sustained"],
                          "append_hbm_frac": by["append"] / stage[0] / 1e6 / peaks["hbm_gbs"],
                          "select_hbm_frac": by["select"] / stage[1] / 1e6 / peaks["hbm_gbs"]},
