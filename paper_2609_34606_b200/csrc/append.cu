@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "hsa_internal.h"
+#include "ptx.cuh"
 
 namespace hsa {
 
@@ -195,23 +196,274 @@ __global__ void state_reduce_kernel(AppendArgs a) {
   }
 }
 
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t st) {
+// ---------------------------------------------------------------------------------------
+// Fused append for head_dim 128 (the measured path): one pass over the chunk's K and V.
+// grid (nsplit, H); a CTA owns a run of consecutive history blocks of one head and, per block,
+//   * copies the new rows into the block's page (and zero-fills the rest of a partial tail page),
+//   * adds their column sums to the block's key sum,
+//   * stages phi(K) (as bf16 hi + lo, so that hi + lo carries ~16 bits) and V in shared memory in
+//     the 128-byte-swizzled MN-major layout and lets the tensor cores accumulate
+//       S_part (128 x 128, fp32 in TMEM) += phi(K)_hi^T V + phi(K)_lo^T V
+//     over the block's tokens (tcgen05, K = tokens), double-buffered against the next block's
+//     loads,
+// and finally writes its partial S and partial z for the fixed-order reduction of stage C.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kAfTile = 64 * 128 * 2;        // [64 tokens x 128 dims] bf16 = two swizzled slabs
+constexpr int kAfStage = 3 * kAfTile;        // phi hi | phi lo | V
+constexpr int kAfRed = 16 * 128 * 4;         // key-sum partials of one block
+constexpr int kAfSmem = 2 * kAfStage + 2 * kAfRed + 64 + 1024;
+
+struct AfBars {
+  uint64_t mma_done[2];
+  uint64_t all_done;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
+
+__device__ __forceinline__ bool af_wait(uint64_t* bar, uint32_t parity, AfBars* bars, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t i = 1; i < (1u << 24); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 0u && bars->abort_flag) return false;
+  }
+  bars->abort_flag = 1;
+  atomicCAS(status, 0, kDevTimeout);
+  return false;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int blocks_per_cta) {
+  constexpr int D = 128;
+  extern __shared__ uint8_t af_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(af_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  float* red = reinterpret_cast<float*>(smem + 2 * kAfStage);            // [2][16][128]
+  AfBars* bars = reinterpret_cast<AfBars*>(smem + 2 * kAfStage + 2 * kAfRed);
+
+  const int h = blockIdx.y, split = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ch = threadIdx.x & 15;   // 16-byte chunk of a row (8 dims)
+  const int rg = threadIdx.x >> 4;   // row group: rows rg, rg+16, rg+32, rg+48 of a block
+  const int64_t b_first = a.n0 / kBlock, b_last = (a.n0 + a.n_new - 1) / kBlock;
+  const int64_t bs = b_first + static_cast<int64_t>(split) * blocks_per_cta;
+  const int64_t be = min64(b_last + 1, bs + blocks_per_cta);
+  const int nblk = static_cast<int>(max64(0, be - bs));
+  const int64_t n_end = a.n0 + a.n_new;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->mma_done[0], 1);
+    mbar_init(&bars->mma_done[1], 1);
+    mbar_init(&bars->all_done, 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  uint4 kreg[4], vreg[4];
+  auto load_block = [&](int64_t b, uint4 (&kk)[4], uint4 (&vv)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t t = b * kBlock + rg + 16 * i;
+      if (t >= a.n0 && t < n_end) {
+        const size_t src = static_cast<size_t>(t - a.n0) * a.tok_stride +
+                           static_cast<size_t>(h) * a.head_stride + ch * 8;
+        kk[i] = *reinterpret_cast<const uint4*>(a.k + src);
+        vv[i] = *reinterpret_cast<const uint4*>(a.v + src);
+      } else {
+        kk[i] = make_uint4(0, 0, 0, 0);
+        vv[i] = make_uint4(0, 0, 0, 0);
+      }
+    }
+  };
+  if (nblk > 0) load_block(bs, kreg, vreg);
+
+  float zacc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) zacc[e] = 0.f;
+  bool ok = true;
+
+#pragma unroll 1
+  for (int bi = 0; bi < nblk; ++bi) {
+    const int64_t b = bs + bi;
+    const int stage = bi & 1;
+    uint8_t* st_hi = smem + stage * kAfStage;
+    uint8_t* st_lo = st_hi + kAfTile;
+    uint8_t* st_v = st_lo + kAfTile;
+    float* my_red = red + stage * (16 * 128);
+    uint4 knext[4], vnext[4];
+    if (bi + 1 < nblk) load_block(b + 1, knext, vnext);  // next block's loads fly under this one
+    // the tensor cores must be done with this stage's previous tiles (block bi - 2)
+    if (bi >= 2) ok = af_wait(&bars->mma_done[stage], ((bi >> 1) - 1) & 1, bars, a.status) && ok;
+    const int page = a.page_table[b];
+    const size_t row_base = (static_cast<size_t>(page) * a.H + h) * kBlock;
+    float ks[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ks[e] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = rg + 16 * i;
+      const int64_t t = b * kBlock + r;
+      const bool fresh = t >= a.n0 && t < n_end;
+      const uint32_t soff = (ch >> 3) * (kAfTile / 2) + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+      uint4 hi4 = make_uint4(0, 0, 0, 0), lo4 = make_uint4(0, 0, 0, 0);
+      if (fresh) {
+        const size_t dst = (row_base + r) * D + ch * 8;
+        *reinterpret_cast<uint4*>(a.k_pool + dst) = kreg[i];
+        *reinterpret_cast<uint4*>(a.v_pool + dst) = vreg[i];
+        const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kreg[i]);
+        uint32_t hw[4], lw[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(k2[e]);
+          ks[2 * e] += f.x;
+          ks[2 * e + 1] += f.y;
+          const float p0 = phi_elu1(f.x), p1 = phi_elu1(f.y);
+          zacc[2 * e] += p0;
+          zacc[2 * e + 1] += p1;
+          const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+          const float2 hf = __bfloat1622float2(hh);
+          const __nv_bfloat162 ll = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+          hw[e] = *reinterpret_cast<const uint32_t*>(&hh);
+          lw[e] = *reinterpret_cast<const uint32_t*>(&ll);
+        }
+        hi4 = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        lo4 = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+      } else if (t >= n_end) {
+        // rows of the partial tail page past the last token: keep the pool free of garbage
+        const size_t dst = (row_base + r) * D + ch * 8;
+        *reinterpret_cast<uint4*>(a.k_pool + dst) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(a.v_pool + dst) = make_uint4(0, 0, 0, 0);
+      }
+      *reinterpret_cast<uint4*>(st_hi + soff) = hi4;
+      *reinterpret_cast<uint4*>(st_lo + soff) = lo4;
+      *reinterpret_cast<uint4*>(st_v + soff) = fresh ? vreg[i] : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) my_red[rg * 128 + ch * 8 + e] = ks[e];
+    fence_proxy_async_smem();  // generic-proxy writes above -> visible to the tensor cores
+    __syncthreads();
+    if (warp == 0) {
+      if (elect_one_sync() && ok) {
+        tc_fence_after();
+        constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 1, 1);
+        constexpr uint32_t hi = desc_hi_sw128(1024);
+        const uint32_t a_hi = desc_lo_sw128(smem_u32(st_hi), kAfTile / 2);
+        const uint32_t a_lo = desc_lo_sw128(smem_u32(st_lo), kAfTile / 2);
+        const uint32_t b_v = desc_lo_sw128(smem_u32(st_v), kAfTile / 2);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_ss_lo(tmem, a_hi + kk * 128, b_v + kk * 128, hi, idesc, (bi > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) tc_mma_ss_lo(tmem, a_lo + kk * 128, b_v + kk * 128, hi, idesc, 1u);
+        tc_commit(&bars->mma_done[stage]);
+      }
+    } else if (threadIdx.x >= 128) {
+      // key sum of the block: fixed-order sum over the 16 row groups
+      const int c = threadIdx.x - 128;
+      float s = 0.f;
+#pragma unroll
+      for (int g2 = 0; g2 < 16; ++g2) s += my_red[g2 * 128 + c];
+      float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + c;
+      const float old = (max64(a.n0, b * kBlock) > b * kBlock) ? *dst : 0.f;  // block partly filled before
+      *dst = old + s;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      kreg[i] = knext[i];
+      vreg[i] = vnext[i];
+    }
+  }
+
+  // all tensor-core work of this CTA done?
+  if (warp == 0) {
+    if (elect_one_sync()) tc_commit(&bars->all_done);
+  }
+  ok = af_wait(&bars->all_done, 0, bars, a.status) && ok;
+  tc_fence_after();
+  float* out = a.spart + (static_cast<size_t>(h) * a.nsplit + split) * (D * D + D);
+  {
+    const int quad = warp & 3, half = warp >> 2;
+    const int row = quad * 32 + lane;
+    const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * 64;
+#pragma unroll
+    for (int c0 = 0; c0 < 64; c0 += 32) {
+      uint32_t v[32];
+      if (nblk > 0) {
+        tmem_ld32(taddr + c0, v);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = 0u;
+      }
+      float4* dst = reinterpret_cast<float4*>(out + row * D + half * 64 + c0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+    }
+  }
+  // z partial: fixed-order sum over the row groups
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[rg * 128 + ch * 8 + e] = zacc[e];
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    float s = 0.f;
+#pragma unroll
+    for (int g2 = 0; g2 < 16; ++g2) s += red[g2 * 128 + threadIdx.x];
+    out[D * D + threadIdx.x] = s;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+cudaError_t append_init() {
+  return cudaFuncSetAttribute(append_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);
+}
+
+cudaError_t launch_append(const AppendArgs& a_in, cudaStream_t st) {
+  AppendArgs a = a_in;
   const int64_t b0 = a.n0 / kBlock;
   const int64_t b1 = (a.n0 + a.n_new - 1) / kBlock;
-  dim3 gridA(static_cast<unsigned>(b1 - b0 + 1), a.H);
-  if (a.D == 128)
-    append_pool_ksum_kernel<128><<<gridA, 256, 0, st>>>(a);
-  else
-    append_pool_ksum_kernel<64><<<gridA, 256, 0, st>>>(a);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || !a.lin_state) return e;
-  dim3 gridB(a.nsplit, a.H);
-  if (a.D == 128)
-    state_partial_kernel<128><<<gridB, 256, 0, st>>>(a);
-  else
-    state_partial_kernel<64><<<gridB, 256, 0, st>>>(a);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
+  if (a.D == 128 && a.lin_state) {
+    const int nb = static_cast<int>(b1 - b0 + 1);
+    const int per = (nb + a.nsplit - 1) / a.nsplit;
+    a.nsplit = (nb + per - 1) / per;  // no empty CTAs
+    dim3 grid(a.nsplit, a.H);
+    append_fused_kernel<<<grid, 256, kAfSmem, st>>>(a, per);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  } else {
+    dim3 gridA(static_cast<unsigned>(b1 - b0 + 1), a.H);
+    if (a.D == 128)
+      append_pool_ksum_kernel<128><<<gridA, 256, 0, st>>>(a);
+    else
+      append_pool_ksum_kernel<64><<<gridA, 256, 0, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess || !a.lin_state) return e;
+    dim3 gridB(a.nsplit, a.H);
+    if (a.D == 128)
+      state_partial_kernel<128><<<gridB, 256, 0, st>>>(a);
+    else
+      state_partial_kernel<64><<<gridB, 256, 0, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
   const int n = a.D * a.D + a.D;
   dim3 gridC((n + 255) / 256, a.H);
   state_reduce_kernel<<<gridC, 256, 0, st>>>(a);

@@ -199,6 +199,7 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   if (e == cudaSuccess) e = cudaMemset(bufs->state, 0, ctx->lay.state_total);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = forward_init();
+  if (e == cudaSuccess) e = append_init();
   if (e != cudaSuccess) { delete ctx; return HSA_ERR_CUDA; }
   const int D = cfg->head_dim;
   const uint64_t pool_rows = static_cast<uint64_t>(cfg->max_pages) * cfg->num_heads * kBlock;
@@ -249,6 +250,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   if (nsplit > by_tokens) nsplit = by_tokens;
   a.nsplit = nsplit;
   a.lin_state = ctx->cfg.lin_mode == HSA_LIN_STATE;
+  a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   cudaError_t e = launch_append(a, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   ctx->n_tokens = n1;

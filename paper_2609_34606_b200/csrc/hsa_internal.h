@@ -38,6 +38,7 @@ struct AppendArgs {
   float* spart;         // [H][nsplit][D*D + D] scratch
   int nsplit;
   int lin_state;  // update the linear state?
+  int32_t* status;  // device status word
 };
 
 struct SelectArgs {
@@ -107,6 +108,7 @@ cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                            const CUtensorMap& tm_state, cudaStream_t st);
 cudaError_t launch_causal_linear(const CausalLinArgs& a, cudaStream_t st);
-cudaError_t forward_init();  // opt in to the shared-memory size the forward kernel needs
+cudaError_t forward_init();
+cudaError_t append_init();  // opt in to the shared-memory size the fused append kernel needs  // opt in to the shared-memory size the forward kernel needs
 
 }  // namespace hsa
