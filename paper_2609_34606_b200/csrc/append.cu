@@ -210,9 +210,12 @@ __global__ void state_reduce_kernel(AppendArgs a) {
 // ---------------------------------------------------------------------------------------
 namespace {
 
-constexpr int kAfTile = 64 * 128 * 2;        // [64 tokens x 128 dims] bf16 = two swizzled slabs
-constexpr int kAfStage = 3 * kAfTile;        // phi hi | phi lo | V
-constexpr int kAfRed = 16 * 128 * 4;         // key-sum partials of one block
+constexpr int kAfThreads = 512;
+constexpr int kAfRowGroups = kAfThreads / 16;   // 32: a thread handles rows rg and rg + 32 of a block
+constexpr int kAfRows = kBlock / kAfRowGroups;  // 2 rows per thread and block
+constexpr int kAfTile = 64 * 128 * 2;           // [64 tokens x 128 dims] bf16 = two swizzled slabs
+constexpr int kAfStage = 3 * kAfTile;           // phi hi | phi lo | V
+constexpr int kAfRed = kAfRowGroups * 128 * 4;  // key-sum partials of one block
 constexpr int kAfSmem = 2 * kAfStage + 2 * kAfRed + 64 + 1024;
 
 struct AfBars {
@@ -233,20 +236,23 @@ __device__ __forceinline__ bool af_wait(uint64_t* bar, uint32_t parity, AfBars* 
   return false;
 }
 
+// elu(x) + 1 with the fast exponential (relative error ~1e-6, far inside the state's tolerance)
+__device__ __forceinline__ float phi_fast(float x) { return x > 0.f ? x + 1.f : __expf(x); }
+
 }  // namespace
 
-__global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int blocks_per_cta) {
+__global__ void __launch_bounds__(kAfThreads, 1) append_fused_kernel(AppendArgs a, int blocks_per_cta) {
   constexpr int D = 128;
   extern __shared__ uint8_t af_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(af_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  float* red = reinterpret_cast<float*>(smem + 2 * kAfStage);            // [2][16][128]
+  float* red = reinterpret_cast<float*>(smem + 2 * kAfStage);  // [2][row groups][128]
   AfBars* bars = reinterpret_cast<AfBars*>(smem + 2 * kAfStage + 2 * kAfRed);
 
   const int h = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ch = threadIdx.x & 15;   // 16-byte chunk of a row (8 dims)
-  const int rg = threadIdx.x >> 4;   // row group: rows rg, rg+16, rg+32, rg+48 of a block
+  const int ch = threadIdx.x & 15;  // 16-byte chunk of a row (8 dims)
+  const int rg = threadIdx.x >> 4;  // row group
   const int64_t b_first = a.n0 / kBlock, b_last = (a.n0 + a.n_new - 1) / kBlock;
   const int64_t bs = b_first + static_cast<int64_t>(split) * blocks_per_cta;
   const int64_t be = min64(b_last + 1, bs + blocks_per_cta);
@@ -269,11 +275,11 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
-  uint4 kreg[4], vreg[4];
-  auto load_block = [&](int64_t b, uint4 (&kk)[4], uint4 (&vv)[4]) {
+  uint4 kreg[kAfRows], vreg[kAfRows];
+  auto load_block = [&](int64_t b, uint4 (&kk)[kAfRows], uint4 (&vv)[kAfRows]) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int64_t t = b * kBlock + rg + 16 * i;
+    for (int i = 0; i < kAfRows; ++i) {
+      const int64_t t = b * kBlock + rg + kAfRowGroups * i;
       if (t >= a.n0 && t < n_end) {
         const size_t src = static_cast<size_t>(t - a.n0) * a.tok_stride +
                            static_cast<size_t>(h) * a.head_stride + ch * 8;
@@ -299,8 +305,8 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
     uint8_t* st_hi = smem + stage * kAfStage;
     uint8_t* st_lo = st_hi + kAfTile;
     uint8_t* st_v = st_lo + kAfTile;
-    float* my_red = red + stage * (16 * 128);
-    uint4 knext[4], vnext[4];
+    float* my_red = red + stage * (kAfRowGroups * 128);
+    uint4 knext[kAfRows], vnext[kAfRows];
     if (bi + 1 < nblk) load_block(b + 1, knext, vnext);  // next block's loads fly under this one
     // the tensor cores must be done with this stage's previous tiles (block bi - 2)
     if (bi >= 2) ok = af_wait(&bars->mma_done[stage], ((bi >> 1) - 1) & 1, bars, a.status) && ok;
@@ -310,43 +316,38 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
 #pragma unroll
     for (int e = 0; e < 8; ++e) ks[e] = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int r = rg + 16 * i;
+    for (int i = 0; i < kAfRows; ++i) {
+      const int r = rg + kAfRowGroups * i;
       const int64_t t = b * kBlock + r;
       const bool fresh = t >= a.n0 && t < n_end;
       const uint32_t soff = (ch >> 3) * (kAfTile / 2) + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-      uint4 hi4 = make_uint4(0, 0, 0, 0), lo4 = make_uint4(0, 0, 0, 0);
-      if (fresh) {
+      // rows that are not new carry zeros (loaded as zeros above): they add nothing anywhere
+      const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kreg[i]);
+      uint32_t hw[4], lw[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(k2[e]);
+        ks[2 * e] += f.x;
+        ks[2 * e + 1] += f.y;
+        const float p0 = fresh ? phi_fast(f.x) : 0.f, p1 = fresh ? phi_fast(f.y) : 0.f;
+        zacc[2 * e] += p0;
+        zacc[2 * e + 1] += p1;
+        const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+        const float2 hf = __bfloat1622float2(hh);
+        const __nv_bfloat162 ll = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+        hw[e] = *reinterpret_cast<const uint32_t*>(&hh);
+        lw[e] = *reinterpret_cast<const uint32_t*>(&ll);
+      }
+      if (fresh || t >= n_end) {
+        // new rows go to the page; rows of a partial tail page past the last token are zeroed so
+        // that the pool never holds garbage the forward kernel could multiply by zero
         const size_t dst = (row_base + r) * D + ch * 8;
         *reinterpret_cast<uint4*>(a.k_pool + dst) = kreg[i];
         *reinterpret_cast<uint4*>(a.v_pool + dst) = vreg[i];
-        const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kreg[i]);
-        uint32_t hw[4], lw[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 f = __bfloat1622float2(k2[e]);
-          ks[2 * e] += f.x;
-          ks[2 * e + 1] += f.y;
-          const float p0 = phi_elu1(f.x), p1 = phi_elu1(f.y);
-          zacc[2 * e] += p0;
-          zacc[2 * e + 1] += p1;
-          const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-          const float2 hf = __bfloat1622float2(hh);
-          const __nv_bfloat162 ll = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
-          hw[e] = *reinterpret_cast<const uint32_t*>(&hh);
-          lw[e] = *reinterpret_cast<const uint32_t*>(&ll);
-        }
-        hi4 = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-        lo4 = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-      } else if (t >= n_end) {
-        // rows of the partial tail page past the last token: keep the pool free of garbage
-        const size_t dst = (row_base + r) * D + ch * 8;
-        *reinterpret_cast<uint4*>(a.k_pool + dst) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(a.v_pool + dst) = make_uint4(0, 0, 0, 0);
       }
-      *reinterpret_cast<uint4*>(st_hi + soff) = hi4;
-      *reinterpret_cast<uint4*>(st_lo + soff) = lo4;
-      *reinterpret_cast<uint4*>(st_v + soff) = fresh ? vreg[i] : make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(st_hi + soff) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      *reinterpret_cast<uint4*>(st_lo + soff) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+      *reinterpret_cast<uint4*>(st_v + soff) = vreg[i];
     }
 #pragma unroll
     for (int e = 0; e < 8; ++e) my_red[rg * 128 + ch * 8 + e] = ks[e];
@@ -367,18 +368,18 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
         for (int kk = 0; kk < 4; ++kk) tc_mma_ss_lo(tmem, a_lo + kk * 128, b_v + kk * 128, hi, idesc, 1u);
         tc_commit(&bars->mma_done[stage]);
       }
-    } else if (threadIdx.x >= 128) {
-      // key sum of the block: fixed-order sum over the 16 row groups
-      const int c = threadIdx.x - 128;
+    } else if (threadIdx.x >= kAfThreads - 128) {
+      // key sum of the block: fixed-order sum over the row groups
+      const int c = threadIdx.x - (kAfThreads - 128);
       float s = 0.f;
 #pragma unroll
-      for (int g2 = 0; g2 < 16; ++g2) s += my_red[g2 * 128 + c];
+      for (int g2 = 0; g2 < kAfRowGroups; ++g2) s += my_red[g2 * 128 + c];
       float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + c;
-      const float old = (max64(a.n0, b * kBlock) > b * kBlock) ? *dst : 0.f;  // block partly filled before
+      const float old = (a.n0 > b * kBlock) ? *dst : 0.f;  // block partly filled before
       *dst = old + s;
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kAfRows; ++i) {
       kreg[i] = knext[i];
       vreg[i] = vnext[i];
     }
@@ -392,25 +393,21 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
   tc_fence_after();
   float* out = a.spart + (static_cast<size_t>(h) * a.nsplit + split) * (D * D + D);
   {
-    const int quad = warp & 3, half = warp >> 2;
+    const int quad = warp & 3, part = warp >> 2;  // 16 warps: 4 lane quadrants x 4 column quarters
     const int row = quad * 32 + lane;
-    const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * 64;
+    uint32_t v[32];
+    if (nblk > 0) {
+      tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + part * 32, v);
+      tc_wait_ld();
+    } else {
 #pragma unroll
-    for (int c0 = 0; c0 < 64; c0 += 32) {
-      uint32_t v[32];
-      if (nblk > 0) {
-        tmem_ld32(taddr + c0, v);
-        tc_wait_ld();
-      } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = 0u;
-      }
-      float4* dst = reinterpret_cast<float4*>(out + row * D + half * 64 + c0);
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+      for (int i = 0; i < 32; ++i) v[i] = 0u;
     }
+    float4* dst = reinterpret_cast<float4*>(out + row * D + part * 32);
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                           __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
   }
   // z partial: fixed-order sum over the row groups
   __syncthreads();
@@ -420,7 +417,7 @@ __global__ void __launch_bounds__(256, 1) append_fused_kernel(AppendArgs a, int 
   if (threadIdx.x < 128) {
     float s = 0.f;
 #pragma unroll
-    for (int g2 = 0; g2 < 16; ++g2) s += red[g2 * 128 + threadIdx.x];
+    for (int g2 = 0; g2 < kAfRowGroups; ++g2) s += red[g2 * 128 + threadIdx.x];
     out[D * D + threadIdx.x] = s;
   }
   tc_fence_before();
@@ -445,7 +442,7 @@ cudaError_t launch_append(const AppendArgs& a_in, cudaStream_t st) {
     const int per = (nb + a.nsplit - 1) / a.nsplit;
     a.nsplit = (nb + per - 1) / per;  // no empty CTAs
     dim3 grid(a.nsplit, a.H);
-    append_fused_kernel<<<grid, 256, kAfSmem, st>>>(a, per);
+    append_fused_kernel<<<grid, kAfThreads, kAfSmem, st>>>(a, per);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   } else {

@@ -25,16 +25,25 @@ __global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
   float acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-  for (int t = tile * kTileM + rg; t < t_hi; t += RP) {
-    const size_t src =
-        static_cast<size_t>(t) * a.tok_stride + static_cast<size_t>(h) * a.head_stride + c8 * 8;
-    const uint4 qq = *reinterpret_cast<const uint4*>(a.q + src);
-    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qq);
+  // all of a thread's rows are requested before any is consumed (independent loads in flight)
+  constexpr int NR = kTileM / RP;
+  uint4 rows[NR];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __bfloat1622float2(q2[i]);
-      acc[2 * i] += f.x;
-      acc[2 * i + 1] += f.y;
+  for (int i = 0; i < NR; ++i) {
+    const int t = tile * kTileM + rg + i * RP;
+    rows[i] = make_uint4(0, 0, 0, 0);
+    if (t < t_hi)
+      rows[i] = *reinterpret_cast<const uint4*>(a.q + static_cast<size_t>(t) * a.tok_stride +
+                                                static_cast<size_t>(h) * a.head_stride + c8 * 8);
+  }
+#pragma unroll
+  for (int i = 0; i < NR; ++i) {
+    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&rows[i]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(q2[e]);
+      acc[2 * e] += f.x;
+      acc[2 * e + 1] += f.y;
     }
   }
 #pragma unroll
@@ -94,21 +103,36 @@ __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   if (threadIdx.x < D) {
     double s = 0.0;
     const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
-    for (int t = tile_lo; t < tile_hi; ++t)
-      s += static_cast<double>(a.qpart[(static_cast<size_t>(t) * a.H + h) * D + threadIdx.x]);
+    // eight independent loads in flight per trip; the sum order stays tile-ascending
+    for (int t0 = tile_lo; t0 < tile_hi; t0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        v[i] = (t0 + i < tile_hi) ? a.qpart[(static_cast<size_t>(t0 + i) * a.H + h) * D + threadIdx.x] : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += static_cast<double>(v[i]);
+    }
     qs[threadIdx.x] = s / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
   }
   __syncthreads();
   constexpr int PER = D / 32;
   uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  constexpr int NB = kScoreBlocksPerCta / 8;  // blocks per warp
+  float kv[NB][PER];
 #pragma unroll
-  for (int i = 0; i < kScoreBlocksPerCta / 8; ++i) {
+  for (int i = 0; i < NB; ++i) {
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * kScoreBlocksPerCta + i * 8 + warp;
+#pragma unroll
+    for (int e = 0; e < PER; ++e)
+      kv[i][e] = b < nblk ? a.ksum[(static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER + e] : 0.f;
+  }
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
     const int64_t b = static_cast<int64_t>(blockIdx.x) * kScoreBlocksPerCta + i * 8 + warp;
     if (b >= nblk) continue;  // warp-uniform
-    const float* ks = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER;
     double dot = 0.0;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) dot += qs[lane * PER + e] * static_cast<double>(ks[e]);
+    for (int e = 0; e < PER; ++e) dot += qs[lane * PER + e] * static_cast<double>(kv[i][e]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
     if (lane == 0) {
