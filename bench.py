@@ -137,7 +137,8 @@ def bench_ours(args, rank: int, world: int):
         dist.init_process_group("nccl", device_id=dev)
     w = W.WORKLOADS[args.workload]
     ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk),
-                         max_topk=max(w.topk, 1), page_order=W.gen_page_order(w, w.n_blocks), device=dev)
+                         max_topk=w.n_blocks if w.budget_set else max(w.topk, 1),
+                         page_order=W.gen_page_order(w, w.n_blocks), device=dev)
     for c in range(w.n_chunks - 1):
         k, v = W.gen_kv_chunk(w, c, layer=rank)
         ctx.append_kv(k.to(dev), v.to(dev))
@@ -245,12 +246,8 @@ def bench_ours(args, rank: int, world: int):
     if sampler is not None:
         sampler.stop()
 
-    ms_step = ms_total / K
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_step, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, ms_e2e = t.tolist()
+    from paper_2609_34606_b200 import sharding
+    ms_step, ms_e2e = sharding.max_over_ranks([ms_total / K, ms_e2e], device=dev)  # slowest rank
     fl = step_flops(w, sel_tokens)
     by = step_bytes(w, sel_tokens)
     peaks = load_peaks()

@@ -238,3 +238,96 @@ def test_safe_pass_when_later_blocks_dominate(cuda_device):
     assert ctx2.safe_pass_tiles() == 0 and ctx2.device_status() == 0
     ctx.destroy()
     ctx2.destroy()
+
+
+def _sampled_forward_check(w, ctx, K, V, q, device, n_random=192):
+    """Selection in full, outputs on sampled rows, for a context whose history is (K, V)."""
+    from paper_2609_34606_b200 import hsa
+    qd = q.to(device)
+    budgets = W.gen_budgets(w)
+    qn = Hn.f32(q)
+    si, sc = ctx.select_blocks(qd, budgets.to(device))
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, scores = O.select_blocks(qn, K, K.shape[0], False, budgets.tolist())
+    Hn.check_selection(sel_gpu, sel_ref, scores)
+    rows = W.sample_rows(w, n_random=n_random).numpy()
+    ref = O.hsa_forward(qn, K, V, K.shape[0], False, sel_gpu, rows=rows, linear_form="state")
+    out = Hn.f64(ctx.forward(qd, si, sc))
+    o_sp = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_LINEAR))
+    assert ctx.device_status() == 0
+    Hn.assert_close(o_sp[rows], ref["O_sp"][rows], "O_sp")
+    Hn.assert_close(out[rows], ref["out"][rows], "out")
+    assert np.isfinite(out).all()
+    return sel_gpu
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4"])
+def test_long_history_and_head_adaptive_budgets_sampled(name, cuda_device):
+    """cfg3: 280,800-token history behind a shuffled page table, top-128; cfg4: scene-segment
+    mixture with per-head budgets from {0,16,32,64,128,all}.  Selection is checked in full, the
+    state in full, outputs on the first / last query tile plus seeded rows."""
+    w = W.WORKLOADS[name]
+    ctx = Hn.build_context(w, cuda_device, max_topk=w.n_blocks if w.budget_set else w.topk)
+    Ks, Vs = [], []
+    for c in range(w.n_chunks):
+        k, v = W.gen_kv_chunk(w, c)
+        ctx.append_kv(k.to(cuda_device), v.to(cuda_device))
+        Ks.append(k.float().numpy())
+        Vs.append(v.float().numpy())
+    K, V = np.concatenate(Ks), np.concatenate(Vs)
+    del Ks, Vs
+    S_ref, z_ref = O.linear_state(K, V)
+    assert np.linalg.norm(Hn.f64(ctx.S) - S_ref) <= 1e-5 * np.linalg.norm(S_ref)
+    assert np.linalg.norm(Hn.f64(ctx.z) - z_ref) <= 1e-5 * np.linalg.norm(z_ref)
+    sel = _sampled_forward_check(w, ctx, K, V, W.gen_query(w), cuda_device)
+    if w.mixture:
+        # structure of the mixture: every head with a budget <= 128 selects inside the queries' segment
+        seg = W.query_segment(w)
+        lo, hi = seg * w.seg_chunks * w.chunk // 64, ((seg + 1) * w.seg_chunks * w.chunk + 63) // 64
+        budgets = W.gen_budgets(w).tolist()
+        for h, b in enumerate(budgets):
+            if 0 < b <= 128:
+                assert all(lo <= x <= hi for x in sel[h][0]), (h, b)
+    ctx.destroy()
+
+
+def test_rollout_steps_sampled(cuda_device):
+    """cfg5 shape: append a chunk, select, forward, 80 times on one layer's context; the oracle
+    checks the steps at chunks 0, 1, 39 and 79 (its linear state is carried along in fp64)."""
+    w = W.WORKLOADS["cfg5"]
+    layer = 29
+    ctx = Hn.build_context(w, cuda_device, max_topk=w.topk)
+    Ks, Vs = [], []
+    S = np.zeros((w.H, w.d, w.d))
+    z = np.zeros((w.H, w.d))
+    budgets = W.gen_budgets(w)
+    bd = budgets.to(cuda_device)
+    sel = ctx.alloc_selection(w.Lq)
+    for c in range(w.n_chunks):
+        k, v = W.gen_kv_chunk(w, c, layer=layer)
+        ctx.append_kv(k.to(cuda_device), v.to(cuda_device))
+        kn, vn = k.float().numpy(), v.float().numpy()
+        Ks.append(kn)
+        Vs.append(vn)
+        dS, dz = O.linear_state(kn, vn)
+        S += dS
+        z += dz
+        q = W.gen_query(w, step=c, layer=layer)
+        qd = q.to(cuda_device)
+        ctx.select_blocks(qd, bd, sel=sel)
+        out = ctx.forward(qd, sel[0], sel[1])
+        if c in (0, 1, 39, 79):
+            K, V = np.concatenate(Ks), np.concatenate(Vs)
+            qn = Hn.f32(q)
+            sel_gpu = Hn.selection_lists(sel[0], sel[1])
+            sel_ref, scores = O.select_blocks(qn, K, K.shape[0], False, budgets.tolist())
+            Hn.check_selection(sel_gpu, sel_ref, scores)
+            rows = W.sample_rows(w, n_random=64).numpy()
+            o_sp = O.sparse_branch(qn, K, V, sel_gpu, K.shape[0], False, rows=rows)
+            o_lin = O.linear_from_state(qn, S, z)
+            ref = (o_sp + o_lin)[rows]
+            Hn.assert_close(Hn.f64(out)[rows], ref, f"out@chunk{c}")
+            assert np.linalg.norm(Hn.f64(ctx.S) - S) <= 1e-5 * np.linalg.norm(S)
+            del K, V
+    assert ctx.device_status() == 0 and ctx.n_tokens == w.N
+    ctx.destroy()
