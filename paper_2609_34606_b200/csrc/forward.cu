@@ -181,7 +181,8 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v,
-                   const __grid_constant__ CUtensorMap tm_state, const FwdParams p) {
+                   const __grid_constant__ CUtensorMap tm_state,
+                   const __grid_constant__ CUtensorMap tm_out, const FwdParams p) {
   using L = Smem<D>;
   constexpr int DH = D / 64;  // 64-element (128-byte) slabs per row
   extern __shared__ uint8_t smem_raw[];
@@ -666,7 +667,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           lin_den += p.lin_den[static_cast<size_t>(row) * p.H + h];
         }
         const float inv_den = (p.do_linear && lin_den > 0.f) ? 1.f / lin_den : 0.f;
-        __nv_bfloat16* orow = p.out + static_cast<size_t>(row) * p.o_ts + static_cast<size_t>(h) * p.o_hs;
         const __nv_bfloat16* gl =
             (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
         const __nv_bfloat16* gs =
@@ -677,40 +677,72 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll 1
         for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
           uint32_t oa[16], ln[16];
+          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 0);
           if (has_o) tmem_ld16(o_tmem + c0, oa);
           if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
           tc_wait_ld();
+          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 1);
+          // gate weights and causal partials are fetched under ONE branch each per trip (a branch
+          // per element costs far more than the arithmetic it guards)
+          float wl[16], ws[16], ladd[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            wl[i] = 1.f;
+            ws[i] = 1.f;
+            ladd[i] = 0.f;
+          }
+          if (gl) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float w0 = __bfloat162float(gl[(c0 + i) * g_ds]);
+              wl[i] = sig ? __fdividef(1.f, 1.f + __expf(-w0)) : w0;
+            }
+          }
+          if (gs) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float w0 = __bfloat162float(gs[(c0 + i) * g_ds]);
+              ws[i] = sig ? __fdividef(1.f, 1.f + __expf(-w0)) : w0;
+            }
+          }
+          if (lnum) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) ladd[i] = lnum[c0 + i];
+          }
           uint32_t packed[8];
 #pragma unroll
           for (int i = 0; i < 16; i += 2) {
             float res[2];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-              float osp = has_o ? __uint_as_float(oa[i + e]) * inv_l : 0.f;
-              float olin = 0.f;
-              if (p.do_linear) {
-                float num = __uint_as_float(ln[i + e]);
-                if (lnum) num += lnum[c0 + i + e];
-                olin = num * inv_den;
-              }
-              if (gl) {
-                float wl = __bfloat162float(gl[(c0 + i + e) * g_ds]);
-                if (sig) wl = __fdividef(1.f, 1.f + __expf(-wl));
-                olin *= wl;
-              }
-              if (gs) {
-                float ws = __bfloat162float(gs[(c0 + i + e) * g_ds]);
-                if (sig) ws = __fdividef(1.f, 1.f + __expf(-ws));
-                osp *= ws;
-              }
-              res[e] = olin + osp;
+              const float osp = has_o ? __uint_as_float(oa[i + e]) * inv_l : 0.f;
+              const float olin = p.do_linear ? (__uint_as_float(ln[i + e]) + ladd[i + e]) * inv_den : 0.f;
+              res[e] = fmaf(wl[i + e], olin, ws[i + e] * osp);
             }
             packed[i >> 1] = pack_bf16(res[0], res[1]);
           }
-          if (wr) {
-            *reinterpret_cast<uint4*>(orow + c0) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 2);
+          // stage the row into the Q tile's shared memory (dead by now; each thread touches only
+          // its own row) in the 128-byte-swizzled layout the output tensor map expects
+          {
+            const int cc = c0 >> 3;  // 16-byte chunk of the row
+            uint8_t* srow = smem + L::kQ + (cc >> 3) * L::kHalf + r * 128;
+            *reinterpret_cast<uint4*>(srow + (((cc & 7) ^ (r & 7)) << 4)) =
+                make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            *reinterpret_cast<uint4*>(srow + ((((cc + 1) & 7) ^ (r & 7)) << 4)) =
+                make_uint4(packed[4], packed[5], packed[6], packed[7]);
           }
+        }
+      }
+      // both epilogue groups have staged their columns: one elected thread stores the tile
+      // (rows past the end of the chunk are clipped by the tensor map)
+      fence_proxy_async_smem();
+      named_bar_sync(2, 128 * kGroups);
+      if (ok && warp == 4) {
+        if (elect_one_sync()) {
+          for (int dh = 0; dh < DH; ++dh) tma_store_3d(&tm_out, smem + L::kQ + dh * L::kHalf, dh * 64, h, row0);
+          tma_store_commit();
+          tma_store_wait_read();  // the tile must stay in shared memory until it has been read
         }
       }
       if (quad == 0) HSA_T(3008 + grp);
@@ -741,13 +773,14 @@ cudaError_t forward_init() {
 }
 
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                           const CUtensorMap& tm_v, const CUtensorMap& tm_state, cudaStream_t st) {
+                           const CUtensorMap& tm_v, const CUtensorMap& tm_state, const CUtensorMap& tm_out,
+                           cudaStream_t st) {
   const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
   dim3 grid(n_tiles, p.H);
   if (D == 128)
-    hsa_forward_kernel<128><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, p);
+    hsa_forward_kernel<128><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
   else
-    hsa_forward_kernel<64><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, p);
+    hsa_forward_kernel<64><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
   return cudaGetLastError();
 }
 

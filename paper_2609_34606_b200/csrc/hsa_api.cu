@@ -328,6 +328,10 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   int r = encode_q(&tm_q, q, n_q, H, D, tok_stride, head_stride);
   if (r != HSA_OK) return r;
 
+  CUtensorMap tm_out;  // same geometry as q: the kernel stores whole [128 rows x 64 dims] tiles
+  r = encode_q(&tm_out, out, n_q, H, D, out_tok_stride, out_head_stride);
+  if (r != HSA_OK) return r;
+
   FwdParams p{};
   p.n_q = n_q;
   p.H = H;
@@ -377,7 +381,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     p.lin_num = c.lin_num;
     p.lin_den = c.lin_den;
   }
-  cudaError_t e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, st);
+  cudaError_t e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;
 }

@@ -106,7 +106,7 @@ cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                           const CUtensorMap& tm_state, cudaStream_t st);
+                           const CUtensorMap& tm_state, const CUtensorMap& tm_out, cudaStream_t st);
 cudaError_t launch_causal_linear(const CausalLinArgs& a, cudaStream_t st);
 cudaError_t forward_init();
 cudaError_t append_init();  // opt in to the shared-memory size the fused append kernel needs  // opt in to the shared-memory size the forward kernel needs
