@@ -225,10 +225,26 @@ def bench_ours(args, rank: int, world: int):
             p1 = time.time()
             time.sleep(0.15)
             probe = sampler.summary(p0, p1)
+    # the two ablation modes of the forward kernel, timed on their own (not part of the step)
+    def time_flags(flags, reps=20):
+        q, k, v, out = devs[0]
+        for _ in range(3):
+            ctx.forward(q, sel[0], sel[1], out=out, flags=flags)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(reps):
+            qq, _, _, oo = devs[i % RING]
+            ctx.forward(qq, sel[0], sel[1], out=oo, flags=flags)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+    ms_lin_only = time_flags(hsa.HSA_FWD_NO_SPARSE)
+    ms_sp_only = time_flags(hsa.HSA_FWD_NO_LINEAR)
     if args.profile:
         if rank == 0:
             print(json.dumps({"profile_run": True, "steps": K, "ms_per_step": ms_total / K,
-                              "stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]}}))
+                              "stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
+                              "linear_only_ms": ms_lin_only, "sparse_only_ms": ms_sp_only}))
         ctx.destroy()
         return
     # end-to-end through the same API with host buffers (H2D inputs + D2H result inside the region)
@@ -272,6 +288,8 @@ def bench_ours(args, rank: int, world: int):
             "stage_gbs": {"append": by["append"] / stage[0] / 1e6, "select": by["select"] / stage[1] / 1e6,
                           "forward": by["forward"] / stage[2] / 1e6},
             "flops_per_step": fl["total"],
+            "forward_modes_ms": {"linear_only": ms_lin_only, "sparse_only": ms_sp_only,
+                                 "linear_only_gbs": (2 * w.Lq * w.H * w.d * 2 + w.H * w.d * w.d * 4) / ms_lin_only / 1e6},
             "clocks": clocks,
             "e2e": {"value": world * tf(fl["total"], ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": 3 * w.Lq * w.H * w.d * 2, "d2h_bytes_per_step": w.Lq * w.H * w.d * 2},

@@ -430,6 +430,41 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const int first = safe ? (grp == 0 ? 0 : nsteps) : grp;
       const int stride = safe ? 1 : kGroups;
 
+      // ---- linear branch operands, prepared before the loop
+      constexpr int HC = D / 2;
+      const bool epi = grp < 2;
+      const int cbase = (grp & 1) * HC;
+      float den_part = 0.f;
+      uint32_t fr[HC / 2];
+      if (ok && p.do_linear && epi) {
+        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
+        // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
+        // and kept in registers until the epilogue
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
+        const uint8_t* qrow = smem + L::kQ + r * 128;
+        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
+#pragma unroll
+        for (int c16 = 0; c16 < HC / 8; ++c16) {
+          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
+          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
+          const int dh = cc >> 3, ch = cc & 7;
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
+          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(q2[i]);
+            const float a0 = f.x > 0.f ? f.x + 1.f : __expf(f.x);
+            const float a1 = f.y > 0.f ? f.y + 1.f : __expf(f.y);
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
+            fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
+            const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
+            den_part = fmaf(rr.x, z[2 * i], den_part);
+            den_part = fmaf(rr.y, z[2 * i + 1], den_part);
+          }
+        }
+      }
+
       // block ids of the next step are fetched one step ahead, off the critical path
       int nb0 = 0, nb1 = 0;
       if (first < nsteps) {
@@ -558,20 +593,23 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               for (int i = 0; i < 32; ++i)
                 if (i >= lim) x[i] = 0xff800000u;  // -inf
             }
-            uint32_t pk[16];
+            // stage by stage over the whole chunk, so that 32 independent operations of each kind
+            // are in flight: scale-and-shift, exponential, row sum, bf16 pack
+            float y[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] = fmaf(__uint_as_float(x[i]), sl2, nt);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] = ex2(y[i]);
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-              const float p0 = ex2(fmaf(__uint_as_float(x[i]), sl2, nt));
-              const float p1 = ex2(fmaf(__uint_as_float(x[i + 1]), sl2, nt));
-              const float p2 = ex2(fmaf(__uint_as_float(x[i + 2]), sl2, nt));
-              const float p3 = ex2(fmaf(__uint_as_float(x[i + 3]), sl2, nt));
-              acc[0] += p0;
-              acc[1] += p1;
-              acc[2] += p2;
-              acc[3] += p3;
-              pk[i >> 1] = pack_bf16(p0, p1);
-              pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+              acc[0] += y[i];
+              acc[1] += y[i + 1];
+              acc[2] += y[i + 2];
+              acc[3] += y[i + 3];
             }
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) pk[i >> 1] = pack_bf16(y[i], y[i + 1]);
             tmem_st16(s_tmem + 16 * c, pk);
             if (quad == 0) HSA_T(3100 + grp * 256 + (j / kGroups) * 8 + c);
           }
@@ -591,40 +629,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
 
       // ---------------------------------------------------------------- epilogue
-      // this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D)
-      // (groups 0 and 1 share the epilogue; group 2 only contributes its partial row sum)
-      constexpr int HC = D / 2;
-      const bool epi = grp < 2;
-      const int cbase = (grp & 1) * HC;
-      float den_part = 0.f;
-      uint32_t fr[HC / 2];
-      if (ok && p.do_linear && epi) {
-        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
-        // MMA) and the partial denominator phi(q) . z -- computed while the last P V drains
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
-        const uint8_t* qrow = smem + L::kQ + r * 128;
-        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
-#pragma unroll
-        for (int c16 = 0; c16 < HC / 8; ++c16) {
-          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
-          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
-          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
-          const int dh = cc >> 3, ch = cc & 7;
-          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
-          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 f = __bfloat1622float2(q2[i]);
-            const float a0 = f.x > 0.f ? f.x + 1.f : __expf(f.x);
-            const float a1 = f.y > 0.f ? f.y + 1.f : __expf(f.y);
-            const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
-            fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
-            const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
-            den_part = fmaf(rr.x, z[2 * i], den_part);
-            den_part = fmaf(rr.y, z[2 * i + 1], den_part);
-          }
-        }
-      }
+      // (this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D))
       if (ok && nsteps > 0) {
         ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
         tc_fence_after();
