@@ -55,7 +55,9 @@ typedef enum {
 /* lin_mode */
 #define HSA_LIN_NONE 0
 #define HSA_LIN_STATE 1      /* running state S = sum phi(k)^T v, z = sum phi(k); phi = elu + 1 */
-#define HSA_LIN_LINFORMER 2  /* Section 3.3 "Linear branch" (Eq. 3); reserved, not built yet    */
+#define HSA_LIN_LINFORMER 2  /* Section 3.3 "Linear branch" (Eq. 3) and Appendix G: per segment of
+                                lin_seg_tokens tokens K~ = E_K^T K, V~ = E_V^T V (lin_rank rows each),
+                                concatenated; O_lin = Softmax(Q K~^T / sqrt(d)) V~.  head_dim 128 only */
 
 /* hsa_config.flags: reserve workspace for causal forwards with the linear branch on */
 #define HSA_CFG_CAUSAL 1u
@@ -77,6 +79,8 @@ typedef struct {
   int32_t gate_act;       /* 0: gates used as given; 1: sigmoid(gate) (Section 3.3, Eq. 5)     */
   float softmax_scale;    /* 0 -> 1/sqrt(head_dim)                                             */
   uint32_t flags;         /* HSA_CFG_* bits                                                    */
+  int32_t lin_rank;       /* HSA_LIN_LINFORMER: projection rank r, a multiple of 128 (else 0)         */
+  int32_t lin_seg_tokens; /* HSA_LIN_LINFORMER: segment length L; every append must be exactly L      */
 } hsa_config;
 
 typedef struct {
@@ -84,6 +88,8 @@ typedef struct {
   size_t v_pool;     /* same                                                                   */
   size_t state;      /* linear-branch state + per-block key sums                               */
   size_t workspace;  /* page table copy, partial sums, status word                             */
+  size_t kc_pool;    /* HSA_LIN_LINFORMER: compressed keys, [segments * r / 64][H][64][d] bf16, else 0  */
+  size_t vc_pool;    /* same for the compressed values                                         */
 } hsa_sizes;
 
 typedef struct {
@@ -91,6 +97,10 @@ typedef struct {
   void* v_pool;     /* device, 256-byte aligned                                                */
   void* state;      /* device, 256-byte aligned; zero-filled by hsa_create (synchronously)     */
   void* workspace;  /* device, 256-byte aligned                                                */
+  void* kc_pool;    /* HSA_LIN_LINFORMER only (else NULL): device, 256-byte aligned            */
+  void* vc_pool;
+  const void* e_k;  /* HSA_LIN_LINFORMER only: device bf16 [H][lin_seg_tokens][lin_rank], 16-byte aligned */
+  const void* e_v;
 } hsa_buffers;
 
 /* Bytes the caller must allocate for a configuration.  Host only, no CUDA call. */

@@ -198,7 +198,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
   const int32_t* sel = p.sel_idx + (static_cast<size_t>(h) * p.n_groups + g) * p.kcap;
   int cnt = p.do_sparse ? p.sel_cnt[static_cast<size_t>(h) * p.n_groups + g] : 0;
-  cnt = max(0, min(cnt, p.kcap));
+  cnt = max(0, min(cnt, min(p.kcap, p.n_blocks)));  // never more blocks than the history holds
   const int nsteps = (cnt + 1) / 2;
 
   if (threadIdx.x == 0) {
@@ -676,6 +676,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
         const __nv_bfloat16* gs =
             (wr && p.g_sp) ? p.g_sp + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
+        const __nv_bfloat16* ext =
+            (wr && p.ext_lin) ? p.ext_lin + (static_cast<size_t>(row) * p.H + h) * D : nullptr;
         const int g_ds = static_cast<int>(p.g_ds);
         const bool sig = p.gate_act == 1;
         // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
@@ -714,6 +716,20 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 16; ++i) ladd[i] = lnum[c0 + i];
           }
+          if (ext) {  // linear branch computed by an earlier pass (Linformer form): already normalised
+            const uint4 e0 = *reinterpret_cast<const uint4*>(ext + c0);
+            const uint4 e1 = *reinterpret_cast<const uint4*>(ext + c0 + 8);
+            const __nv_bfloat162* b0 = reinterpret_cast<const __nv_bfloat162*>(&e0);
+            const __nv_bfloat162* b1 = reinterpret_cast<const __nv_bfloat162*>(&e1);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 f0 = __bfloat1622float2(b0[i]), f1 = __bfloat1622float2(b1[i]);
+              ladd[2 * i] = f0.x;
+              ladd[2 * i + 1] = f0.y;
+              ladd[8 + 2 * i] = f1.x;
+              ladd[8 + 2 * i + 1] = f1.y;
+            }
+          }
           uint32_t packed[8];
 #pragma unroll
           for (int i = 0; i < 16; i += 2) {
@@ -721,7 +737,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               const float osp = has_o ? __uint_as_float(oa[i + e]) * inv_l : 0.f;
-              const float olin = p.do_linear ? (__uint_as_float(ln[i + e]) + ladd[i + e]) * inv_den : 0.f;
+              const float olin = p.do_linear ? (__uint_as_float(ln[i + e]) + ladd[i + e]) * inv_den
+                                             : ladd[i + e];  // 0 unless an external linear output is given
               res[e] = fmaf(wl[i + e], olin, ws[i + e] * osp);
             }
             packed[i >> 1] = pack_bf16(res[0], res[1]);

@@ -38,7 +38,9 @@ struct Layout {
   // state
   size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
   // workspace
-  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ws_total;
+  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ws_total;
+  // Linformer
+  size_t n_cpages, cpool;
 };
 
 bool config_ok(const hsa_config* c) {
@@ -48,7 +50,13 @@ bool config_ok(const hsa_config* c) {
   if (c->page_tokens != HSA_PAGE_TOKENS) return false;
   if (c->max_pages < 1 || c->max_q_tokens < 1 || c->max_topk < 1) return false;
   if (static_cast<int64_t>(c->max_pages) * c->num_heads * kBlock >= (1ll << 31)) return false;
-  if (c->lin_mode != HSA_LIN_NONE && c->lin_mode != HSA_LIN_STATE) return false;
+  if (c->lin_mode != HSA_LIN_NONE && c->lin_mode != HSA_LIN_STATE && c->lin_mode != HSA_LIN_LINFORMER)
+    return false;
+  if (c->lin_mode == HSA_LIN_LINFORMER) {
+    if (c->head_dim != 128) return false;
+    if (c->lin_rank < 128 || c->lin_rank > 2048 || (c->lin_rank % 128) != 0) return false;
+    if (c->lin_seg_tokens < 1 || c->lin_seg_tokens > c->max_q_tokens) return false;
+  }
   if (c->gate_act != 0 && c->gate_act != 1) return false;
   if (!(c->softmax_scale >= 0.f)) return false;
   return true;
@@ -76,6 +84,15 @@ Layout make_layout(const hsa_config* c) {
     L.lin_num = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 4, 256);
     L.lin_den = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * 4, 256);
   }
+  if (c->lin_mode == HSA_LIN_LINFORMER) {
+    const size_t max_segs = (P * kBlock) / static_cast<size_t>(c->lin_seg_tokens);
+    L.n_cpages = (max_segs > 0 ? max_segs : 1) * (static_cast<size_t>(c->lin_rank) / kBlock);
+    L.cpool = L.n_cpages * H * kBlock * D * 2;
+    L.ctable = o; o = align_up(o + L.n_cpages * 4, 256);
+    L.csel = o;   o = align_up(o + H * L.n_cpages * 4, 256);
+    L.ccnt = o;   o = align_up(o + H * 4, 256);
+    L.olin = o;   o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 2, 256);
+  }
   L.ws_total = o;
   return L;
 }
@@ -92,7 +109,8 @@ struct hsa_ctx {
   int64_t n_tokens;
   int32_t last_append;  // tokens of the most recent append (0 after a rewind)
   int nsm;
-  CUtensorMap tm_k, tm_v, tm_state;
+  CUtensorMap tm_k, tm_v, tm_state, tm_kc, tm_vc, tm_olin;
+  int32_t n_segs;  // Linformer: complete segments compressed so far
   int last_cuda_error;
 };
 
@@ -151,6 +169,8 @@ int hsa_query_sizes(const hsa_config* cfg, hsa_sizes* out) {
   out->v_pool = pool;
   out->state = L.state_total;
   out->workspace = L.ws_total;
+  out->kc_pool = L.cpool;
+  out->vc_pool = L.cpool;
   return HSA_OK;
 }
 
@@ -185,6 +205,15 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   ctx->n_tokens = 0;
   ctx->last_append = 0;
   ctx->last_cuda_error = 0;
+  ctx->n_segs = 0;
+  const bool linformer = cfg->lin_mode == HSA_LIN_LINFORMER;
+  if (linformer) {
+    if (!bufs->kc_pool || !bufs->vc_pool || !bufs->e_k || !bufs->e_v || !aligned(bufs->kc_pool, 256) ||
+        !aligned(bufs->vc_pool, 256) || !aligned(bufs->e_k, 16) || !aligned(bufs->e_v, 16)) {
+      delete ctx;
+      return HSA_ERR_INVALID_ARG;
+    }
+  }
 
   cudaError_t e;
   int dev = 0;
@@ -200,6 +229,19 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = forward_init();
   if (e == cudaSuccess) e = append_init();
+  if (e == cudaSuccess && linformer) {
+    e = linformer_init();
+    // identity page table and "every page" selection of the compressed pool
+    std::vector<int32_t> iota(ctx->lay.n_cpages);
+    for (size_t i = 0; i < iota.size(); ++i) iota[i] = static_cast<int32_t>(i);
+    if (e == cudaSuccess)
+      e = cudaMemcpy(ws + ctx->lay.ctable, iota.data(), iota.size() * 4, cudaMemcpyHostToDevice);
+    for (int hh = 0; hh < cfg->num_heads && e == cudaSuccess; ++hh)
+      e = cudaMemcpy(ws + ctx->lay.csel + static_cast<size_t>(hh) * iota.size() * 4, iota.data(),
+                     iota.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(ws + ctx->lay.ccnt, 0, static_cast<size_t>(cfg->num_heads) * 4);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  }
   if (e != cudaSuccess) { delete ctx; return HSA_ERR_CUDA; }
   const int D = cfg->head_dim;
   const uint64_t pool_rows = static_cast<uint64_t>(cfg->max_pages) * cfg->num_heads * kBlock;
@@ -208,6 +250,11 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   if (r == HSA_OK)
     r = encode_2d_rows(&ctx->tm_state, static_cast<uint8_t*>(bufs->state) + ctx->lay.hilo,
                        static_cast<uint64_t>(cfg->num_heads) * 4 * D, D);
+  if (r == HSA_OK && linformer) {
+    const uint64_t crows = static_cast<uint64_t>(ctx->lay.n_cpages) * cfg->num_heads * kBlock;
+    r = encode_2d_rows(&ctx->tm_kc, bufs->kc_pool, crows, D);
+    if (r == HSA_OK) r = encode_2d_rows(&ctx->tm_vc, bufs->vc_pool, crows, D);
+  }
   if (r != HSA_OK) { delete ctx; return r; }
   *out = ctx;
   return HSA_OK;
@@ -251,8 +298,31 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   a.nsplit = nsplit;
   a.lin_state = ctx->cfg.lin_mode == HSA_LIN_STATE;
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  const bool linformer = ctx->cfg.lin_mode == HSA_LIN_LINFORMER;
+  if (linformer && (n_tokens != ctx->cfg.lin_seg_tokens || ctx->n_tokens != static_cast<int64_t>(ctx->n_segs) * n_tokens))
+    return HSA_ERR_UNSUPPORTED;  // this mode appends whole segments only
   cudaError_t e = launch_append(a, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (linformer) {
+    LinformerArgs la{};
+    la.k = a.k;
+    la.v = a.v;
+    la.tok_stride = tok_stride;
+    la.head_stride = head_stride;
+    la.e_k = static_cast<const __nv_bfloat16*>(ctx->buf.e_k);
+    la.e_v = static_cast<const __nv_bfloat16*>(ctx->buf.e_v);
+    la.kc_pool = static_cast<__nv_bfloat16*>(ctx->buf.kc_pool);
+    la.vc_pool = static_cast<__nv_bfloat16*>(ctx->buf.vc_pool);
+    la.ccnt = reinterpret_cast<int32_t*>(ws + ctx->lay.ccnt);
+    la.H = a.H;
+    la.rank = ctx->cfg.lin_rank;
+    la.seg_tokens = ctx->cfg.lin_seg_tokens;
+    la.seg_index = ctx->n_segs;
+    la.status = a.status;
+    e = launch_linformer_compress(la, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->n_segs += 1;
+  }
   ctx->n_tokens = n1;
   ctx->last_append = n_tokens;
   return HSA_OK;
@@ -311,6 +381,9 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   if (flags & ~(HSA_FWD_NO_LINEAR | HSA_FWD_NO_SPARSE)) return HSA_ERR_INVALID_ARG;
   const bool do_sparse = !(flags & HSA_FWD_NO_SPARSE);
   const bool do_linear = !(flags & HSA_FWD_NO_LINEAR) && ctx->cfg.lin_mode == HSA_LIN_STATE;
+  const bool do_linformer = !(flags & HSA_FWD_NO_LINEAR) && ctx->cfg.lin_mode == HSA_LIN_LINFORMER &&
+                            ctx->n_segs > 0;
+  if (do_linformer && causal) return HSA_ERR_UNSUPPORTED;
   if (do_sparse && (!sel_idx_dev || !sel_cnt_dev)) return HSA_ERR_INVALID_ARG;
   if ((g_lin || g_sp) && (gate_tok_stride < 0 || gate_head_stride < 0 || gate_dim_stride < 0))
     return HSA_ERR_INVALID_ARG;
@@ -381,6 +454,38 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     p.lin_num = c.lin_num;
     p.lin_den = c.lin_den;
   }
+  if (do_linformer) {
+    // pass 1: plain softmax attention of the chunk over every compressed row -> O_lin (bf16) in the
+    // workspace; pass 2 below picks it up in its epilogue
+    uint8_t* olin = ws + ctx->lay.olin;
+    CUtensorMap tm_olin;
+    r = encode_q(&tm_olin, olin, n_q, H, D, static_cast<int64_t>(H) * D, D);
+    if (r != HSA_OK) return r;
+    FwdParams p1{};
+    p1.n_q = n_q;
+    p1.H = H;
+    p1.n_tokens = static_cast<int64_t>(ctx->n_segs) * ctx->cfg.lin_rank;
+    p1.q_pos0 = p1.n_tokens;
+    p1.causal = 0;
+    p1.sel_idx = reinterpret_cast<const int32_t*>(ws + ctx->lay.csel);
+    p1.sel_cnt = reinterpret_cast<const int32_t*>(ws + ctx->lay.ccnt);
+    p1.kcap = static_cast<int>(ctx->lay.n_cpages);
+    p1.group_tokens = 0;
+    p1.n_groups = 1;
+    p1.page_table = reinterpret_cast<const int32_t*>(ws + ctx->lay.ctable);
+    p1.n_blocks = static_cast<int>(p1.n_tokens / kBlock);
+    p1.z = p.z;
+    p1.out = reinterpret_cast<__nv_bfloat16*>(olin);
+    p1.o_ts = static_cast<int64_t>(H) * D;
+    p1.o_hs = D;
+    p1.scale_log2 = p.scale_log2;
+    p1.do_linear = 0;
+    p1.do_sparse = 1;
+    p1.status = p.status;
+    cudaError_t e1 = launch_forward(p1, D, tm_q, ctx->tm_kc, ctx->tm_vc, ctx->tm_state, tm_olin, st);
+    if (e1 != cudaSuccess) return cuda_fail(ctx, e1);
+    p.ext_lin = reinterpret_cast<const __nv_bfloat16*>(olin);
+  }
   cudaError_t e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;
@@ -395,6 +500,10 @@ int hsa_get_info(hsa_ctx* ctx, int64_t* n_tokens, int32_t* n_blocks) {
 
 int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens) {
   if (!ctx || n_tokens < 0 || n_tokens > ctx->n_tokens) return HSA_ERR_INVALID_ARG;
+  if (ctx->cfg.lin_mode == HSA_LIN_LINFORMER) {
+    if (n_tokens % ctx->cfg.lin_seg_tokens) return HSA_ERR_UNSUPPORTED;
+    ctx->n_segs = static_cast<int32_t>(n_tokens / ctx->cfg.lin_seg_tokens);
+  }
   ctx->n_tokens = n_tokens;
   ctx->last_append = 0;
   return HSA_OK;

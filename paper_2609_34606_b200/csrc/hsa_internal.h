@@ -85,6 +85,7 @@ struct FwdParams {
   int do_linear, do_sparse;
   const float* lin_num;  // causal intra-chunk partials [n_q][H][D] (or null)
   const float* lin_den;  // [n_q][H]
+  const __nv_bfloat16* ext_lin;  // linear-branch output computed elsewhere, [n_q][H][D] (or null)
   int32_t* status;
 };
 
@@ -102,7 +103,22 @@ struct CausalLinArgs {
   float* lin_den;
 };
 
+struct LinformerArgs {
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  int64_t tok_stride, head_stride;
+  const __nv_bfloat16* e_k;  // [H][seg_tokens][rank]
+  const __nv_bfloat16* e_v;
+  __nv_bfloat16* kc_pool;    // [compressed pages][H][64][128]
+  __nv_bfloat16* vc_pool;
+  int32_t* ccnt;             // [H] number of valid compressed pages
+  int H, rank, seg_tokens, seg_index;
+  int32_t* status;
+};
+
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+cudaError_t launch_linformer_compress(const LinformerArgs& a, cudaStream_t st);
+cudaError_t linformer_init();
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,

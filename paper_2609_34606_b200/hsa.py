@@ -28,7 +28,7 @@ HSA_ERR_UNSUPPORTED = -3
 HSA_ERR_CUDA = -4
 HSA_ERR_DEVICE_TIMEOUT = -5
 HSA_ERR_DEVICE_BOUNDS = -6
-HSA_LIN_NONE, HSA_LIN_STATE = 0, 1
+HSA_LIN_NONE, HSA_LIN_STATE, HSA_LIN_LINFORMER = 0, 1, 2
 HSA_CFG_CAUSAL = 1
 HSA_FWD_NO_LINEAR, HSA_FWD_NO_SPARSE = 1, 2
 PAGE_TOKENS = 64
@@ -47,17 +47,18 @@ class hsa_config(C.Structure):
     _fields_ = [("num_heads", C.c_int32), ("head_dim", C.c_int32), ("page_tokens", C.c_int32),
                 ("max_pages", C.c_int32), ("max_q_tokens", C.c_int32), ("max_topk", C.c_int32),
                 ("lin_mode", C.c_int32), ("gate_act", C.c_int32), ("softmax_scale", C.c_float),
-                ("flags", C.c_uint32)]
+                ("flags", C.c_uint32), ("lin_rank", C.c_int32), ("lin_seg_tokens", C.c_int32)]
 
 
 class hsa_sizes(C.Structure):
     _fields_ = [("k_pool", C.c_size_t), ("v_pool", C.c_size_t), ("state", C.c_size_t),
-                ("workspace", C.c_size_t)]
+                ("workspace", C.c_size_t), ("kc_pool", C.c_size_t), ("vc_pool", C.c_size_t)]
 
 
 class hsa_buffers(C.Structure):
     _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("state", C.c_void_p),
-                ("workspace", C.c_void_p)]
+                ("workspace", C.c_void_p), ("kc_pool", C.c_void_p), ("vc_pool", C.c_void_p),
+                ("e_k", C.c_void_p), ("e_v", C.c_void_p)]
 
 
 def _load() -> C.CDLL:
@@ -236,19 +237,24 @@ class HSAContext:
     def __init__(self, H: int, d: int, max_pages: int, max_q_tokens: int, max_topk: int,
                  lin_mode: int = HSA_LIN_STATE, gate_act: int = 0, softmax_scale: float = 0.0,
                  causal: bool = False, page_order: Optional[torch.Tensor] = None,
-                 device: str | torch.device = "cuda:0"):
+                 device: str | torch.device = "cuda:0", lin_rank: int = 0, lin_seg_tokens: int = 0,
+                 e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None):
         self.device = torch.device(device)
         self.H, self.d = H, d
         self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
         self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
-                              softmax_scale, HSA_CFG_CAUSAL if causal else 0)
+                              softmax_scale, HSA_CFG_CAUSAL if causal else 0, lin_rank, lin_seg_tokens)
         self.sizes = hsa_query_sizes(self.cfg)
         with torch.cuda.device(self.device):
             mk = lambda n: torch.empty(max(n, 16), dtype=torch.uint8, device=self.device)
             self.k_pool, self.v_pool = mk(self.sizes.k_pool), mk(self.sizes.v_pool)
             self.state, self.workspace = mk(self.sizes.state), mk(self.sizes.workspace)
+            self.kc_pool = mk(self.sizes.kc_pool) if self.sizes.kc_pool else None
+            self.vc_pool = mk(self.sizes.vc_pool) if self.sizes.vc_pool else None
+            self.e_k, self.e_v = e_k, e_v   # keep the projection weights alive
             bufs = hsa_buffers(self.k_pool.data_ptr(), self.v_pool.data_ptr(), self.state.data_ptr(),
-                               self.workspace.data_ptr())
+                               self.workspace.data_ptr(), _ptr(self.kc_pool), _ptr(self.vc_pool),
+                               _ptr(e_k), _ptr(e_v))
             self.ctx = hsa_create(self.cfg, bufs, page_order)
         self._off_S, self._off_z, self._off_ksum = hsa_state_layout(self.ctx)
 

@@ -81,6 +81,7 @@ WORKLOADS = {
                         mixture=True, seg_chunks=2, budget_set=(0, 2, 4, 8, 16, ALL)),
     "mid_causal": Workload("mid_causal", H=2, d=128, Lq=300, chunk=300, n_chunks=5, topk=6,
                            seed=14, causal=True, q_inside=True),
+    "mid_linformer": Workload("mid_linformer", H=3, d=128, Lq=300, chunk=328, n_chunks=4, topk=6, seed=16),
     "mid_shuffle": Workload("mid_shuffle", H=2, d=128, Lq=260, chunk=260, n_chunks=9, topk=12,
                             seed=15, shuffle_pages=True),
 }
@@ -174,3 +175,11 @@ def sample_rows(w: Workload, n_random: int = 512, tile: int = 128) -> torch.Tens
 def random_rows(w: Workload, n: int) -> torch.Tensor:
     """n distinct seeded query rows (all rows if n >= Lq)."""
     return torch.randperm(w.Lq, generator=_gen(_tensor_seed(w, 10, 0)))[:min(n, w.Lq)].to(torch.int64)
+
+
+def gen_linformer_weights(w: Workload, rank: int, seg_tokens: int):
+    """Synthetic Linformer projections (E_K, E_V): bf16 [H, seg_tokens, rank] ~ N(0, 1/seg_tokens)."""
+    shape = (w.H, seg_tokens, rank)
+    ek = torch.randn(*shape, generator=_gen(_tensor_seed(w, 11, 0))) / seg_tokens ** 0.5
+    ev = torch.randn(*shape, generator=_gen(_tensor_seed(w, 11, 1))) / seg_tokens ** 0.5
+    return ek.to(torch.bfloat16), ev.to(torch.bfloat16)

@@ -331,3 +331,45 @@ def test_rollout_steps_sampled(cuda_device):
             del K, V
     assert ctx.device_status() == 0 and ctx.n_tokens == w.N
     ctx.destroy()
+
+
+def test_linformer_linear_branch(cuda_device):
+    """The paper's own linear branch: per appended segment K~ = E_K^T K, V~ = E_V^T V (rank rows),
+    softmax attention over all compressed rows, merged with the sparse branch."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["mid_linformer"]
+    rank, seg = 128, w.chunk
+    ek, ev = W.gen_linformer_weights(w, rank, seg)
+    ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk), max_topk=w.n_blocks,
+                         lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=rank, lin_seg_tokens=seg,
+                         e_k=ek.to(cuda_device), e_v=ev.to(cuda_device), device=cuda_device)
+    ctx.k_pool.fill_(0xFF)
+    ctx.v_pool.fill_(0xFF)
+    ctx.kc_pool.fill_(0xFF)
+    ctx.vc_pool.fill_(0xFF)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    budgets = W.gen_budgets(w)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    si, sc = ctx.select_blocks(qd, budgets.to(cuda_device))
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, scores = O.select_blocks(qn, Kn, w.N, False, budgets.tolist())
+    Hn.check_selection(sel_gpu, sel_ref, scores)
+    Kt, Vt = O.linformer_compress(Kn, Vn, Hn.f32(ek), Hn.f32(ev), seg)
+    assert Kt.shape[0] == w.n_chunks * rank
+    o_lin_ref = O.linformer_branch(qn, Kt, Vt)
+    o_sp_ref = O.sparse_branch(qn, Kn, Vn, sel_gpu, w.N, False)
+    out = Hn.f64(ctx.forward(qd, si, sc))
+    o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
+    o_sp = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_LINEAR))
+    assert ctx.device_status() == 0
+    Hn.assert_close(o_sp, o_sp_ref, "O_sp")
+    Hn.assert_close(o_lin, o_lin_ref, "O_lin (Linformer)")
+    Hn.assert_close(out, o_lin_ref + o_sp_ref, "out")
+    # whole segments only
+    k, v = W.gen_kv_chunk(w, 0)
+    with pytest.raises(hsa.HSAError) as e:
+        ctx.append_kv(k[:100].to(cuda_device), v[:100].to(cuda_device))
+    assert e.value.code in (hsa.HSA_ERR_UNSUPPORTED, hsa.HSA_ERR_OUT_OF_PAGES)
+    ctx.destroy()
