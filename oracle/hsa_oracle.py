@@ -399,3 +399,64 @@ def hsa_forward(q, K, V, q_pos0: int, causal: bool, sel, group_tokens: int = 0,
             O_lin[~keep] = 0.0
     out = merge(O_lin, O_sp, g_lin, g_sp, gate_act)
     return {"out": out, "O_sp": O_sp, "O_lin": O_lin}
+
+
+# --------------------------------------------------------------------------
+# head-adaptive block budgets (Appendix "Sparse Branch"): for head h and query
+# group i, p_{i,:} are the block attention weights (softmax of the pooled
+# scores over the candidate blocks), sigma sorts them in descending order,
+#   K_i = min{k : sum_{m<=k} p_{sigma(m)} >= tau_h},     S(i) = first K_i blocks,
+#   G^(h) = mean_i [ (1/N) sum_{m=1..N} (N - 2m + 1) p_{sigma(m)} ]   (Gini, Eq. 12),
+#   tau_h = tau_min + G^(h) (tau_max - tau_min)                        (Eq. 13).
+# Exact ties in the sort go to the lower block index.
+# --------------------------------------------------------------------------
+def block_weights(scores_row, cand):
+    """Softmax of the candidate blocks' pooled scores (zeros elsewhere)."""
+    p = np.zeros_like(scores_row)
+    idx = np.nonzero(cand)[0]
+    if idx.size:
+        e = np.exp(scores_row[idx] - scores_row[idx].max())
+        p[idx] = e / e.sum()
+    return p
+
+
+def gini_of_weights(p_sorted_desc):
+    N = p_sorted_desc.size
+    if N == 0:
+        return 0.0
+    m = np.arange(1, N + 1)
+    return float(((N - 2 * m + 1) * p_sorted_desc).sum() / N)
+
+
+def adaptive_selection(q, K, q_pos0: int, causal: bool, tau_min: float, tau_max: float,
+                       group_tokens: int = 0, scale: float | None = None):
+    """Returns (sel, gini, tau): sel[h][g] ascending block ids chosen by the cumulative-mass
+    rule, gini[h], tau[h]."""
+    Lq, H, _ = q.shape
+    N = K.shape[0]
+    s = block_scores(q, K, group_tokens, scale)
+    groups = group_bounds(Lq, group_tokens)
+    sel, gini, tau = [], np.zeros(H), np.zeros(H)
+    for h in range(H):
+        orders, weights, gs = [], [], []
+        for g, (_, e) in enumerate(groups):
+            cand = candidate_mask(N, q_pos0, e, causal)
+            p = block_weights(s[h, g], cand)
+            idx = np.nonzero(cand)[0]
+            order = idx[np.argsort(-s[h, g][idx], kind="stable")]     # descending, ties -> lower index
+            orders.append(order)
+            weights.append(p[order])
+            gs.append(gini_of_weights(p[order]))
+        gini[h] = float(np.mean(gs)) if gs else 0.0
+        tau[h] = tau_min + gini[h] * (tau_max - tau_min)
+        row = []
+        for order, pw in zip(orders, weights):
+            if order.size == 0:
+                row.append(np.zeros(0, np.int32))
+                continue
+            cum = np.cumsum(pw)
+            hit = np.nonzero(cum >= tau[h])[0]
+            k = int(hit[0]) + 1 if hit.size else order.size
+            row.append(np.sort(order[:k]).astype(np.int32))
+        sel.append(row)
+    return sel, gini, tau

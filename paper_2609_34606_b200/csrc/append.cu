@@ -173,8 +173,16 @@ __global__ void state_reduce_kernel(AppendArgs a) {
   const int h = blockIdx.y;
   if (idx >= DD + D) return;
   const float* part = a.spart + static_cast<size_t>(h) * a.nsplit * (DD + D) + idx;
+  // partials are fetched four at a time (independent loads in flight); the sum order stays fixed
   float add = 0.f;
-  for (int s = 0; s < a.nsplit; ++s) add += part[static_cast<size_t>(s) * (DD + D)];
+  for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
+    float v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      v[i] = (s0 + i < a.nsplit) ? part[static_cast<size_t>(s0 + i) * (DD + D)] : 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) add += v[i];
+  }
   if (idx < DD) {
     const size_t o = static_cast<size_t>(h) * DD + idx;
     const float s_old = a.S[o];

@@ -306,3 +306,67 @@ def test_float32_inputs_are_computed_in_float64():
     a = O.hsa_forward(q, K, V, N, False, sel32)["out"]
     b = O.hsa_forward(q.astype(np.float64), K.astype(np.float64), V.astype(np.float64), N, False, sel64)["out"]
     assert a.dtype == np.float64 and np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- head-adaptive budgets (Gini / tau rule)
+def test_gini_closed_forms():
+    N = 37
+    assert abs(O.gini_of_weights(np.full(N, 1.0 / N))) < 1e-15               # uniform -> 0
+    onehot = np.zeros(N)
+    onehot[0] = 1.0
+    assert abs(O.gini_of_weights(onehot) - (N - 1) / N) < 1e-15              # one-hot -> (N-1)/N
+    # two equal masses: (1/N) * ((N-1) + (N-3)) / 2
+    two = np.zeros(N)
+    two[:2] = 0.5
+    assert abs(O.gini_of_weights(two) - (N - 2) / N) < 1e-15
+    assert O.gini_of_weights(np.zeros(0)) == 0.0
+
+
+def test_block_weights_are_a_softmax_over_candidates():
+    s = np.array([0.3, -1.0, 2.0, 0.0, 5.0])
+    cand = np.array([True, True, True, False, True])
+    p = O.block_weights(s, cand)
+    ref = torch.softmax(torch.tensor(s[cand]), 0).numpy()
+    assert np.allclose(p[cand], ref, atol=1e-15) and p[3] == 0.0 and abs(p.sum() - 1) < 1e-15
+
+
+def test_adaptive_selection_minimal_prefix_and_threshold_map():
+    H, d, Lq, N = 3, 16, 40, 64 * 23 + 7
+    q, K = rnd((Lq, H, d), 60, 3.0), rnd((N, H, d), 61)
+    for tmin, tmax in [(0.35, 1.0), (0.5, 0.5), (0.0, 0.9)]:
+        sel, gini, tau = O.adaptive_selection(q, K, N, False, tmin, tmax)
+        s = O.block_scores(q, K)
+        for h in range(H):
+            p = O.block_weights(s[h, 0], np.ones(s.shape[2], bool))
+            # brute force: sort pairs in Python, walk the prefix
+            order = sorted(range(p.size), key=lambda b: (-s[h, 0, b], b))
+            g_ref = sum((p.size - 2 * (m + 1) + 1) * p[b] for m, b in enumerate(order)) / p.size
+            assert abs(gini[h] - g_ref) < 1e-14
+            assert abs(tau[h] - (tmin + g_ref * (tmax - tmin))) < 1e-14
+            acc, k = 0.0, 0
+            for b in order:
+                acc += p[b]
+                k += 1
+                if acc >= tau[h]:
+                    break
+            assert sorted(order[:k]) == list(sel[h][0])
+            if k > 1:                                   # minimal: one block fewer falls short
+                assert sum(p[b] for b in order[:k - 1]) < tau[h]
+    # monotone in the threshold; tau = 0 keeps exactly one block; peaked head keeps fewer blocks
+    a, _, _ = O.adaptive_selection(q, K, N, False, 0.3, 0.3)
+    b, _, _ = O.adaptive_selection(q, K, N, False, 0.8, 0.8)
+    z, _, _ = O.adaptive_selection(q, K, N, False, 0.0, 0.0)
+    for h in range(H):
+        assert set(a[h][0]) <= set(b[h][0]) and len(z[h][0]) == 1
+
+
+def test_adaptive_selection_per_group_gini_is_averaged():
+    H, d, Lq, N = 1, 8, 48, 64 * 9
+    q, K = rnd((Lq, H, d), 62, 2.0), rnd((N, H, d), 63)
+    sel, gini, tau = O.adaptive_selection(q, K, N, False, 0.2, 0.9, group_tokens=16)
+    s = O.block_scores(q, K, 16)
+    gs = []
+    for g in range(3):
+        p = O.block_weights(s[0, g], np.ones(9, bool))
+        gs.append(O.gini_of_weights(np.sort(p)[::-1]))
+    assert abs(gini[0] - np.mean(gs)) < 1e-14 and len(sel[0]) == 3
