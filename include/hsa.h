@@ -61,6 +61,8 @@ typedef enum {
 
 /* hsa_config.flags: reserve workspace for causal forwards with the linear branch on */
 #define HSA_CFG_CAUSAL 1u
+/* hsa_config.flags: reserve workspace for hsa_select_blocks_adaptive (needs max_pages <= 8192) */
+#define HSA_CFG_ADAPTIVE 2u
 
 /* hsa_forward flags: the paper's "linear only" / "sparse only" ablation modes (Table 4) */
 #define HSA_FWD_NO_LINEAR 1u
@@ -135,6 +137,19 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
                       int64_t head_stride, int64_t q_pos0, int32_t causal,
                       const int32_t* budgets_dev, int32_t q_group_tokens,
                       int32_t* sel_idx_dev, int32_t* sel_cnt_dev, void* stream);
+
+/* Head-adaptive selection (Appendix F, Eq. 12-13): instead of a given budget, each (head, group)
+ * keeps the shortest prefix of its blocks, sorted by pooled score, whose softmax mass reaches
+ *   tau_h = tau_min + G_h (tau_max - tau_min),
+ * G_h being the Gini coefficient of the sorted block weights averaged over the head's groups
+ * (the paper's best setting is tau_max = 1.00, tau_min = 0.35).  Same candidates, tie rule and
+ * output layout as hsa_select_blocks.  gini_tau_out_dev: optional device fp32 [2][H] receiving G_h
+ * and tau_h.  Needs HSA_CFG_ADAPTIVE; HSA_ERR_UNSUPPORTED when the history has more than 8192
+ * blocks. */
+int hsa_select_blocks_adaptive(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
+                               int64_t head_stride, int64_t q_pos0, int32_t causal, float tau_min,
+                               float tau_max, int32_t q_group_tokens, int32_t* sel_idx_dev,
+                               int32_t* sel_cnt_dev, float* gini_tau_out_dev, void* stream);
 
 /* Block selection for callers that cannot allocate device memory (the paper has no counterpart;
  * this is a convenience of this library).  Some callers run where cudaMalloc is off limits --

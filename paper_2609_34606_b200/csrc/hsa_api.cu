@@ -38,7 +38,7 @@ struct Layout {
   // state
   size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
   // workspace
-  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ws_total;
+  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ad_w, ad_idx, ad_gini, ad_wsum, ws_total;
   // Linformer
   size_t n_cpages, cpool;
 };
@@ -59,6 +59,7 @@ bool config_ok(const hsa_config* c) {
   }
   if (c->gate_act != 0 && c->gate_act != 1) return false;
   if (!(c->softmax_scale >= 0.f)) return false;
+  if ((c->flags & HSA_CFG_ADAPTIVE) && c->max_pages > 8192) return false;
   return true;
 }
 
@@ -83,6 +84,12 @@ Layout make_layout(const hsa_config* c) {
   if (c->flags & HSA_CFG_CAUSAL) {
     L.lin_num = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 4, 256);
     L.lin_den = o;  o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * 4, 256);
+  }
+  if (c->flags & HSA_CFG_ADAPTIVE) {
+    L.ad_w = o;    o = align_up(o + H * tiles * P * 8, 256);
+    L.ad_idx = o;  o = align_up(o + H * tiles * P * 4, 256);
+    L.ad_gini = o; o = align_up(o + H * tiles * 8, 256);
+    L.ad_wsum = o; o = align_up(o + H * tiles * 8, 256);
   }
   if (c->lin_mode == HSA_LIN_LINFORMER) {
     const size_t max_segs = (P * kBlock) / static_cast<size_t>(c->lin_seg_tokens);
@@ -364,6 +371,56 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
   a.kcap = ctx->cfg.max_topk;
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   cudaError_t e = launch_select(a, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return HSA_OK;
+}
+
+int hsa_select_blocks_adaptive(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
+                               int64_t head_stride, int64_t q_pos0, int32_t causal, float tau_min,
+                               float tau_max, int32_t q_group_tokens, int32_t* sel_idx_dev,
+                               int32_t* sel_cnt_dev, float* gini_tau_out_dev, void* stream) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (!(ctx->cfg.flags & HSA_CFG_ADAPTIVE)) return HSA_ERR_UNSUPPORTED;
+  if (n_q < 1 || n_q > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, q, tok_stride, head_stride)) return HSA_ERR_INVALID_ARG;
+  if (!sel_idx_dev || !sel_cnt_dev) return HSA_ERR_INVALID_ARG;
+  if (q_group_tokens < 0 || (q_group_tokens % kTileM) != 0) return HSA_ERR_INVALID_ARG;
+  if (!(tau_min >= 0.f) || !(tau_max <= 1.f) || !(tau_min <= tau_max)) return HSA_ERR_INVALID_ARG;
+  const int64_t nblk = (ctx->n_tokens + kBlock - 1) / kBlock;
+  if (nblk > 8192) return HSA_ERR_UNSUPPORTED;
+  uint8_t* stt = static_cast<uint8_t*>(ctx->buf.state);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  SelectArgs a{};
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.n_q = n_q;
+  a.tok_stride = tok_stride;
+  a.head_stride = head_stride;
+  a.q_pos0 = q_pos0;
+  a.causal = causal != 0;
+  a.n_tokens = ctx->n_tokens;
+  a.H = ctx->cfg.num_heads;
+  a.D = ctx->cfg.head_dim;
+  a.max_pages = ctx->cfg.max_pages;
+  a.ksum = reinterpret_cast<const float*>(stt + ctx->lay.ksum);
+  a.budgets = nullptr;
+  a.group_tokens = q_group_tokens;
+  a.n_groups = q_group_tokens > 0 ? (n_q + q_group_tokens - 1) / q_group_tokens : 1;
+  a.scale = ctx->scale;
+  a.qpart = reinterpret_cast<float*>(ws + ctx->lay.qpart);
+  a.keys = reinterpret_cast<uint32_t*>(ws + ctx->lay.keys);
+  a.sel_idx = sel_idx_dev;
+  a.sel_cnt = sel_cnt_dev;
+  a.kcap = ctx->cfg.max_topk;
+  a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  AdaptiveArgs ad{};
+  ad.sorted_w = reinterpret_cast<double*>(ws + ctx->lay.ad_w);
+  ad.sorted_idx = reinterpret_cast<int32_t*>(ws + ctx->lay.ad_idx);
+  ad.gini_part = reinterpret_cast<double*>(ws + ctx->lay.ad_gini);
+  ad.wsum = reinterpret_cast<double*>(ws + ctx->lay.ad_wsum);
+  ad.tau_min = tau_min;
+  ad.tau_max = tau_max;
+  ad.gini_out = gini_tau_out_dev;
+  cudaError_t e = launch_select_adaptive(a, ad, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;
 }

@@ -119,7 +119,17 @@ struct LinformerArgs {
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
 cudaError_t launch_linformer_compress(const LinformerArgs& a, cudaStream_t st);
 cudaError_t linformer_init();
+struct AdaptiveArgs {
+  double* sorted_w;      // [H][n_groups][max_pages] softmax numerators in sorted order
+  int32_t* sorted_idx;   // [H][n_groups][max_pages] block ids in sorted order
+  double* gini_part;     // [H][n_groups]
+  double* wsum;          // [H][n_groups] sum of the numerators
+  float tau_min, tau_max;
+  float* gini_out;       // [2][H]: Gini and threshold per head (or null)
+};
+
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, cudaStream_t st);
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                            const CUtensorMap& tm_state, const CUtensorMap& tm_out, cudaStream_t st);

@@ -252,6 +252,191 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Head-adaptive selection (Appendix "Sparse Branch"): block weights p = softmax of the pooled
+// scores over the candidates, sorted in descending order; Gini coefficient of the sorted weights
+// per (head, group); tau_h = tau_min + mean_g(Gini) (tau_max - tau_min); the selection is the
+// shortest sorted prefix whose mass reaches tau_h.  Two kernels after the score kernel:
+//   adaptive_sort_kernel  one CTA per (group, head): bitonic sort of (score, block) pairs,
+//                         fp64 softmax numerators in sorted order, Gini of the group
+//   adaptive_pick_kernel  one CTA per (group, head): threshold of the head, prefix length by an
+//                         fp64 scan, ascending list of the chosen blocks
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  const uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(u);
+}
+
+__device__ __forceinline__ double block_sum_f64(double v, double* scratch /*[256]*/) {
+  scratch[threadIdx.x] = v;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (static_cast<int>(threadIdx.x) < o) scratch[threadIdx.x] += scratch[threadIdx.x + o];
+    __syncthreads();
+  }
+  const double r = scratch[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(256) adaptive_sort_kernel(SelectArgs a, AdaptiveArgs ad) {
+  extern __shared__ unsigned long long skeys[];  // [np2]
+  __shared__ double scratch[256];
+  const int g = blockIdx.x, h = blockIdx.y;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
+  const int q_hi = min(a.n_q, g * gtok + gtok);
+  const int64_t p_last = a.q_pos0 + q_hi - 1;
+  int64_t ncand64 = nblk;
+  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
+  const int ncand = static_cast<int>(ncand64);
+  int np2 = 1;
+  while (np2 < ncand) np2 <<= 1;
+  const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  for (int i = threadIdx.x; i < np2; i += 256)
+    skeys[i] = i < ncand ? ((static_cast<unsigned long long>(gkeys[i]) << 32) | (0xffffffffu - static_cast<uint32_t>(i)))
+                         : 0ull;  // padding sorts last
+  __syncthreads();
+  // bitonic sort, descending: larger score first, equal scores -> lower block index first
+  for (int k = 2; k <= np2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = threadIdx.x; i < np2; i += 256) {
+        const int ixj = i ^ j;
+        if (ixj > i) {
+          const unsigned long long x = skeys[i], y = skeys[ixj];
+          const bool desc = (i & k) == 0;
+          if (desc ? (x < y) : (x > y)) {
+            skeys[i] = y;
+            skeys[ixj] = x;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  const size_t base = (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  const double smax = ncand > 0 ? static_cast<double>(key_to_float(static_cast<uint32_t>(skeys[0] >> 32))) : 0.0;
+  double esum = 0.0, gsum = 0.0;
+  for (int m = threadIdx.x; m < ncand; m += 256) {
+    const unsigned long long kv = skeys[m];
+    const double sc = static_cast<double>(key_to_float(static_cast<uint32_t>(kv >> 32)));
+    const double e = exp(sc - smax);
+    ad.sorted_w[base + m] = e;
+    ad.sorted_idx[base + m] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(kv & 0xffffffffu));
+    esum += e;
+    gsum += static_cast<double>(ncand - 2 * (m + 1) + 1) * e;
+  }
+  esum = block_sum_f64(esum, scratch);
+  gsum = block_sum_f64(gsum, scratch);
+  if (threadIdx.x == 0) {
+    ad.wsum[static_cast<size_t>(h) * a.n_groups + g] = esum;
+    ad.gini_part[static_cast<size_t>(h) * a.n_groups + g] =
+        (ncand > 0 && esum > 0.0) ? gsum / (esum * static_cast<double>(ncand)) : 0.0;
+  }
+}
+
+__global__ void __launch_bounds__(256) adaptive_pick_kernel(SelectArgs a, AdaptiveArgs ad) {
+  extern __shared__ unsigned char flags[];  // [ncand] 1 = selected
+  __shared__ double scratch[256];
+  __shared__ int warp_sums[8];
+  __shared__ int sh_k;
+  const int g = blockIdx.x, h = blockIdx.y;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
+  const int q_hi = min(a.n_q, g * gtok + gtok);
+  const int64_t p_last = a.q_pos0 + q_hi - 1;
+  int64_t ncand64 = nblk;
+  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
+  const int ncand = static_cast<int>(ncand64);
+  // threshold of the head: mean Gini over the groups, in group order
+  double gmean = 0.0;
+  for (int gg = 0; gg < a.n_groups; ++gg) gmean += ad.gini_part[static_cast<size_t>(h) * a.n_groups + gg];
+  gmean /= static_cast<double>(a.n_groups);
+  const double tau = static_cast<double>(ad.tau_min) + gmean * (static_cast<double>(ad.tau_max) - static_cast<double>(ad.tau_min));
+  if (threadIdx.x == 0 && g == 0 && ad.gini_out) {
+    ad.gini_out[h] = static_cast<float>(gmean);
+    ad.gini_out[a.H + h] = static_cast<float>(tau);
+  }
+  const size_t base = (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  const double target = tau * ad.wsum[static_cast<size_t>(h) * a.n_groups + g];  // mass to reach
+  // prefix length: thread t owns the sorted positions [t*per, t*per + per)
+  const int per = (ncand + 255) / 256;
+  const int lo = min(ncand, static_cast<int>(threadIdx.x) * per), hi = min(ncand, lo + per);
+  double local = 0.0;
+  for (int m = lo; m < hi; ++m) local += ad.sorted_w[base + m];
+  // exclusive prefix of the per-thread sums, in thread order
+  scratch[threadIdx.x] = local;
+  __syncthreads();
+  double before = 0.0;
+  for (int t = 0; t < static_cast<int>(threadIdx.x); ++t) before += scratch[t];
+  if (threadIdx.x == 0) sh_k = ncand;  // mass never reached (rounding at tau ~ 1): keep everything
+  __syncthreads();
+  {
+    double cum = before;
+    for (int m = lo; m < hi; ++m) {
+      cum += ad.sorted_w[base + m];
+      if (cum >= target) {
+        atomicMin(&sh_k, m + 1);
+        break;
+      }
+    }
+  }
+  for (int i = threadIdx.x; i < ncand; i += 256) flags[i] = 0;
+  __syncthreads();
+  const int kk = sh_k;
+  for (int m = threadIdx.x; m < kk; m += 256) flags[ad.sorted_idx[base + m]] = 1;
+  __syncthreads();
+  // ascending compaction of the flagged blocks
+  int my_sel = 0;
+  for (int b = lo; b < hi; ++b) my_sel += flags[b];
+  int total = 0;
+  int pos = block_exclusive_scan(my_sel, warp_sums, &total);
+  int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
+  for (int b = lo; b < hi; ++b) {
+    if (flags[b]) {
+      if (pos < a.kcap) out[pos] = b;
+      ++pos;
+    }
+  }
+  if (threadIdx.x == 0) {
+    a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
+    if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
+  }
+}
+
+cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, cudaStream_t st) {
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  dim3 g1(n_tiles, a.H);
+  if (a.D == 128)
+    qsum_partial_kernel<128><<<g1, 256, 0, st>>>(a);
+  else
+    qsum_partial_kernel<64><<<g1, 256, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  if (nblk > 0) {
+    dim3 g2(static_cast<unsigned>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta), a.n_groups, a.H);
+    if (a.D == 128)
+      block_scores_kernel<128><<<g2, 256, 0, st>>>(a);
+    else
+      block_scores_kernel<64><<<g2, 256, 0, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  int np2 = 1;
+  while (np2 < nblk) np2 <<= 1;
+  const size_t smem_sort = static_cast<size_t>(np2) * 8;
+  if (smem_sort > 40 * 1024)
+    cudaFuncSetAttribute(adaptive_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         static_cast<int>(smem_sort));
+  dim3 g3(a.n_groups, a.H);
+  adaptive_sort_kernel<<<g3, 256, smem_sort, st>>>(a, ad);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  adaptive_pick_kernel<<<g3, 256, static_cast<size_t>(nblk > 0 ? nblk : 1), st>>>(a, ad);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   dim3 g1(n_tiles, a.H);

@@ -30,12 +30,14 @@ HSA_ERR_DEVICE_TIMEOUT = -5
 HSA_ERR_DEVICE_BOUNDS = -6
 HSA_LIN_NONE, HSA_LIN_STATE, HSA_LIN_LINFORMER = 0, 1, 2
 HSA_CFG_CAUSAL = 1
+HSA_CFG_ADAPTIVE = 2
 HSA_FWD_NO_LINEAR, HSA_FWD_NO_SPARSE = 1, 2
 PAGE_TOKENS = 64
 TILE_M = 128
 
 EXPORTS = [
-    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_noalloc",
+    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_adaptive",
+    "hsa_select_blocks_noalloc",
     "hsa_forward",
     "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
     "hsa_last_cuda_error",
@@ -72,6 +74,8 @@ def _load() -> C.CDLL:
     lib.hsa_create.argtypes = [C.POINTER(vp), C.POINTER(hsa_config), C.POINTER(hsa_buffers), vp]
     lib.hsa_append_kv.argtypes = [vp, vp, vp, i32, i64, i64, vp]
     lib.hsa_select_blocks.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp, vp]
+    lib.hsa_select_blocks_adaptive.argtypes = [vp, vp, i32, i64, i64, i64, i32, C.c_float, C.c_float, i32, vp, vp,
+                                               vp, vp]
     lib.hsa_select_blocks_noalloc.argtypes = [vp, i32, i64, i64, i32, i32, vp, i32, i64, i64, i32, C.c_float,
                                               vp, i32, vp, vp, vp, vp]
     lib.hsa_forward.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, vp, i32, vp, vp, i64, i64, i64,
@@ -158,6 +162,16 @@ def hsa_select_blocks(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budg
                                   sel_cnt.data_ptr(), _stream()), "hsa_select_blocks")
 
 
+def hsa_select_blocks_adaptive(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, tau_min: float,
+                               tau_max: float, q_group_tokens: int, sel_idx: torch.Tensor,
+                               sel_cnt: torch.Tensor, gini_tau: Optional[torch.Tensor] = None) -> None:
+    ts, hs = _thd(q, "q")
+    _check(_lib.hsa_select_blocks_adaptive(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
+                                           float(tau_min), float(tau_max), int(q_group_tokens),
+                                           sel_idx.data_ptr(), sel_cnt.data_ptr(), _ptr(gini_tau), _stream()),
+           "hsa_select_blocks_adaptive")
+
+
 def hsa_select_blocks_noalloc(q: torch.Tensor, ksum: torch.Tensor, n_tokens: int, q_pos0: int, causal: bool,
                               softmax_scale: float, budgets: torch.Tensor, sel_idx: torch.Tensor,
                               sel_cnt: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
@@ -237,13 +251,14 @@ class HSAContext:
     def __init__(self, H: int, d: int, max_pages: int, max_q_tokens: int, max_topk: int,
                  lin_mode: int = HSA_LIN_STATE, gate_act: int = 0, softmax_scale: float = 0.0,
                  causal: bool = False, page_order: Optional[torch.Tensor] = None,
-                 device: str | torch.device = "cuda:0", lin_rank: int = 0, lin_seg_tokens: int = 0,
+                 device: str | torch.device = "cuda:0", adaptive: bool = False, lin_rank: int = 0, lin_seg_tokens: int = 0,
                  e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None):
         self.device = torch.device(device)
         self.H, self.d = H, d
         self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
         self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
-                              softmax_scale, HSA_CFG_CAUSAL if causal else 0, lin_rank, lin_seg_tokens)
+                              softmax_scale, (HSA_CFG_CAUSAL if causal else 0) | (HSA_CFG_ADAPTIVE if adaptive else 0),
+                              lin_rank, lin_seg_tokens)
         self.sizes = hsa_query_sizes(self.cfg)
         with torch.cuda.device(self.device):
             mk = lambda n: torch.empty(max(n, 16), dtype=torch.uint8, device=self.device)
@@ -302,6 +317,16 @@ class HSAContext:
         sel_idx, sel_cnt = sel if sel is not None else self.alloc_selection(q.shape[0], group_tokens)
         hsa_select_blocks(self.ctx, q, q_pos0, causal, budgets, group_tokens, sel_idx, sel_cnt)
         return sel_idx, sel_cnt
+
+    def select_blocks_adaptive(self, q: torch.Tensor, tau_min: float, tau_max: float,
+                               q_pos0: Optional[int] = None, causal: bool = False, group_tokens: int = 0):
+        """Cumulative-mass selection with the Gini threshold map; returns (sel_idx, sel_cnt, gini_tau)
+        with gini_tau fp32 [2, H] = (Gini, threshold) per head."""
+        q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
+        sel_idx, sel_cnt = self.alloc_selection(q.shape[0], group_tokens)
+        gt = torch.zeros(2, self.H, dtype=torch.float32, device=self.device)
+        hsa_select_blocks_adaptive(self.ctx, q, q_pos0, causal, tau_min, tau_max, group_tokens, sel_idx, sel_cnt, gt)
+        return sel_idx, sel_cnt, gt
 
     def forward(self, q: torch.Tensor, sel_idx, sel_cnt, q_pos0: Optional[int] = None,
                 causal: bool = False, group_tokens: int = 0, g_lin=None, g_sp=None, flags: int = 0,

@@ -373,3 +373,41 @@ def test_linformer_linear_branch(cuda_device):
         ctx.append_kv(k[:100].to(cuda_device), v[:100].to(cuda_device))
     assert e.value.code in (hsa.HSA_ERR_UNSUPPORTED, hsa.HSA_ERR_OUT_OF_PAGES)
     ctx.destroy()
+
+
+@pytest.mark.parametrize("name,group_tokens", [("mid_mix", 0), ("mid_d128", 0), ("mid_d128", 128), ("cfg1_sharp", 0)])
+def test_head_adaptive_selection(name, group_tokens, cuda_device):
+    """Cumulative-mass selection with the Gini threshold map (tau_max = 1.00, tau_min = 0.35, the
+    paper's best setting) against the oracle; a prefix length may differ only where the cumulative
+    mass at the boundary is within 1e-6 of the threshold."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS[name]
+    order = W.gen_page_order(w, w.n_blocks)
+    ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk), max_topk=w.n_blocks,
+                         adaptive=True, page_order=order, device=cuda_device)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    tmin, tmax = 0.35, 1.0
+    si, sc, gt = ctx.select_blocks_adaptive(qd, tmin, tmax, group_tokens=group_tokens)
+    assert ctx.device_status() == 0
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, gini, tau = O.adaptive_selection(qn, Kn, w.N, False, tmin, tmax, group_tokens)
+    assert np.allclose(gt[0].cpu().numpy(), gini, atol=1e-5) and np.allclose(gt[1].cpu().numpy(), tau, atol=1e-5)
+    s = O.block_scores(qn, Kn, group_tokens)
+    for h in range(w.H):
+        for g in range(len(sel_ref[h])):
+            a, b = list(sel_gpu[h][g]), list(sel_ref[h][g])
+            if a != b:
+                # tolerated only at a knife-edge of the cumulative mass
+                p = O.block_weights(s[h, g], np.ones(s.shape[2], bool))
+                cum = np.cumsum(np.sort(p)[::-1])
+                k = min(len(a), len(b))
+                assert abs(len(a) - len(b)) <= 1 and abs(cum[k - 1] - tau[h]) <= 1e-6, (h, g, len(a), len(b))
+            assert a == sorted(set(a)) and len(a) >= 1
+    # the selection drives the forward pass like any other
+    ref = O.hsa_forward(qn, Kn, Vn, w.N, False, sel_gpu, group_tokens)
+    out = Hn.f64(ctx.forward(qd, si, sc, group_tokens=group_tokens))
+    Hn.assert_close(out, ref["out"], "out")
+    ctx.destroy()
