@@ -109,6 +109,7 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 }  // namespace
 
 struct hsa_ctx {
+  hsa::GridBarrierHost select_bar;  // running total of the selection kernel's grid-barrier counter
   hsa_config cfg;
   hsa_buffers buf;
   Layout lay;
@@ -370,6 +371,8 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
   a.sel_cnt = sel_cnt_dev;
   a.kcap = ctx->cfg.max_topk;
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  a.barrier = reinterpret_cast<unsigned*>(ws + ctx->lay.status + 8);
+  a.bar_host = &ctx->select_bar;
   cudaError_t e = launch_select(a, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;

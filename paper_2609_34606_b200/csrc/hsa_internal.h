@@ -41,6 +41,12 @@ struct AppendArgs {
   int32_t* status;  // device status word
 };
 
+// Host-side view of a grid-barrier arrive counter that is never cleared between launches.
+struct GridBarrierHost {
+  unsigned total = 0;  // value the device counter reaches once every launch so far has finished
+  bool valid = false;  // false: the device counter has to be cleared before the next launch
+};
+
 struct SelectArgs {
   const __nv_bfloat16* q;
   int n_q;
@@ -59,6 +65,8 @@ struct SelectArgs {
   int32_t* sel_cnt;
   int kcap;
   int32_t* status;
+  unsigned* barrier;  // grid-barrier arrive counter for the single-launch path (null: three launches)
+  GridBarrierHost* bar_host;  // host-side running total of that counter (null: cleared per launch)
 };
 
 struct FwdParams {

@@ -2,6 +2,8 @@
 //   s[h,g,b] = mean_q(g) . (Ksum[h,b] / cnt_b) * scale
 // and an exact per-(head, group) top-k by radix select, all on the device:
 // query partial sums -> scores (many CTAs) -> top-k (one CTA per head and group).
+// The three stages run as one cooperative launch with two grid barriers where the device
+// supports it, else as three launches.
 #include <cuda_bf16.h>
 
 #include <cmath>
@@ -15,11 +17,9 @@ namespace hsa {
 // Stage 1: column sums of q over one 128-token tile and one head -> qpart[tile][h][D].
 // ---------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
+__device__ __forceinline__ void qsum_item(const SelectArgs& a, int tile, int h, float (*red)[D]) {
   constexpr int CH = D / 8;
   constexpr int RP = 256 / CH;
-  __shared__ float red[RP][D];
-  const int tile = blockIdx.x, h = blockIdx.y;
   const int c8 = threadIdx.x % CH, rg = threadIdx.x / CH;
   const int t_hi = min(a.n_q, tile * kTileM + kTileM);
   float acc[8];
@@ -55,6 +55,12 @@ __global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
     for (int r = 0; r < RP; ++r) s += red[r][threadIdx.x];
     a.qpart[(static_cast<size_t>(tile) * a.H + h) * D + threadIdx.x] = s;
   }
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
+  __shared__ float red[256 / (D / 8)][D];
+  qsum_item<D>(a, blockIdx.x, blockIdx.y, red);
 }
 
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -93,26 +99,35 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
 constexpr int kScoreBlocksPerCta = 32;
 
 template <int D>
-__global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
-  __shared__ double qs[D];
-  const int g = blockIdx.y, h = blockIdx.z;
+__device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  if (threadIdx.x < D) {
-    double s = 0.0;
+  {
+    // 256 / D threads per column, each summing an interleaved subset of the tile partials with
+    // up to 16 loads in flight; the subsets are then added in a fixed order
+    constexpr int WAYS = 256 / D;
+    const int col = threadIdx.x % D, way = threadIdx.x / D;
     const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
-    // eight independent loads in flight per trip; the sum order stays tile-ascending
-    for (int t0 = tile_lo; t0 < tile_hi; t0 += 8) {
-      float v[8];
+    double s = 0.0;
+    for (int t0 = tile_lo + way; t0 < tile_hi; t0 += 16 * WAYS) {
+      float v[16];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        v[i] = (t0 + i < tile_hi) ? a.qpart[(static_cast<size_t>(t0 + i) * a.H + h) * D + threadIdx.x] : 0.f;
+      for (int i = 0; i < 16; ++i)
+        v[i] = (t0 + i * WAYS < tile_hi) ? __ldcg(&a.qpart[(static_cast<size_t>(t0 + i * WAYS) * a.H + h) * D + col]) : 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) s += static_cast<double>(v[i]);
+      for (int i = 0; i < 16; ++i) s += static_cast<double>(v[i]);
     }
-    qs[threadIdx.x] = s / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
+    double* part = qs + D;  // [WAYS][D]
+    part[way * D + col] = s;
+    __syncthreads();
+    if (threadIdx.x < D) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < WAYS; ++w) t += part[w * D + threadIdx.x];
+      qs[threadIdx.x] = t / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
+    }
   }
   __syncthreads();
   constexpr int PER = D / 32;
@@ -121,14 +136,14 @@ __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   float kv[NB][PER];
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
-    const int64_t b = static_cast<int64_t>(blockIdx.x) * kScoreBlocksPerCta + i * 8 + warp;
+    const int64_t b = static_cast<int64_t>(chunk) * kScoreBlocksPerCta + i * 8 + warp;
 #pragma unroll
     for (int e = 0; e < PER; ++e)
       kv[i][e] = b < nblk ? a.ksum[(static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER + e] : 0.f;
   }
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
-    const int64_t b = static_cast<int64_t>(blockIdx.x) * kScoreBlocksPerCta + i * 8 + warp;
+    const int64_t b = static_cast<int64_t>(chunk) * kScoreBlocksPerCta + i * 8 + warp;
     if (b >= nblk) continue;  // warp-uniform
     double dot = 0.0;
 #pragma unroll
@@ -142,19 +157,29 @@ __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   }
 }
 
+template <int D>
+__global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
+  __shared__ double qs[D + 256];  // mean query, then the per-way partial sums
+  scores_item<D>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs);
+}
+
 // ---------------------------------------------------------------------------------------
 // Stage 3: one CTA per (group, head): k-th largest key by a 4-pass 8-bit radix select, then an
 // index-ordered compaction.  Exact ties at the threshold go to the lower block index.
 // dynamic smem: uint32 keys[ncand]
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
-  extern __shared__ uint32_t keys[];
-  __shared__ int hist[256];
-  __shared__ int warp_sums[8];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_krem;
+struct TopkShared {
+  int hist[256];
+  int warp_sums[8];
+  uint32_t prefix;
+  int krem;
+};
 
-  const int g = blockIdx.x, h = blockIdx.y;
+__device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
+  int* hist = sh->hist;
+  int* warp_sums = sh->warp_sums;
+  uint32_t& sh_prefix = sh->prefix;
+  int& sh_krem = sh->krem;
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_hi = min(a.n_q, g * gtok + gtok);
@@ -164,7 +189,7 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
   const int ncand = static_cast<int>(ncand64);
   const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
-  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = gkeys[b];
+  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
   if (threadIdx.x == 0) {
     sh_prefix = 0;
     sh_krem = 0;
@@ -249,6 +274,69 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   if (threadIdx.x == 0) {
     a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
     if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
+  }
+}
+
+__global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
+  extern __shared__ uint32_t topk_keys[];
+  __shared__ TopkShared sh;
+  topk_item(a, blockIdx.x, blockIdx.y, topk_keys, &sh);
+}
+
+// ---------------------------------------------------------------------------------------
+// The three stages in ONE cooperative launch (one CTA per SM, all co-resident): query tile sums,
+// grid barrier, scores, grid barrier, top-k.  Saves two launches and their drain / ramp-up.
+// The barrier is an arrive counter in global memory (cleared by the host before the launch)
+// that one thread per CTA polls with a time bound; on expiry the CTA records a timeout in the
+// status word and carries on, so the kernel always terminates.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void grid_barrier(unsigned* ctr, unsigned target, int32_t* status) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+    unsigned long long t0 = 0;
+    for (unsigned i = 0;; ++i) {
+      unsigned v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+      if (static_cast<int32_t>(v - target) >= 0) break;  // the counter only grows; wrap-safe
+      if ((i & 63u) == 63u) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        if (now - t0 > 2000000000ull) {
+          atomicCAS(status, 0, kDevTimeout);
+          break;
+        }
+      }
+    }
+    __threadfence();
+  }
+  __syncthreads();
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
+  extern __shared__ uint32_t fused_keys[];
+  __shared__ __align__(16) unsigned char scratch[256 / (D / 8) * D * 4];  // tile-sum partials / mean query
+  __shared__ TopkShared sh;
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+  const int n_chunks = static_cast<int>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta);
+  for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
+    qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
+    __syncthreads();
+  }
+  grid_barrier(bar_ctr, bar_base + gridDim.x, a.status);
+  for (int it = blockIdx.x; it < n_chunks * a.n_groups * a.H; it += gridDim.x) {
+    const int chunk = it % n_chunks, gh = it / n_chunks;
+    scores_item<D>(a, chunk, gh % a.n_groups, gh / a.n_groups, reinterpret_cast<double*>(scratch));
+    __syncthreads();
+  }
+  grid_barrier(bar_ctr, bar_base + 2 * gridDim.x, a.status);
+  for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
+    topk_item(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
+    __syncthreads();
   }
 }
 
@@ -437,7 +525,61 @@ cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, 
   return cudaGetLastError();
 }
 
+namespace {
+// cooperative launch support and SM count of the current device (queried once per device)
+bool coop_info(int* nsm) {
+  static int cached_dev = -1, cached_coop = 0, cached_sm = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (dev != cached_dev) {
+    cudaDeviceGetAttribute(&cached_coop, cudaDevAttrCooperativeLaunch, dev);
+    cudaDeviceGetAttribute(&cached_sm, cudaDevAttrMultiProcessorCount, dev);
+    cached_dev = dev;
+  }
+  *nsm = cached_sm;
+  return cached_coop != 0 && cached_sm > 0;
+}
+}  // namespace
+
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
+  int nsm = 0;
+  if (a.barrier && coop_info(&nsm)) {
+    // one cooperative launch for all three stages
+    const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;
+    const size_t smem_keys = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
+    SelectArgs aa = a;
+    unsigned* ctr = a.barrier;
+    const void* fn = a.D == 128 ? reinterpret_cast<const void*>(select_fused_kernel<128>)
+                                : reinterpret_cast<const void*>(select_fused_kernel<64>);
+    if (smem_keys > 24 * 1024)
+      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_keys));
+    // 256 threads, 48..57 registers and under 12 KB of shared memory per CTA plus the keys:
+    // three CTAs per SM are co-resident while the keys stay below 48 KB
+    int per_sm = 3;
+    if (smem_keys > 48 * 1024) {
+      int occ = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, 256, smem_keys) != cudaSuccess || occ < 1) occ = 1;
+      per_sm = occ < 3 ? occ : 3;
+    }
+    const unsigned grid = static_cast<unsigned>(nsm * per_sm);
+    // The arrive counter only grows: each launch adds 2 * grid to it, and the host keeps the
+    // running total so that no clearing launch is needed.  Without a host total (or after a
+    // failed launch) the counter is cleared on the stream first.
+    unsigned base = 0;
+    if (a.bar_host && a.bar_host->valid) {
+      base = a.bar_host->total;
+    } else {
+      cudaError_t e0 = cudaMemsetAsync(a.barrier, 0, sizeof(unsigned), st);
+      if (e0 != cudaSuccess) return e0;
+    }
+    void* params[3] = {&aa, &ctr, &base};
+    cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(256), params, smem_keys, st);
+    if (a.bar_host) {
+      a.bar_host->valid = (e == cudaSuccess);
+      a.bar_host->total = base + 2 * grid;
+    }
+    return e;
+  }
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   dim3 g1(n_tiles, a.H);
   if (a.D == 128)
@@ -551,5 +693,6 @@ extern "C" int hsa_select_blocks_noalloc(const void* q, int32_t n_q, int64_t tok
   a.sel_cnt = sel_cnt_dev;
   a.kcap = max_topk;
   a.status = status_dev ? status_dev : reinterpret_cast<int32_t*>(sc);
+  a.barrier = reinterpret_cast<unsigned*>(sc + 16);
   return launch_select(a, st) == cudaSuccess ? HSA_OK : HSA_ERR_CUDA;
 }
