@@ -172,17 +172,17 @@ __global__ void state_reduce_kernel(AppendArgs a) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   const int h = blockIdx.y;
   if (idx >= DD + D) return;
+  // results of the kernel before this one are needed from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const float* part = a.spart + static_cast<size_t>(h) * a.nsplit * (DD + D) + idx;
-  // partials are fetched four at a time (independent loads in flight); the sum order stays fixed
+  // all partials are fetched at once (independent loads in flight); the sum order stays fixed
+  float v[kStateSplitMax];
+#pragma unroll
+  for (int i = 0; i < kStateSplitMax; ++i)
+    v[i] = (i < a.nsplit) ? __ldcg(&part[static_cast<size_t>(i) * (DD + D)]) : 0.f;
   float add = 0.f;
-  for (int s0 = 0; s0 < a.nsplit; s0 += 4) {
-    float v[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-      v[i] = (s0 + i < a.nsplit) ? part[static_cast<size_t>(s0 + i) * (DD + D)] : 0.f;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) add += v[i];
-  }
+  for (int i = 0; i < kStateSplitMax; ++i) add += v[i];
   if (idx < DD) {
     const size_t o = static_cast<size_t>(h) * DD + idx;
     const float s_old = a.S[o];
@@ -205,30 +205,60 @@ __global__ void state_reduce_kernel(AppendArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Fused append for head_dim 128 (the measured path): one pass over the chunk's K and V.
-// grid (nsplit, H); a CTA owns a run of consecutive history blocks of one head and, per block,
-//   * copies the new rows into the block's page (and zero-fills the rest of a partial tail page),
-//   * adds their column sums to the block's key sum,
-//   * stages phi(K) (as bf16 hi + lo, so that hi + lo carries ~16 bits) and V in shared memory in
-//     the 128-byte-swizzled MN-major layout and lets the tensor cores accumulate
-//       S_part (128 x 128, fp32 in TMEM) += phi(K)_hi^T V + phi(K)_lo^T V
-//     over the block's tokens (tcgen05, K = tokens), double-buffered against the next block's
-//     loads,
-// and finally writes its partial S and partial z for the fixed-order reduction of stage C.
+// Fused append for head_dim 128 (the measured path): one pass over the chunk's K and V in which
+// no thread touches global memory for the bulk data.
+// grid (nsplit, H); a CTA owns a run of consecutive history blocks of one head.  Per block
+//   * the producer lane brings the block's rows of K and V into a 4-deep ring by TMA (rows
+//     outside the chunk arrive as zeros) and sends the same tiles on to the block's page by
+//     TMA store (a block that already held tokens before this call is written row by row by
+//     the workers instead, so that its old rows stay),
+//   * sixteen worker warps (two groups on alternate blocks) read K from the ring, build phi(K) as bf16 hi + lo (hi + lo carries
+//     ~16 bits) in the 128-byte-swizzled MN-major layout,
+//   * the MMA lane lets the tensor cores accumulate, over the block's tokens (tcgen05, K = tokens)
+//       S_part (128 x 128, fp32 in TMEM) += phi(K)_hi^T V + phi(K)_lo^T V      (V straight from the ring)
+//       z_part (128 x 16)                 += phi(K)_hi^T 1 + phi(K)_lo^T 1
+//       ksum_b (128 x 16)                  = K^T 1                              (K straight from the ring)
+//     and four more warps read ksum_b back as soon as it is final,
+// and finally the CTA writes its partial S and z for the fixed-order reduction of stage C.
+// Every wait is bounded; on expiry the CTA records a timeout and leaves.
 // ---------------------------------------------------------------------------------------
+#ifdef HSA_TIMING
+__device__ long long g_af_timing[1024];
+#define AF_T(slot)                                                                   \
+  do {                                                                               \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (slot) < 1024) { \
+      long long t_;                                                                  \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                          \
+      g_af_timing[(slot)] = t_;                                                      \
+    }                                                                                \
+  } while (0)
+#else
+#define AF_T(slot) \
+  do {             \
+  } while (0)
+#endif
+
 namespace {
 
-constexpr int kAfThreads = 512;
-constexpr int kAfRowGroups = kAfThreads / 16;   // 32: a thread handles rows rg and rg + 32 of a block
-constexpr int kAfRows = kBlock / kAfRowGroups;  // 2 rows per thread and block
-constexpr int kAfTile = 64 * 128 * 2;           // [64 tokens x 128 dims] bf16 = two swizzled slabs
-constexpr int kAfStage = 3 * kAfTile;           // phi hi | phi lo | V
-constexpr int kAfRed = kAfRowGroups * 128 * 4;  // key-sum partials of one block
-constexpr int kAfSmem = 2 * kAfStage + 2 * kAfRed + 64 + 1024;
+constexpr int kAfDepth = 4;                      // ring stages
+constexpr int kAfWorkers = 512;                  // worker threads (warps 2..17)
+constexpr int kAfThreads = 64 + kAfWorkers + 128;  // + producer warp + MMA warp + 4 key-sum warps
+constexpr int kAfTile = 64 * 128 * 2;            // [64 tokens x 128 dims] bf16 = two swizzled slabs
+constexpr int kAfStage = 2 * kAfTile;            // K | V
+constexpr int kAfHilo = 2 * kAfTile;             // phi hi | phi lo
+constexpr int kAfOnes = 2048;                    // [16 x 64] bf16 ones (K-major operand)
+constexpr int kAfSmem = kAfDepth * kAfStage + 2 * kAfHilo + kAfOnes + 256 + 1024;
+constexpr uint32_t kAfTmemCols = 256;
+constexpr uint32_t kAfColZ = 128, kAfColKs = 144;  // TMEM columns: S 0..127, z, ksum[2]
+constexpr int kAfPitch = 132;                      // floats per row of the staged partial state
+static_assert(128 * kAfPitch * 4 <= 2 * kAfHilo + kAfOnes, "partial state is staged in the hi/lo + ones area");
 
 struct AfBars {
-  uint64_t mma_done[2];
-  uint64_t all_done;
+  uint64_t full[kAfDepth];      // ring stage landed
+  uint64_t consumed[kAfDepth];  // tensor cores are done with the stage
+  uint64_t phi_ready[2];        // hi/lo buffer written
+  uint64_t mma_done[2];         // tensor cores are done with the hi/lo buffer (and ksum is final)
+  uint64_t ks_read[2];          // key-sum buffer read back
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -245,212 +275,322 @@ __device__ __forceinline__ bool af_wait(uint64_t* bar, uint32_t parity, AfBars* 
 }
 
 // elu(x) + 1 with the fast exponential (relative error ~1e-6, far inside the state's tolerance)
-__device__ __forceinline__ float phi_fast(float x) { return x > 0.f ? x + 1.f : __expf(x); }
+__device__ __forceinline__ float phi_fast(float x) {
+  float e;  // branch-free: elu(x) + 1 = max(x, 0) + exp(min(x, 0))
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(x, 0.f) * 1.4426950408889634f));
+  return fmaxf(x, 0.f) + e;
+}
+
+__device__ __forceinline__ void tma_store_2d(const void* tmap, const void* smem_src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(tmap)),
+               "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
 
 }  // namespace
 
-__global__ void __launch_bounds__(kAfThreads, 1) append_fused_kernel(AppendArgs a, int blocks_per_cta) {
+__global__ void __launch_bounds__(kAfThreads, 1)
+append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CUtensorMap tm_kin,
+                    const __grid_constant__ CUtensorMap tm_vin, const __grid_constant__ CUtensorMap tm_kpool,
+                    const __grid_constant__ CUtensorMap tm_vpool) {
   constexpr int D = 128;
   extern __shared__ uint8_t af_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(af_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  float* red = reinterpret_cast<float*>(smem + 2 * kAfStage);  // [2][row groups][128]
-  AfBars* bars = reinterpret_cast<AfBars*>(smem + 2 * kAfStage + 2 * kAfRed);
+  uint8_t* ring = smem;
+  uint8_t* hilo = smem + kAfDepth * kAfStage;
+  uint8_t* ones = hilo + 2 * kAfHilo;
+  AfBars* bars = reinterpret_cast<AfBars*>(ones + kAfOnes);
+
+  // the reduction kernel behind this one may be scheduled early; it waits for this grid itself
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int h = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ch = threadIdx.x & 15;  // 16-byte chunk of a row (8 dims)
-  const int rg = threadIdx.x >> 4;  // row group
+  if (warp == 0) AF_T(0);
   const int64_t b_first = a.n0 / kBlock, b_last = (a.n0 + a.n_new - 1) / kBlock;
   const int64_t bs = b_first + static_cast<int64_t>(split) * blocks_per_cta;
   const int64_t be = min64(b_last + 1, bs + blocks_per_cta);
   const int nblk = static_cast<int>(max64(0, be - bs));
   const int64_t n_end = a.n0 + a.n_new;
 
+  auto issue_loads = [&](int bi) {
+    const int s = bi % kAfDepth;
+    uint8_t* st = ring + s * kAfStage;
+    const int32_t row0 = static_cast<int32_t>((bs + bi) * kBlock - a.n0);  // may be negative: zero fill
+    mbar_expect_tx(&bars->full[s], kAfStage);
+    tma_load_3d(st, &tm_kin, &bars->full[s], 0, h, row0);
+    tma_load_3d(st + kAfTile / 2, &tm_kin, &bars->full[s], 64, h, row0);
+    tma_load_3d(st + kAfTile, &tm_vin, &bars->full[s], 0, h, row0);
+    tma_load_3d(st + kAfTile + kAfTile / 2, &tm_vin, &bars->full[s], 64, h, row0);
+  };
   if (threadIdx.x == 0) {
-    mbar_init(&bars->mma_done[0], 1);
-    mbar_init(&bars->mma_done[1], 1);
-    mbar_init(&bars->all_done, 1);
+    for (int s = 0; s < kAfDepth; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->consumed[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bars->phi_ready[s], kAfWorkers / 2);  // one worker group per buffer
+      mbar_init(&bars->mma_done[s], 1);
+      mbar_init(&bars->ks_read[s], 4);
+    }
     bars->abort_flag = 0;
     fence_mbar_init();
+    // the first ring fill starts before the rest of the CTA is set up
+    for (int bi = 0; bi < nblk && bi < kAfDepth; ++bi) issue_loads(bi);
+    tma_prefetch_desc(&tm_kpool);
+    tma_prefetch_desc(&tm_vpool);
   }
-  if (warp == 0) {
-    tmem_alloc(&bars->tmem_base, 128);
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, kAfTmemCols);
     tmem_relinquish();
   }
+  // bf16 1.0 everywhere: under any swizzle the tile reads as all ones
+  for (int i = threadIdx.x; i < kAfOnes / 4; i += kAfThreads) reinterpret_cast<uint32_t*>(ones)[i] = 0x3F803F80u;
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
+  if (warp == 0) AF_T(1);
 
-  uint4 kreg[kAfRows], vreg[kAfRows];
-  auto load_block = [&](int64_t b, uint4 (&kk)[kAfRows], uint4 (&vv)[kAfRows]) {
-#pragma unroll
-    for (int i = 0; i < kAfRows; ++i) {
-      const int64_t t = b * kBlock + rg + kAfRowGroups * i;
-      if (t >= a.n0 && t < n_end) {
-        const size_t src = static_cast<size_t>(t - a.n0) * a.tok_stride +
-                           static_cast<size_t>(h) * a.head_stride + ch * 8;
-        kk[i] = *reinterpret_cast<const uint4*>(a.k + src);
-        vv[i] = *reinterpret_cast<const uint4*>(a.v + src);
-      } else {
-        kk[i] = make_uint4(0, 0, 0, 0);
-        vv[i] = make_uint4(0, 0, 0, 0);
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (elect_one_sync()) {
+      bool ok = true;
+      for (int bi = 0; bi < nblk && ok; ++bi) {
+        const int s = bi % kAfDepth;
+        ok = af_wait(&bars->full[s], (bi / kAfDepth) & 1, bars, a.status);
+        if (!ok) break;
+        AF_T(16 + bi * 8 + 0);
+        const int64_t b = bs + bi;
+        if (b * kBlock >= a.n0) {  // the block holds nothing older: whole tiles go to its page
+          uint8_t* st = ring + s * kAfStage;
+          const int32_t prow = (a.page_table[b] * a.H + h) * kBlock;
+          tma_store_2d(&tm_kpool, st, 0, prow);
+          tma_store_2d(&tm_kpool, st + kAfTile / 2, 64, prow);
+          tma_store_2d(&tm_vpool, st + kAfTile, 0, prow);
+          tma_store_2d(&tm_vpool, st + kAfTile + kAfTile / 2, 64, prow);
+        }
+        tma_store_commit();
+        AF_T(16 + bi * 8 + 1);
+        if (bi >= 1 && bi - 1 + kAfDepth < nblk) {
+          // refill the stage of block bi - 1: its stores have read it, the tensor cores are done
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          AF_T(16 + bi * 8 + 2);
+          ok = af_wait(&bars->consumed[(bi - 1) % kAfDepth], ((bi - 1) / kAfDepth) & 1, bars, a.status);
+          AF_T(16 + bi * 8 + 3);
+          if (ok) issue_loads(bi - 1 + kAfDepth);
+        }
       }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // every page write has landed
+      AF_T(2);
     }
-  };
-  if (nblk > 0) load_block(bs, kreg, vreg);
-
-  float zacc[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) zacc[e] = 0.f;
-  bool ok = true;
-
-#pragma unroll 1
-  for (int bi = 0; bi < nblk; ++bi) {
-    const int64_t b = bs + bi;
-    const int stage = bi & 1;
-    uint8_t* st_hi = smem + stage * kAfStage;
-    uint8_t* st_lo = st_hi + kAfTile;
-    uint8_t* st_v = st_lo + kAfTile;
-    float* my_red = red + stage * (kAfRowGroups * 128);
-    uint4 knext[kAfRows], vnext[kAfRows];
-    if (bi + 1 < nblk) load_block(b + 1, knext, vnext);  // next block's loads fly under this one
-    // the tensor cores must be done with this stage's previous tiles (block bi - 2)
-    if (bi >= 2) ok = af_wait(&bars->mma_done[stage], ((bi >> 1) - 1) & 1, bars, a.status) && ok;
-    const int page = a.page_table[b];
-    const size_t row_base = (static_cast<size_t>(page) * a.H + h) * kBlock;
-    float ks[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) ks[e] = 0.f;
-#pragma unroll
-    for (int i = 0; i < kAfRows; ++i) {
-      const int r = rg + kAfRowGroups * i;
-      const int64_t t = b * kBlock + r;
-      const bool fresh = t >= a.n0 && t < n_end;
-      const uint32_t soff = (ch >> 3) * (kAfTile / 2) + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-      // rows that are not new carry zeros (loaded as zeros above): they add nothing anywhere
-      const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kreg[i]);
-      uint32_t hw[4], lw[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(k2[e]);
-        ks[2 * e] += f.x;
-        ks[2 * e + 1] += f.y;
-        const float p0 = fresh ? phi_fast(f.x) : 0.f, p1 = fresh ? phi_fast(f.y) : 0.f;
-        zacc[2 * e] += p0;
-        zacc[2 * e + 1] += p1;
-        const __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-        const float2 hf = __bfloat1622float2(hh);
-        const __nv_bfloat162 ll = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
-        hw[e] = *reinterpret_cast<const uint32_t*>(&hh);
-        lw[e] = *reinterpret_cast<const uint32_t*>(&ll);
-      }
-      if (fresh || t >= n_end) {
-        // new rows go to the page; rows of a partial tail page past the last token are zeroed so
-        // that the pool never holds garbage the forward kernel could multiply by zero
-        const size_t dst = (row_base + r) * D + ch * 8;
-        *reinterpret_cast<uint4*>(a.k_pool + dst) = kreg[i];
-        *reinterpret_cast<uint4*>(a.v_pool + dst) = vreg[i];
-      }
-      *reinterpret_cast<uint4*>(st_hi + soff) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-      *reinterpret_cast<uint4*>(st_lo + soff) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-      *reinterpret_cast<uint4*>(st_v + soff) = vreg[i];
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) my_red[rg * 128 + ch * 8 + e] = ks[e];
-    fence_proxy_async_smem();  // generic-proxy writes above -> visible to the tensor cores
-    __syncthreads();
-    if (warp == 0) {
-      if (elect_one_sync() && ok) {
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (one lane)
+    if (elect_one_sync()) {
+      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 1, 1);
+      constexpr uint32_t idesc_1 = idesc_bf16_f32(128, 16, 1, 0);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      const uint32_t b_ones = desc_lo_sw128(smem_u32(ones), 16);
+      for (int bi = 0; bi < nblk; ++bi) {
+        const int s = bi % kAfDepth, hb = bi & 1;
+        if (!af_wait(&bars->phi_ready[hb], (bi >> 1) & 1, bars, a.status)) break;
+        AF_T(256 + bi * 4 + 0);
         tc_fence_after();
-        constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 1, 1);
-        constexpr uint32_t hi = desc_hi_sw128(1024);
-        const uint32_t a_hi = desc_lo_sw128(smem_u32(st_hi), kAfTile / 2);
-        const uint32_t a_lo = desc_lo_sw128(smem_u32(st_lo), kAfTile / 2);
-        const uint32_t b_v = desc_lo_sw128(smem_u32(st_v), kAfTile / 2);
+        uint8_t* st = ring + s * kAfStage;
+        const uint32_t a_k = desc_lo_sw128(smem_u32(st), kAfTile / 2);
+        const uint32_t b_v = desc_lo_sw128(smem_u32(st + kAfTile), kAfTile / 2);
+        const uint32_t a_hi = desc_lo_sw128(smem_u32(hilo + hb * kAfHilo), kAfTile / 2);
+        const uint32_t a_lo = desc_lo_sw128(smem_u32(hilo + hb * kAfHilo + kAfTile), kAfTile / 2);
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
-          tc_mma_ss_lo(tmem, a_hi + kk * 128, b_v + kk * 128, hi, idesc, (bi > 0 || kk > 0) ? 1u : 0u);
+          tc_mma_ss_lo(tmem, a_hi + kk * 128, b_v + kk * 128, hi, idesc_s, (bi > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) tc_mma_ss_lo(tmem, a_lo + kk * 128, b_v + kk * 128, hi, idesc, 1u);
-        tc_commit(&bars->mma_done[stage]);
+        for (int kk = 0; kk < 4; ++kk) tc_mma_ss_lo(tmem, a_lo + kk * 128, b_v + kk * 128, hi, idesc_s, 1u);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_ss_lo(tmem + kAfColZ, a_hi + kk * 128, b_ones, hi, idesc_1, (bi > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) tc_mma_ss_lo(tmem + kAfColZ, a_lo + kk * 128, b_ones, hi, idesc_1, 1u);
+        if (bi >= 2 && !af_wait(&bars->ks_read[hb], ((bi >> 1) - 1) & 1, bars, a.status)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_ss_lo(tmem + kAfColKs + hb * 16, a_k + kk * 128, b_ones, hi, idesc_1, kk > 0 ? 1u : 0u);
+        tc_commit(&bars->consumed[s]);
+        tc_commit(&bars->mma_done[hb]);
+        AF_T(256 + bi * 4 + 1);
       }
-    } else if (threadIdx.x >= kAfThreads - 128) {
-      // key sum of the block: fixed-order sum over the row groups
-      const int c = threadIdx.x - (kAfThreads - 128);
-      float s = 0.f;
-#pragma unroll
-      for (int g2 = 0; g2 < kAfRowGroups; ++g2) s += my_red[g2 * 128 + c];
-      float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + c;
-      const float old = (a.n0 > b * kBlock) ? *dst : 0.f;  // block partly filled before
-      *dst = old + s;
     }
-#pragma unroll
-    for (int i = 0; i < kAfRows; ++i) {
-      kreg[i] = knext[i];
-      vreg[i] = vnext[i];
-    }
-  }
-
-  // all tensor-core work of this CTA done?
-  if (warp == 0) {
-    if (elect_one_sync()) tc_commit(&bars->all_done);
-  }
-  ok = af_wait(&bars->all_done, 0, bars, a.status) && ok;
-  tc_fence_after();
-  float* out = a.spart + (static_cast<size_t>(h) * a.nsplit + split) * (D * D + D);
-  {
-    const int quad = warp & 3, part = warp >> 2;  // 16 warps: 4 lane quadrants x 4 column quarters
-    const int row = quad * 32 + lane;
-    uint32_t v[32];
-    if (nblk > 0) {
-      tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + part * 32, v);
+  } else if (warp >= 2 + kAfWorkers / 32) {
+    // ------------------------------------------------------------------ key-sum warps
+    // one warp per TMEM lane quadrant: key sum of each block, as soon as its MMAs are done
+    const int quad = warp & 3;
+    for (int bj = 0; bj < nblk; ++bj) {
+      if (!af_wait(&bars->mma_done[bj & 1], (bj >> 1) & 1, bars, a.status)) break;
+      tc_fence_after();
+      uint32_t v[16];
+      tmem_ld16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + kAfColKs + (bj & 1) * 16, v);
       tc_wait_ld();
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = 0u;
+      tc_fence_before();
+      if (lane == 0) mbar_arrive(&bars->ks_read[bj & 1]);
+      const int64_t b = bs + bj;
+      float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + quad * 32 + lane;
+      const float old = (a.n0 > b * kBlock) ? *dst : 0.f;  // block partly filled before
+      *dst = old + __uint_as_float(v[0]);
     }
-    float4* dst = reinterpret_cast<float4*>(out + row * D + part * 32);
+  } else {
+    // ------------------------------------------------------------------ workers
+    // two groups of eight warps take alternate blocks, so that one group's waits hide under the
+    // other's arithmetic
+    const int w = threadIdx.x - 64;
+    const int grp = w >> 8, wg = w & 255;
+    const int ch = wg & 15;  // 16-byte chunk of a row (8 dims)
+    const int rg = wg >> 4;  // rows rg, rg + 16, rg + 32, rg + 48 of a block
+    const int quad = warp & 3;
+    bool ok = true;
+    uint32_t soff[4];  // the thread's four 16-byte chunks inside a swizzled [64 x 128] tile
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-      dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                           __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+    for (int i = 0; i < 4; ++i) {
+      const int r = rg + 16 * i;
+      soff[i] = (ch >> 3) * (kAfTile / 2) + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+    }
+#pragma unroll 1
+    for (int bi = grp; bi < nblk && ok; bi += 2) {
+      const int s = bi % kAfDepth, hb = bi & 1;
+      const int64_t b = bs + bi;
+      ok = af_wait(&bars->full[s], (bi / kAfDepth) & 1, bars, a.status);
+      if (!ok) break;
+      if (warp == 2) AF_T(512 + bi * 4 + 0);
+      const uint8_t* st_k = ring + s * kAfStage;
+      uint4 kreg[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) kreg[i] = *reinterpret_cast<const uint4*>(st_k + soff[i]);
+      if (b * kBlock < a.n0) {
+        // block partly filled before this call: only its new rows (and the zero rows past the
+        // last token) are written, by hand
+        const size_t row_base = (static_cast<size_t>(a.page_table[b]) * a.H + h) * kBlock;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int r = rg + 16 * i;
+          const int64_t t = b * kBlock + r;
+          if (t >= a.n0) {
+            const size_t dst = (row_base + r) * D + ch * 8;
+            *reinterpret_cast<uint4*>(a.k_pool + dst) = kreg[i];
+            *reinterpret_cast<uint4*>(a.v_pool + dst) = *reinterpret_cast<const uint4*>(st_k + kAfTile + soff[i]);
+          }
+        }
+      }
+      if (bi >= 2) {
+        ok = af_wait(&bars->mma_done[hb], ((bi >> 1) - 1) & 1, bars, a.status);
+        if (!ok) break;
+      }
+      if (warp == 2) AF_T(512 + bi * 4 + 1);
+      uint8_t* st_hi = hilo + hb * kAfHilo;
+      uint8_t* st_lo = st_hi + kAfTile;
+      // rows outside the chunk (only in its first and last block) add nothing to the state
+      const bool whole = b * kBlock >= a.n0 && b * kBlock + kBlock <= n_end;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kreg[i]);
+        uint32_t hw[4], lw[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = phi_fast(__uint_as_float(kw[e] << 16));
+          const float p1 = phi_fast(__uint_as_float(kw[e] & 0xffff0000u));
+          hw[e] = pack_bf16(p0, p1);
+          lw[e] = pack_bf16(p0 - __uint_as_float(hw[e] << 16), p1 - __uint_as_float(hw[e] & 0xffff0000u));
+        }
+        if (!whole) {
+          const int64_t t = b * kBlock + rg + 16 * i;
+          if (t < a.n0 || t >= n_end) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) hw[e] = lw[e] = 0u;
+          }
+        }
+        *reinterpret_cast<uint4*>(st_hi + soff[i]) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        *reinterpret_cast<uint4*>(st_lo + soff[i]) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+      }
+      fence_proxy_async_smem();  // generic-proxy writes above -> visible to the tensor cores
+      mbar_arrive(&bars->phi_ready[hb]);
+      if (warp == 2) AF_T(512 + bi * 4 + 2);
+    }
+    // the partial state, once every MMA is done: the last two blocks' barriers, in block order (a
+    // group has not watched the other group's barrier, so it must not skip a phase of it)
+    for (int bj = max(0, nblk - 2); bj < nblk && ok; ++bj)
+      ok = af_wait(&bars->mma_done[bj & 1], (bj >> 1) & 1, bars, a.status);
+    if (warp == 2) AF_T(3);
+    tc_fence_after();
+    float* out = a.spart + (static_cast<size_t>(h) * a.nsplit + split) * (D * D + D);
+    const int row = quad * 32 + lane;
+    {
+      // TMEM -> shared memory (row pitch 132 floats: conflict-free both ways) -> coalesced rows
+      float* stage = reinterpret_cast<float*>(hilo);
+      uint32_t v[32];
+      const int col = ((warp - 2) >> 2) * 32;  // four warps per lane quadrant, 32 columns each
+      if (nblk > 0 && ok) {
+        tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + col, v);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = 0u;
+      }
+      float4* srow = reinterpret_cast<float4*>(stage + row * kAfPitch + col);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        srow[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                              __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+      asm volatile("bar.sync 1, %0;" ::"n"(kAfWorkers) : "memory");
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int f = w + kAfWorkers * i;  // float4 index of the [128][128] partial state
+        const int r2 = f >> 5, c4 = f & 31;
+        reinterpret_cast<float4*>(out)[f] = *reinterpret_cast<const float4*>(stage + r2 * kAfPitch + c4 * 4);
+      }
+    }
+    if (warp < 6) {
+      uint32_t v[16];
+      v[0] = 0u;
+      if (nblk > 0 && ok) {
+        tmem_ld16(tmem + (static_cast<uint32_t>(quad * 32) << 16) + kAfColZ, v);
+        tc_wait_ld();
+      }
+      out[D * D + row] = __uint_as_float(v[0]);
+    }
   }
-  // z partial: fixed-order sum over the row groups
-  __syncthreads();
-#pragma unroll
-  for (int e = 0; e < 8; ++e) red[rg * 128 + ch * 8 + e] = zacc[e];
-  __syncthreads();
-  if (threadIdx.x < 128) {
-    float s = 0.f;
-#pragma unroll
-    for (int g2 = 0; g2 < kAfRowGroups; ++g2) s += red[g2 * 128 + threadIdx.x];
-    out[D * D + threadIdx.x] = s;
-  }
+  if (warp == 2) AF_T(4);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 128);
+    tmem_dealloc(tmem, kAfTmemCols);
   }
+  if (warp == 0) AF_T(5);
 }
+
+#ifdef HSA_TIMING
+extern "C" int hsa_debug_read_af_timing(long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_af_timing, sizeof(long long) * n));
+}
+#endif
 
 cudaError_t append_init() {
   return cudaFuncSetAttribute(append_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);
 }
 
-cudaError_t launch_append(const AppendArgs& a_in, cudaStream_t st) {
+cudaError_t launch_append(const AppendArgs& a_in, const AppendMaps* maps, cudaStream_t st) {
   AppendArgs a = a_in;
   const int64_t b0 = a.n0 / kBlock;
   const int64_t b1 = (a.n0 + a.n_new - 1) / kBlock;
   cudaError_t e;
-  if (a.D == 128 && a.lin_state) {
+  if (a.D == 128 && a.lin_state && maps) {
     const int nb = static_cast<int>(b1 - b0 + 1);
     const int per = (nb + a.nsplit - 1) / a.nsplit;
     a.nsplit = (nb + per - 1) / per;  // no empty CTAs
     dim3 grid(a.nsplit, a.H);
-    append_fused_kernel<<<grid, kAfThreads, kAfSmem, st>>>(a, per);
+    append_fused_kernel<<<grid, kAfThreads, kAfSmem, st>>>(a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   } else {
@@ -469,10 +609,20 @@ cudaError_t launch_append(const AppendArgs& a_in, cudaStream_t st) {
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
+  // The reduction may be scheduled while the kernel before it drains (programmatic dependent
+  // launch); it waits for that kernel's results itself before it reads anything.
   const int n = a.D * a.D + a.D;
-  dim3 gridC((n + 255) / 256, a.H);
-  state_reduce_kernel<<<gridC, 256, 0, st>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((n + 255) / 256, a.H);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, state_reduce_kernel, a);
 }
 
 }  // namespace hsa

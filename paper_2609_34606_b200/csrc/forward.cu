@@ -663,6 +663,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tc_fence_after();
       }
       if (quad == 0) HSA_T(3006 + grp);
+      // The output tile is staged in the Q tile's shared memory.  A tile with no step and no linear
+      // branch has not looked at Q at all: its TMA load may still be in flight and must land first.
+      if (ok && epi && nsteps == 0 && !p.do_linear)
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
       if (ok && epi) {  // warp-uniform: the TMEM loads below are warp-collective
         const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
         float lin_den = den;

@@ -142,13 +142,14 @@ int encode_2d_rows(CUtensorMap* tm, void* base, uint64_t rows, int D) {
   return r == CUDA_SUCCESS ? HSA_OK : HSA_ERR_CUDA;
 }
 
-int encode_q(CUtensorMap* tm, const void* q, int n_q, int H, int D, int64_t ts, int64_t hs) {
+int encode_q(CUtensorMap* tm, const void* q, int n_q, int H, int D, int64_t ts, int64_t hs,
+             int box_rows = kTileM) {
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return HSA_ERR_CUDA;
   cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(H),
                         static_cast<cuuint64_t>(n_q)};
   cuuint64_t strides[2] = {static_cast<cuuint64_t>(hs) * 2, static_cast<cuuint64_t>(ts) * 2};
-  cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(kTileM)};
+  cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(box_rows)};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box,
                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -309,7 +310,16 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   const bool linformer = ctx->cfg.lin_mode == HSA_LIN_LINFORMER;
   if (linformer && (n_tokens != ctx->cfg.lin_seg_tokens || ctx->n_tokens != static_cast<int64_t>(ctx->n_segs) * n_tokens))
     return HSA_ERR_UNSUPPORTED;  // this mode appends whole segments only
-  cudaError_t e = launch_append(a, static_cast<cudaStream_t>(stream));
+  AppendMaps maps;
+  const bool fused = a.D == 128 && a.lin_state;
+  if (fused) {
+    if (encode_q(&maps.kin, k, n_tokens, a.H, a.D, tok_stride, head_stride, kBlock) != HSA_OK ||
+        encode_q(&maps.vin, v, n_tokens, a.H, a.D, tok_stride, head_stride, kBlock) != HSA_OK)
+      return HSA_ERR_CUDA;
+    maps.kpool = ctx->tm_k;
+    maps.vpool = ctx->tm_v;
+  }
+  cudaError_t e = launch_append(a, fused ? &maps : nullptr, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   if (linformer) {
     LinformerArgs la{};

@@ -124,7 +124,12 @@ struct LinformerArgs {
   int32_t* status;
 };
 
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+// tensor maps of the fused append kernel: the chunk's K and V ([tokens][H][d], box 64 dims x 1 x 64
+// tokens) and the two pools ([rows][d], box 64 x 64), all with the 128-byte swizzle
+struct AppendMaps {
+  CUtensorMap kin, vin, kpool, vpool;
+};
+cudaError_t launch_append(const AppendArgs& a, const AppendMaps* maps, cudaStream_t st);
 cudaError_t launch_linformer_compress(const LinformerArgs& a, cudaStream_t st);
 cudaError_t linformer_init();
 struct AdaptiveArgs {

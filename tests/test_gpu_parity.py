@@ -139,6 +139,24 @@ def test_edge_cases(cuda_device):
     ctx.destroy()
 
 
+def test_tiles_without_work_write_exact_zeros(cuda_device):
+    """A tile with no selected block and no linear branch never looks at its queries; its output
+    must still be exact zeros (the output tile is staged where the query tile lands), every time."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["cfg2"]
+    ctx = Hn.build_context(w, cuda_device, max_topk=w.topk)
+    k, v = W.gen_kv_chunk(w, 0)
+    ctx.append_kv(k.to(cuda_device), v.to(cuda_device))
+    q = (W.gen_query(w) + 3.0).to(cuda_device)   # nowhere near zero, so stale queries would show
+    si, sc = ctx.select_blocks(q, torch.zeros(w.H, dtype=torch.int32, device=cuda_device))
+    assert int(sc.sum()) == 0
+    for _ in range(25):
+        out = ctx.forward(q, si, sc, flags=hsa.HSA_FWD_NO_LINEAR)
+        assert int(torch.count_nonzero(out.view(torch.int16) & 0x7FFF)) == 0
+    assert ctx.device_status() == 0
+    ctx.destroy()
+
+
 def test_bad_selection_index_is_flagged_not_followed(cuda_device):
     from paper_2609_34606_b200 import hsa
     w = W.WORKLOADS["mid_d64"]
