@@ -238,6 +238,7 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = forward_init();
   if (e == cudaSuccess) e = append_init();
+  if (e == cudaSuccess) e = linear_only_init();
   if (e == cudaSuccess && linformer) {
     e = linformer_init();
     // identity page table and "every page" selection of the compressed pool
@@ -556,7 +557,11 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     if (e1 != cudaSuccess) return cuda_fail(ctx, e1);
     p.ext_lin = reinterpret_cast<const __nv_bfloat16*>(olin);
   }
-  cudaError_t e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st);
+  cudaError_t e;
+  if (D == 128 && do_linear && !do_sparse && !p.ext_lin)
+    e = launch_linear_only(p, ctx->nsm, tm_q, ctx->tm_state, tm_out, st);  // nothing but Q in, out out
+  else
+    e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;
 }

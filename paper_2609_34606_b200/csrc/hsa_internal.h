@@ -147,7 +147,11 @@ cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                            const CUtensorMap& tm_state, const CUtensorMap& tm_out, cudaStream_t st);
 cudaError_t launch_causal_linear(const CausalLinArgs& a, cudaStream_t st);
+// linear branch alone (head_dim 128): lean HBM-bound kernel, nsm = SMs of the device
+cudaError_t launch_linear_only(const FwdParams& p, int nsm, const CUtensorMap& tm_q, const CUtensorMap& tm_state,
+                               const CUtensorMap& tm_out, cudaStream_t st);
+cudaError_t linear_only_init();
 cudaError_t forward_init();
-cudaError_t append_init();  // opt in to the shared-memory size the fused append kernel needs  // opt in to the shared-memory size the forward kernel needs
+cudaError_t append_init();  // opt in to the shared-memory size the fused append kernel needs
 
 }  // namespace hsa
