@@ -4,7 +4,9 @@
 A "step" is one pass of the whole hot path for one query chunk of the
 1.3B-class video-DiT layer workload (H=12, d=128, chunk 4680 tokens, history
 10 chunks = 46,800 tokens, top-64 blocks per head): restore the 9-chunk state,
-hsa_append_kv (chunk 10) -> hsa_select_blocks -> hsa_forward.
+hsa_append_kv (chunk 10) -> hsa_select_blocks -> hsa_forward.  By default the
+step is captured once per input set in a CUDA graph and the timed loop replays
+the graphs (`--launch eager` issues the same calls one by one instead).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -143,7 +145,11 @@ def bench_ours(args, rank: int, world: int):
         k, v = W.gen_kv_chunk(w, c, layer=rank)
         ctx.append_kv(k.to(dev), v.to(dev))
     n_before = ctx.n_tokens
-    snapshot = ctx.state.clone()
+    # what a step changes and the next step must find as it was: the running state S, z (and the
+    # key sum of a partly filled last block, if the history does not end on a block boundary)
+    S_snap, z_snap = ctx.S.clone(), ctx.z.clone()
+    tail_blk = n_before // 64 if n_before % 64 else None
+    ksum_snap = ctx.ksum[:, tail_blk].clone() if tail_blk is not None else None
     # host (pinned) and device copies of RING distinct input sets
     host, devs = [], []
     for r in range(RING):
@@ -162,7 +168,10 @@ def bench_ours(args, rank: int, world: int):
             q.copy_(hq, non_blocking=True)
             k.copy_(hk, non_blocking=True)
             v.copy_(hv, non_blocking=True)
-        ctx.state.copy_(snapshot)
+        ctx.S.copy_(S_snap)
+        ctx.z.copy_(z_snap)
+        if tail_blk is not None:
+            ctx.ksum[:, tail_blk].copy_(ksum_snap)
         ctx.rewind(n_before)
         if ev:
             ev[0].record()
@@ -194,18 +203,68 @@ def bench_ours(args, rank: int, world: int):
     sel_tokens = [sum(min(64, w.N - 64 * int(b)) for b in idx[h, 0, :cnt[h]].tolist()) for h in range(w.H)]
 
     K = args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    # eager pass with events between the calls: per-stage times (launch gaps included)
+    Ks = max(3, min(K, 50))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(Ks)]
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s0.record()
+    for i in range(Ks):
+        step(i, evs[i])
+    s1.record()
+    torch.cuda.synchronize()
+    ms_eager = s0.elapsed_time(s1) / Ks
+    stage = [sum(evs[i][s].elapsed_time(evs[i][s + 1]) for i in range(Ks)) / Ks for s in range(3)]
+
+    def capture(fn):
+        """One CUDA graph per input set, each holding fn(slot)."""
+        gs = []
+        for r in range(RING):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn(r)
+            gs.append(g)
+        return gs
+
+    def time_graphs(gs, reps):
+        for g in gs:
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for i in range(reps):
+            gs[i % RING].replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    # each call on its own, replayed from graphs: the kernels' own durations without launch gaps
+    def only_append(r):
+        ctx.rewind(n_before)
+        ctx.append_kv(devs[r][1], devs[r][2])
+    kern = {"append": time_graphs(capture(only_append), 40),
+            "select": time_graphs(capture(lambda r: ctx.select_blocks(devs[r][0], budgets, sel=sel)), 40),
+            "forward": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3])), 40),
+            "linear_only": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3],
+                                                                     flags=hsa.HSA_FWD_NO_SPARSE)), 40),
+            "sparse_only": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3],
+                                                                     flags=hsa.HSA_FWD_NO_LINEAR)), 40)}
+    step(0)  # leaves the context as a full step does
+
+    graphs = capture(step) if args.launch == "graph" else None
+    run = (lambda i: graphs[i % RING].replay()) if graphs else step
+    for i in range(max(args.warmup, 3)):
+        run(i)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     wall0 = time.time()
     e0.record()
     for i in range(K):
-        step(i, evs[i])
+        run(i)
     e1.record()
     barrier()
     wall1 = time.time()
     ms_total = e0.elapsed_time(e1)
-    stage = [sum(evs[i][s].elapsed_time(evs[i][s + 1]) for i in range(K)) / K for s in range(3)]
     status = ctx.device_status()
 
     # clocks: extend with an identical, untimed loop if the timed region was too short to sample
@@ -217,7 +276,7 @@ def bench_ours(args, rank: int, world: int):
             p0 = time.time()
             i = 0
             while time.time() - p0 < 1.5:
-                step(i)
+                run(i)
                 i += 1
                 if i % 50 == 0:
                     torch.cuda.synchronize()
@@ -225,26 +284,13 @@ def bench_ours(args, rank: int, world: int):
             p1 = time.time()
             time.sleep(0.15)
             probe = sampler.summary(p0, p1)
-    # the two ablation modes of the forward kernel, timed on their own (not part of the step)
-    def time_flags(flags, reps=20):
-        q, k, v, out = devs[0]
-        for _ in range(3):
-            ctx.forward(q, sel[0], sel[1], out=out, flags=flags)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for i in range(reps):
-            qq, _, _, oo = devs[i % RING]
-            ctx.forward(qq, sel[0], sel[1], out=oo, flags=flags)
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps
-    ms_lin_only = time_flags(hsa.HSA_FWD_NO_SPARSE)
-    ms_sp_only = time_flags(hsa.HSA_FWD_NO_LINEAR)
+    ms_lin_only, ms_sp_only = kern["linear_only"], kern["sparse_only"]
     if args.profile:
         if rank == 0:
-            print(json.dumps({"profile_run": True, "steps": K, "ms_per_step": ms_total / K,
-                              "stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
-                              "linear_only_ms": ms_lin_only, "sparse_only_ms": ms_sp_only}))
+            print(json.dumps({"profile_run": True, "launch": args.launch, "steps": K, "ms_per_step": ms_total / K,
+                              "eager_ms_per_step": ms_eager,
+                              "eager_stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
+                              "kernel_ms": kern}))
         ctx.destroy()
         return
     # end-to-end through the same API with host buffers (H2D inputs + D2H result inside the region)
@@ -272,36 +318,43 @@ def bench_ours(args, rank: int, world: int):
             clocks = dict(probe, note="timed region shorter than 3 samples; sampled over an identical "
                                       "1.5 s loop run right after it")
         tf = lambda f, ms: f / (ms * 1e-3) / 1e12
-        fwd_tf = tf(fl["forward"], stage[2])
+        fwd_tf = tf(fl["forward"], kern["forward"])
         line = {
             "metric": METRIC, "value": world * tf(fl["total"], ms_step), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{w.name}: H={w.H} d={w.d} chunk={w.Lq} history={w.N} tokens "
                                    f"({w.n_blocks} blocks of 64) top-{w.topk} blocks/head",
-                       "step": "restore 9-chunk state + hsa_append_kv + hsa_select_blocks + hsa_forward",
+                       "step": "restore the 9-chunk running state (S, z) + hsa_append_kv + hsa_select_blocks + "
+                               "hsa_forward",
+                       "launch": ("one CUDA graph per input set holds the step; the timed loop replays them"
+                                  if args.launch == "graph" else "eager: every call issued from the host"),
                        "l2": f"inputs rotate over {RING} distinct (q,k,v,out) sets "
                              f"({RING * 4 * w.Lq * w.H * w.d * 2 / 1e6:.0f} MB > 126 MB L2)",
                        "replicas": world},
             "ms_per_chunk": ms_step,
-            "stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
-            "stage_gbs": {"append": by["append"] / stage[0] / 1e6, "select": by["select"] / stage[1] / 1e6,
-                          "forward": by["forward"] / stage[2] / 1e6},
+            "eager_ms_per_step": ms_eager,
+            "eager_stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
+            "kernel_ms": {k2: kern[k2] for k2 in ("append", "select", "forward")},
+            "kernel_gbs": {k2: by[k2] / kern[k2] / 1e6 for k2 in ("append", "select", "forward")},
             "flops_per_step": fl["total"],
             "forward_modes_ms": {"linear_only": ms_lin_only, "sparse_only": ms_sp_only,
                                  "linear_only_gbs": (2 * w.Lq * w.H * w.d * 2 + w.H * w.d * w.d * 4) / ms_lin_only / 1e6},
             "clocks": clocks,
             "e2e": {"value": world * tf(fl["total"], ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": 3 * w.Lq * w.H * w.d * 2, "d2h_bytes_per_step": w.Lq * w.H * w.d * 2},
-            "gpu_launches": 6 * K,
+            "gpu_launches": 4 * K,  # append_fused, state_reduce, select_fused, hsa_forward per step
             "device_status": status,
             "roofline": {"kernel": "hsa_forward_kernel<128>", "bound": "tensor", "achieved": fwd_tf,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tf / peaks["bf16_tflops"],
                          "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": by["forward"],
                          "peak_source": peaks["source"] + " (burst)",
                          "frac_of_sustained": fwd_tf / peaks["bf16_tflops_sustained"],
-                         "append_hbm_frac": by["append"] / stage[0] / 1e6 / peaks["hbm_gbs"],
-                         "select_hbm_frac": by["select"] / stage[1] / 1e6 / peaks["hbm_gbs"]},
+                         "timing": "average duration of the call replayed from CUDA graphs, CUDA events",
+                         "append_hbm_frac": by["append"] / kern["append"] / 1e6 / peaks["hbm_gbs"],
+                         "select_hbm_frac": by["select"] / kern["select"] / 1e6 / peaks["hbm_gbs"],
+                         "linear_only_hbm_frac": (2 * w.Lq * w.H * w.d * 2 + w.H * w.d * w.d * 4) / ms_lin_only
+                                                 / 1e6 / peaks["hbm_gbs"]},
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, rows=args.cpu_rows)
@@ -388,7 +441,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--cpu-rows", type=int, default=2048)
+    ap.add_argument("--cpu-rows", type=int, default=4680)
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
+                    help="how the timed steps are issued: replayed CUDA graphs (default) or call by call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", action="store_true",
                     help="profiling run: set-up, warm-up and the K timed steps only (no clock probe loop, "
