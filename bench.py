@@ -147,7 +147,10 @@ def bench_ours(args, rank: int, world: int):
     n_before = ctx.n_tokens
     # what a step changes and the next step must find as it was: the running state S, z (and the
     # key sum of a partly filled last block, if the history does not end on a block boundary)
-    S_snap, z_snap = ctx.S.clone(), ctx.z.clone()
+    # (S and z sit next to each other at the start of the state buffer: one copy restores both)
+    assert ctx.S.data_ptr() == ctx.state.data_ptr() and ctx.z.data_ptr() > ctx.S.data_ptr()
+    sz_bytes = ctx.z.data_ptr() - ctx.state.data_ptr() + ctx.z.numel() * 4
+    sz_snap = ctx.state[:sz_bytes].clone()
     tail_blk = n_before // 64 if n_before % 64 else None
     ksum_snap = ctx.ksum[:, tail_blk].clone() if tail_blk is not None else None
     # host (pinned) and device copies of RING distinct input sets
@@ -168,8 +171,7 @@ def bench_ours(args, rank: int, world: int):
             q.copy_(hq, non_blocking=True)
             k.copy_(hk, non_blocking=True)
             v.copy_(hv, non_blocking=True)
-        ctx.S.copy_(S_snap)
-        ctx.z.copy_(z_snap)
+        ctx.state[:sz_bytes].copy_(sz_snap)
         if tail_blk is not None:
             ctx.ksum[:, tail_blk].copy_(ksum_snap)
         ctx.rewind(n_before)
