@@ -218,51 +218,56 @@ def bench_ours(args, rank: int, world: int):
     ms_eager = s0.elapsed_time(s1) / Ks
     stage = [sum(evs[i][s].elapsed_time(evs[i][s + 1]) for i in range(Ks)) / Ks for s in range(3)]
 
-    def capture(fn):
-        """One CUDA graph per input set, each holding fn(slot)."""
-        gs = []
-        for r in range(RING):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                fn(r)
-            gs.append(g)
-        return gs
+    def capture(fn, n):
+        """One CUDA graph holding fn(0), fn(1), ... fn(n - 1) (the input sets rotate inside fn)."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n):
+                fn(i)
+        return g
 
-    def time_graphs(gs, reps):
-        for g in gs:
-            g.replay()
+    def time_graph(g, n, reps=3):
+        """Mean duration of one of the n calls held by the graph."""
+        g.replay()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record()
-        for i in range(reps):
-            gs[i % RING].replay()
+        for _ in range(reps):
+            g.replay()
         b.record()
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps
+        return a.elapsed_time(b) / (reps * n)
 
     # each call on its own, replayed from graphs: the kernels' own durations without launch gaps
-    def only_append(r):
+    def only_append(i):
         ctx.rewind(n_before)
-        ctx.append_kv(devs[r][1], devs[r][2])
-    kern = {"append": time_graphs(capture(only_append), 40),
-            "select": time_graphs(capture(lambda r: ctx.select_blocks(devs[r][0], budgets, sel=sel)), 40),
-            "forward": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3])), 40),
-            "linear_only": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3],
-                                                                     flags=hsa.HSA_FWD_NO_SPARSE)), 40),
-            "sparse_only": time_graphs(capture(lambda r: ctx.forward(devs[r][0], sel[0], sel[1], out=devs[r][3],
-                                                                     flags=hsa.HSA_FWD_NO_LINEAR)), 40)}
+        ctx.append_kv(devs[i % RING][1], devs[i % RING][2])
+    NK = 5 * RING  # calls per graph
+    fwd = lambda flags: (lambda i: ctx.forward(devs[i % RING][0], sel[0], sel[1], out=devs[i % RING][3], flags=flags))
+    kern = {"append": time_graph(capture(only_append, NK), NK),
+            "select": time_graph(capture(lambda i: ctx.select_blocks(devs[i % RING][0], budgets, sel=sel), NK), NK),
+            "forward": time_graph(capture(fwd(0), NK), NK),
+            "linear_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_SPARSE), NK), NK),
+            "sparse_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_LINEAR), NK), NK)}
     step(0)  # leaves the context as a full step does
 
-    graphs = capture(step) if args.launch == "graph" else None
-    run = (lambda i: graphs[i % RING].replay()) if graphs else step
-    for i in range(max(args.warmup, 3)):
-        run(i)
+    # the timed loop: K steps, as replays of a graph that holds GS steps plus single-step graphs for
+    # the remainder (or call by call with --launch eager)
+    GS = 2 * RING
+    if args.launch == "graph":
+        g_many, g_one = capture(step, GS), [capture(lambda i, r=r: step(r), 1) for r in range(RING)]
+        plan = [g_many] * (K // GS) + [g_one[i % RING] for i in range(K % GS)]
+        run_all = lambda: [g.replay() for g in plan]
+        warm = lambda: (g_many.replay(), [g.replay() for g in g_one])
+    else:
+        run_all = lambda: [step(i) for i in range(K)]
+        warm = lambda: [step(i) for i in range(max(args.warmup, 3))]
+    warm()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     wall0 = time.time()
     e0.record()
-    for i in range(K):
-        run(i)
+    run_all()
     e1.record()
     barrier()
     wall1 = time.time()
@@ -278,9 +283,9 @@ def bench_ours(args, rank: int, world: int):
             p0 = time.time()
             i = 0
             while time.time() - p0 < 1.5:
-                run(i)
+                run_all()
                 i += 1
-                if i % 50 == 0:
+                if i % 4 == 0:
                     torch.cuda.synchronize()
             torch.cuda.synchronize()
             p1 = time.time()
@@ -329,7 +334,8 @@ def bench_ours(args, rank: int, world: int):
                                    f"({w.n_blocks} blocks of 64) top-{w.topk} blocks/head",
                        "step": "restore the 9-chunk running state (S, z) + hsa_append_kv + hsa_select_blocks + "
                                "hsa_forward",
-                       "launch": ("one CUDA graph per input set holds the step; the timed loop replays them"
+                       "launch": (f"CUDA graphs: the timed loop replays a graph of {2 * RING} consecutive steps "
+                                  "(single-step graphs for the remainder)"
                                   if args.launch == "graph" else "eager: every call issued from the host"),
                        "l2": f"inputs rotate over {RING} distinct (q,k,v,out) sets "
                              f"({RING * 4 * w.Lq * w.H * w.d * 2 / 1e6:.0f} MB > 126 MB L2)",

@@ -80,6 +80,9 @@ struct Bars {
 };
 static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory slot");
 
+#ifndef HSA_INTERLEAVE
+#define HSA_INTERLEAVE 8
+#endif
 #ifdef HSA_TIMING
 __device__ long long g_hsa_timing[4096];
 #define HSA_T(slot)                                                      \
@@ -120,6 +123,12 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// same, but ordered against the other volatile statements (keeps a hand-made instruction order)
+__device__ __forceinline__ float ex2v(float x) {
+  float y;
+  asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
@@ -593,6 +602,26 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               for (int i = 0; i < 32; ++i)
                 if (i >= lim) x[i] = 0xff800000u;  // -inf
             }
+#if HSA_INTERLEAVE
+            // software pipeline over the chunk's 32 columns: scale-and-shift of column i, the
+            // exponential of column i - LAG and the row sum / bf16 pack of column i - LAG - LAG2 are
+            // issued next to each other, so that the FMA-pipe work fills the issue slots between
+            // two exponentials (the SFU takes one warp instruction per 8 cycles)
+            float y[32];
+            uint32_t pk[16];
+            constexpr int LAG = HSA_INTERLEAVE;
+            constexpr int LAG2 = LAG;
+#pragma unroll
+            for (int i = 0; i < 32 + LAG + LAG2; ++i) {
+              if (i < 32) y[i] = fmaf(__uint_as_float(x[i]), sl2, nt);
+              if (i >= LAG && i - LAG < 32) y[i - LAG] = ex2v(y[i - LAG]);
+              if (i >= LAG + LAG2 && i - LAG - LAG2 < 32) {
+                const int k = i - LAG - LAG2;
+                acc[k & 3] += y[k];
+                if (k & 1) pk[k >> 1] = pack_bf16(y[k - 1], y[k]);
+              }
+            }
+#else
             // stage by stage over the whole chunk, so that 32 independent operations of each kind
             // are in flight: scale-and-shift, exponential, row sum, bf16 pack
             float y[32];
@@ -610,6 +639,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) pk[i >> 1] = pack_bf16(y[i], y[i + 1]);
+#endif
             tmem_st16(s_tmem + 16 * c, pk);
             if (quad == 0) HSA_T(3100 + grp * 256 + (j / kGroups) * 8 + c);
           }
