@@ -138,6 +138,31 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
                       const int32_t* budgets_dev, int32_t q_group_tokens,
                       int32_t* sel_idx_dev, int32_t* sel_cnt_dev, void* stream);
 
+/* Selection with the two sparse granularities of Section 3.3 ("Inter- and intra-chunk sparse
+ * granularity"): history before the current chunk is scored and selected in coarse blocks of
+ * inter_block_pages pages (2 = the paper's B_inter = 128 tokens), the current chunk's own tokens in
+ * single pages (B_intra = 64); both kinds come out as one ascending list of 64-token pages, so the
+ * forward kernel is the same.
+ *   inter_block_pages   1 or 2 (0 = 1).  A coarse block is scored by the mean key over all of its
+ *                       tokens; selecting it selects its pages.  budgets_dev counts coarse blocks.
+ *   intra_first_page    first page of the current chunk (the page that holds its first token), or
+ *                       < 0 for no intra-chunk region.  Pages from here on are candidates of their
+ *                       own, outside budgets_dev.
+ *   intra_budgets_dev   device int32[H] budgets for those pages, or NULL = every one of them
+ *                       (the chunk always attends to itself).
+ * max_topk must hold inter_block_pages * budget + the intra-chunk pages.  opts == NULL is
+ * hsa_select_blocks.  Everything else as hsa_select_blocks. */
+typedef struct {
+  int32_t inter_block_pages;
+  int32_t intra_first_page;
+  const int32_t* intra_budgets_dev;
+} hsa_select_opts;
+int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
+                         int64_t head_stride, int64_t q_pos0, int32_t causal,
+                         const int32_t* budgets_dev, int32_t q_group_tokens,
+                         const hsa_select_opts* opts, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
+                         void* stream);
+
 /* Head-adaptive selection (Appendix F, Eq. 12-13): instead of a given budget, each (head, group)
  * keeps the shortest prefix of its blocks, sorted by pooled score, whose softmax mass reaches
  *   tau_h = tau_min + G_h (tau_max - tau_min),

@@ -167,6 +167,76 @@ def select_blocks(q, K, q_pos0: int, causal: bool, budgets, group_tokens: int = 
 
 
 # --------------------------------------------------------------------------
+# Two sparse granularities (Sec. 3.3, "Inter- and intra-chunk sparse
+# granularity"): history before the current chunk is partitioned into coarse
+# blocks of B_inter = inter_pages * 64 tokens, the current chunk's own tokens
+# into blocks of B_intra = 64; both go through the same block-sparse
+# attention, so a selection is reported as a list of 64-token pages.
+# The paper fixes the two block sizes only; that each kind has its own budget
+# and that a coarse block is scored by the mean key over all its tokens are
+# this implementation's readings.
+# --------------------------------------------------------------------------
+def mixed_candidates(N: int, inter_pages: int, intra_first_page: int):
+    """Token ranges [(t0, t1), ...] of the candidates in history order: runs of
+    inter_pages pages below intra_first_page (the last run may be short), then
+    single pages.  intra_first_page < 0 or beyond the history: no intra part.
+    Returns (ranges, n_inter)."""
+    nb = n_blocks(N)
+    p0 = intra_first_page if 0 <= intra_first_page < nb else nb
+    ip = max(1, int(inter_pages))
+    ranges = []
+    for first in range(0, p0, ip):
+        last = min(p0, first + ip)
+        ranges.append((BLOCK * first, min(N, BLOCK * last)))
+    n_inter = len(ranges)
+    for pg in range(p0, nb):
+        ranges.append((BLOCK * pg, min(N, BLOCK * (pg + 1))))
+    return ranges, n_inter
+
+
+def select_blocks_mixed(q, K, q_pos0: int, causal: bool, budgets, inter_pages: int = 2,
+                        intra_first_page: int = -1, intra_budgets=None, group_tokens: int = 0,
+                        scale: float | None = None):
+    """Per (head, group): the budgets[h] best inter-chunk candidates and the
+    intra_budgets[h] best intra-chunk candidates (None: all of them), by the
+    pooled score mean_q . mean_k(candidate) * scale; ties to the earlier
+    candidate.  Returns (sel, scores): sel[h][g] = ascending int32 page ids,
+    scores[h, g, c] per candidate."""
+    Lq, H, d = q.shape
+    N = K.shape[0]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    ranges, n_inter = mixed_candidates(N, inter_pages, intra_first_page)
+    groups = group_bounds(Lq, group_tokens)
+    kbar = np.zeros((len(ranges), H, d))
+    for c, (t0, t1) in enumerate(ranges):
+        kbar[c] = _f64(K[t0:t1]).mean(axis=0)
+    first_tok = np.array([t0 for t0, _ in ranges], dtype=np.int64)
+    scores = np.zeros((H, len(groups), len(ranges)))
+    sel = []
+    for h in range(H):
+        row = []
+        for g, (a, e) in enumerate(groups):
+            qbar = _f64(q[a:e, h]).mean(axis=0)
+            scores[h, g] = (kbar[:, h, :] @ qbar) * scale
+            cand = np.ones(len(ranges), bool)
+            if causal:
+                cand &= first_tok <= (q_pos0 + e - 1)
+            inter = cand.copy()
+            inter[n_inter:] = False
+            intra = cand.copy()
+            intra[:n_inter] = False
+            chosen = list(select_topk(scores[h, g], inter, int(budgets[h])))
+            chosen += list(select_topk(scores[h, g], intra, -1 if intra_budgets is None else int(intra_budgets[h])))
+            pages = []
+            for c in sorted(chosen):
+                t0, t1 = ranges[c]
+                pages += list(range(t0 // BLOCK, (t1 + BLOCK - 1) // BLOCK))
+            row.append(np.array(pages, dtype=np.int32))
+        sel.append(row)
+    return sel, scores
+
+
+# --------------------------------------------------------------------------
 # sparse branch: O_sp = SDPA_block(Q, K, V; S^(h))  (Sparse branch, Eq. 4),
 # i.e. Eq. "attention" with M = 0 exactly on the visible keys of the selected
 # blocks and -inf elsewhere.

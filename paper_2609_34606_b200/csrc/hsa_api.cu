@@ -351,7 +351,16 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
                       int64_t q_pos0, int32_t causal, const int32_t* budgets_dev,
                       int32_t q_group_tokens, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
                       void* stream) {
+  return hsa_select_blocks_ex(ctx, q, n_q, tok_stride, head_stride, q_pos0, causal, budgets_dev, q_group_tokens,
+                              nullptr, sel_idx_dev, sel_cnt_dev, stream);
+}
+
+int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                         int64_t q_pos0, int32_t causal, const int32_t* budgets_dev,
+                         int32_t q_group_tokens, const hsa_select_opts* opts, int32_t* sel_idx_dev,
+                         int32_t* sel_cnt_dev, void* stream) {
   if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (opts && (opts->inter_block_pages < 0 || opts->inter_block_pages > 2)) return HSA_ERR_INVALID_ARG;
   if (n_q < 1 || n_q > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
   if (!tensor_args_ok(ctx, q, tok_stride, head_stride)) return HSA_ERR_INVALID_ARG;
   if (!budgets_dev || !sel_idx_dev || !sel_cnt_dev) return HSA_ERR_INVALID_ARG;
@@ -384,6 +393,11 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   a.barrier = reinterpret_cast<unsigned*>(ws + ctx->lay.status + 8);
   a.bar_host = &ctx->select_bar;
+  if (opts) {
+    a.inter_pages = opts->inter_block_pages;
+    a.intra_first_page1 = opts->intra_first_page >= 0 ? static_cast<int64_t>(opts->intra_first_page) + 1 : 0;
+    a.intra_budgets = opts->intra_budgets_dev;
+  }
   cudaError_t e = launch_select(a, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return HSA_OK;

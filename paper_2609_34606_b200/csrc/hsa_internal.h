@@ -67,6 +67,11 @@ struct SelectArgs {
   int32_t* status;
   unsigned* barrier;  // grid-barrier arrive counter for the single-launch path (null: three launches)
   GridBarrierHost* bar_host;  // host-side running total of that counter (null: cleared per launch)
+  // candidate geometry: pages before the first intra-chunk page are selected in runs of inter_pages pages against
+  // budgets[], the pages from it on one by one against intra_budgets[] (null: all of them)
+  int inter_pages;           // 0 or 1: every page on its own
+  int64_t intra_first_page1;  // first intra-chunk page + 1; 0: no intra-chunk region
+  const int32_t* intra_budgets;
 };
 
 struct FwdParams {

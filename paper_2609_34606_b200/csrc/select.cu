@@ -92,13 +92,60 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
 }
 
 // ---------------------------------------------------------------------------------------
+// Candidates.  A candidate is a run of consecutive pages that is scored and selected as one:
+// pages [0, p0) form "inter-chunk" candidates of `inter_pages` pages each (the last one may be
+// short), pages [p0, nblk) are "intra-chunk" candidates of one page each.  The default
+// (inter_pages = 1, p0 = nblk) makes every page its own candidate.
+// ---------------------------------------------------------------------------------------
+struct CandGeom {
+  int nblk, p0;
+  int ip;      // pages per inter-chunk candidate
+  int ni, nc;  // inter-chunk candidates, all candidates
+};
+// MIXED = false is the plain case, known at compile time: one page per candidate, no intra part
+template <bool MIXED>
+__device__ __forceinline__ CandGeom cand_geom(const SelectArgs& a) {
+  CandGeom g;
+  g.nblk = static_cast<int>((a.n_tokens + kBlock - 1) / kBlock);
+  if (!MIXED) {
+    g.ip = 1;
+    g.p0 = g.ni = g.nc = g.nblk;
+    return g;
+  }
+  g.ip = a.inter_pages > 1 ? a.inter_pages : 1;
+  g.p0 = (a.intra_first_page1 > 0 && a.intra_first_page1 <= g.nblk) ? static_cast<int>(a.intra_first_page1 - 1) : g.nblk;
+  g.ni = (g.p0 + g.ip - 1) / g.ip;
+  g.nc = g.ni + (g.nblk - g.p0);
+  return g;
+}
+template <bool MIXED>
+__device__ __forceinline__ int cand_first_page(const CandGeom& g, int c) {
+  if (!MIXED) return c;
+  return c < g.ni ? c * g.ip : g.p0 + (c - g.ni);
+}
+template <bool MIXED>
+__device__ __forceinline__ int cand_pages(const CandGeom& g, int c) {
+  if (!MIXED) return 1;
+  return c < g.ni ? min(g.ip, g.p0 - c * g.ip) : 1;
+}
+// candidates whose first token is at or before position p_last (they form a prefix)
+template <bool MIXED>
+__device__ __forceinline__ int cand_visible(const CandGeom& g, int64_t p_last) {
+  if (p_last < 0) return 0;
+  const int pg = static_cast<int>(min64(p_last / kBlock, g.nblk));  // page that holds p_last
+  if (!MIXED) return min(g.nblk, pg + 1);
+  if (pg < g.p0) return min(g.ni, pg / g.ip + 1);
+  return min(g.nc, g.ni + (pg - g.p0) + 1);
+}
+
+// ---------------------------------------------------------------------------------------
 // Stage 2: pooled scores.  grid (ceil(nblk/32), n_groups, H); one warp per block, four blocks
 // per warp.  The mean query of the group is rebuilt from the tile partials in fp64 (fixed
 // order), the dot product runs in fp64 and is rounded once to the fp32 sort key.
 // ---------------------------------------------------------------------------------------
 constexpr int kScoreBlocksPerCta = 32;
 
-template <int D>
+template <int D, bool MIXED>
 __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
@@ -132,35 +179,43 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   __syncthreads();
   constexpr int PER = D / 32;
   uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
-  constexpr int NB = kScoreBlocksPerCta / 8;  // blocks per warp
-  float kv[NB][PER];
+  const CandGeom cg = cand_geom<MIXED>(a);
+  constexpr int NB = kScoreBlocksPerCta / 8;  // candidates per warp
+  constexpr int NP = MIXED ? 2 : 1;           // pages per candidate at most
+  float kv[NB][NP][PER];
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
-    const int64_t b = static_cast<int64_t>(chunk) * kScoreBlocksPerCta + i * 8 + warp;
+    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+    const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
+    const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
 #pragma unroll
-    for (int e = 0; e < PER; ++e)
-      kv[i][e] = b < nblk ? a.ksum[(static_cast<size_t>(h) * a.max_pages + b) * D + lane * PER + e] : 0.f;
+    for (int pg = 0; pg < NP; ++pg)
+#pragma unroll
+      for (int e = 0; e < PER; ++e)
+        kv[i][pg][e] = pg < np ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp + pg) * D + lane * PER + e] : 0.f;
   }
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
-    const int64_t b = static_cast<int64_t>(chunk) * kScoreBlocksPerCta + i * 8 + warp;
-    if (b >= nblk) continue;  // warp-uniform
+    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+    if (c >= cg.nc) continue;  // warp-uniform
     double dot = 0.0;
 #pragma unroll
-    for (int e = 0; e < PER; ++e) dot += qs[lane * PER + e] * static_cast<double>(kv[i][e]);
+    for (int e = 0; e < PER; ++e)
+      dot += qs[lane * PER + e] * (static_cast<double>(kv[i][0][e]) + (MIXED ? static_cast<double>(kv[i][NP - 1][e]) : 0.0));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
     if (lane == 0) {
-      const int64_t cnt = min64(kBlock, a.n_tokens - b * kBlock);
-      keys[b] = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
+      const int64_t t0 = static_cast<int64_t>(cand_first_page<MIXED>(cg, c)) * kBlock;
+      const int64_t cnt = min64(static_cast<int64_t>(cand_pages<MIXED>(cg, c)) * kBlock, a.n_tokens - t0);
+      keys[c] = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
     }
   }
 }
 
-template <int D>
+template <int D, bool MIXED>
 __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   __shared__ double qs[D + 256];  // mean query, then the per-way partial sums
-  scores_item<D>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs);
+  scores_item<D, MIXED>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -175,30 +230,16 @@ struct TopkShared {
   int krem;
 };
 
-__device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
+// The `budget` largest keys of keys[0, n) (ties at the threshold to the lower index), emitted in
+// index order as the pages of candidates c0 + i; returns the number of pages emitted (whether or
+// not they fitted below kcap).  All 256 threads call it; keys live in shared memory.
+template <bool MIXED>
+__device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budget, const CandGeom& cg, int c0,
+                                          int32_t* out, int out_pos0, int kcap, TopkShared* sh) {
   int* hist = sh->hist;
   int* warp_sums = sh->warp_sums;
-  uint32_t& sh_prefix = sh->prefix;
-  int& sh_krem = sh->krem;
-  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
-  const int q_hi = min(a.n_q, g * gtok + gtok);
-  const int64_t p_last = a.q_pos0 + q_hi - 1;
-  // candidate blocks are a prefix [0, ncand)
-  int64_t ncand64 = nblk;
-  if (a.causal) ncand64 = max64(0, min64(nblk, p_last / kBlock + (p_last >= 0 ? 1 : 0)));
-  const int ncand = static_cast<int>(ncand64);
-  const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
-  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
-  if (threadIdx.x == 0) {
-    sh_prefix = 0;
-    sh_krem = 0;
-  }
-  __syncthreads();
-
-  int budget = a.budgets[h];
-  if (budget < 0 || budget > ncand) budget = ncand;
-  const bool take_all = (budget >= ncand);
+  if (budget < 0 || budget > n) budget = n;
+  const bool take_all = (budget >= n);
   uint32_t thr = 0;
   int need_ties = 0;
   if (!take_all && budget > 0) {
@@ -208,7 +249,7 @@ __device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uin
       const int shift = pass * 8;
       hist[threadIdx.x] = 0;
       __syncthreads();
-      for (int b = threadIdx.x; b < ncand; b += 256) {
+      for (int b = threadIdx.x; b < n; b += 256) {
         const uint32_t k = keys[b];
         if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
       }
@@ -219,12 +260,12 @@ __device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uin
       int tot;
       const int above = block_exclusive_scan(mine, warp_sums, &tot);  // keys in strictly higher bins
       if (above < krem && above + mine >= krem) {                     // exactly one thread
-        sh_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
-        sh_krem = krem - above;  // still to take among keys matching the longer prefix
+        sh->prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+        sh->krem = krem - above;  // still to take among keys matching the longer prefix
       }
       __syncthreads();
-      prefix = sh_prefix;
-      krem = sh_krem;
+      prefix = sh->prefix;
+      krem = sh->krem;
       mask |= 255u << shift;
     }
     thr = prefix;
@@ -232,55 +273,78 @@ __device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uin
   }
 
   // index-ordered compaction: thread t owns the contiguous range [t*per, t*per+per)
-  const int per = (ncand + 255) / 256;
-  const int lo = min(ncand, static_cast<int>(threadIdx.x) * per), hi = min(ncand, lo + per);
+  const int per = (n + 255) / 256;
+  const int lo = min(n, static_cast<int>(threadIdx.x) * per), hi = min(n, lo + per);
   int ties_before = 0, dummy;
   if (!take_all && budget > 0) {
     int my_ties = 0;
     for (int b = lo; b < hi; ++b) my_ties += (keys[b] == thr);
     ties_before = block_exclusive_scan(my_ties, warp_sums, &dummy);
   }
-  int my_sel = 0;
-  if (take_all) {
-    my_sel = hi - lo;
-  } else if (budget > 0) {
+  auto chosen = [&](int b, int& t) -> bool {
+    if (take_all) return true;
+    if (budget == 0) return false;
+    const uint32_t k = keys[b];
+    if (k == thr) return t++ < need_ties;
+    return k > thr;
+  };
+  int my_pages = 0;
+  {
     int t = ties_before;
-    for (int b = lo; b < hi; ++b) {
-      const uint32_t k = keys[b];
-      if (k > thr) ++my_sel;
-      else if (k == thr) { if (t < need_ties) ++my_sel; ++t; }
-    }
+    for (int b = lo; b < hi; ++b)
+      if (chosen(b, t)) my_pages += cand_pages<MIXED>(cg, c0 + b);
   }
   int total = 0;
-  int pos = block_exclusive_scan(my_sel, warp_sums, &total);
-  int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
+  int pos = out_pos0 + block_exclusive_scan(my_pages, warp_sums, &total);
   {
     int t = ties_before;
     for (int b = lo; b < hi; ++b) {
-      bool sel;
-      if (take_all) sel = true;
-      else if (budget == 0) sel = false;
-      else {
-        const uint32_t k = keys[b];
-        sel = (k > thr);
-        if (k == thr) { sel = (t < need_ties); ++t; }
-      }
-      if (sel) {
-        if (pos < a.kcap) out[pos] = b;
-        ++pos;
+      if (chosen(b, t)) {
+        const int fp = cand_first_page<MIXED>(cg, c0 + b);
+        const int np = cand_pages<MIXED>(cg, c0 + b);
+        for (int pg = 0; pg < np; ++pg, ++pos)
+          if (pos < kcap) out[pos] = fp + pg;
       }
     }
   }
+  __syncthreads();  // hist / warp_sums are reused by the next call
+  return total;
+}
+
+template <bool MIXED>
+__device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
+  const CandGeom cg = cand_geom<MIXED>(a);
+  const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
+  const int q_hi = min(a.n_q, g * gtok + gtok);
+  const int64_t p_last = a.q_pos0 + q_hi - 1;
+  // candidates are a prefix [0, ncand): all of them, or those that start at or before the group's
+  // last query position
+  const int ncand = a.causal ? cand_visible<MIXED>(cg, p_last) : cg.nc;
+  const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
+  if (threadIdx.x == 0) {
+    sh->prefix = 0;
+    sh->krem = 0;
+  }
+  __syncthreads();
+  int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
+  // inter-chunk candidates against the head's budget, then intra-chunk ones against theirs
+  const int n_inter = min(ncand, cg.ni);
+  int total = topk_range<MIXED>(keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh);
+  if (MIXED && ncand > n_inter)
+    total += topk_range<MIXED>(keys + n_inter, ncand - n_inter, a.intra_budgets ? a.intra_budgets[h] : -1, cg, cg.ni, out,
+                        total, a.kcap, sh);
   if (threadIdx.x == 0) {
     a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
     if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
   }
 }
 
+template <bool MIXED>
 __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   extern __shared__ uint32_t topk_keys[];
   __shared__ TopkShared sh;
-  topk_item(a, blockIdx.x, blockIdx.y, topk_keys, &sh);
+  topk_item<MIXED>(a, blockIdx.x, blockIdx.y, topk_keys, &sh);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -315,14 +379,13 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctr, unsigned target, int
   __syncthreads();
 }
 
-template <int D>
-__global__ void __launch_bounds__(256) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
+template <int D, bool MIXED>
+__global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
   extern __shared__ uint32_t fused_keys[];
   __shared__ __align__(16) unsigned char scratch[256 / (D / 8) * D * 4];  // tile-sum partials / mean query
   __shared__ TopkShared sh;
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
-  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  const int n_chunks = static_cast<int>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta);
+  const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
     qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
@@ -330,12 +393,12 @@ __global__ void __launch_bounds__(256) select_fused_kernel(SelectArgs a, unsigne
   grid_barrier(bar_ctr, bar_base + gridDim.x, a.status);
   for (int it = blockIdx.x; it < n_chunks * a.n_groups * a.H; it += gridDim.x) {
     const int chunk = it % n_chunks, gh = it / n_chunks;
-    scores_item<D>(a, chunk, gh % a.n_groups, gh / a.n_groups, reinterpret_cast<double*>(scratch));
+    scores_item<D, MIXED>(a, chunk, gh % a.n_groups, gh / a.n_groups, reinterpret_cast<double*>(scratch));
     __syncthreads();
   }
   grid_barrier(bar_ctr, bar_base + 2 * gridDim.x, a.status);
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
-    topk_item(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
+    topk_item<MIXED>(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
     __syncthreads();
   }
 }
@@ -505,9 +568,9 @@ cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, 
   if (nblk > 0) {
     dim3 g2(static_cast<unsigned>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta), a.n_groups, a.H);
     if (a.D == 128)
-      block_scores_kernel<128><<<g2, 256, 0, st>>>(a);
+      block_scores_kernel<128, false><<<g2, 256, 0, st>>>(a);
     else
-      block_scores_kernel<64><<<g2, 256, 0, st>>>(a);
+      block_scores_kernel<64, false><<<g2, 256, 0, st>>>(a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -543,14 +606,17 @@ bool coop_info(int* nsm) {
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   int nsm = 0;
+  const bool mixed = a.inter_pages > 1 || a.intra_first_page1 > 0;
   if (a.barrier && coop_info(&nsm)) {
     // one cooperative launch for all three stages
     const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;
     const size_t smem_keys = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
     SelectArgs aa = a;
     unsigned* ctr = a.barrier;
-    const void* fn = a.D == 128 ? reinterpret_cast<const void*>(select_fused_kernel<128>)
-                                : reinterpret_cast<const void*>(select_fused_kernel<64>);
+    const void* fn = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(select_fused_kernel<128, true>)
+                                         : reinterpret_cast<const void*>(select_fused_kernel<128, false>))
+                                : (mixed ? reinterpret_cast<const void*>(select_fused_kernel<64, true>)
+                                         : reinterpret_cast<const void*>(select_fused_kernel<64, false>));
     if (smem_keys > 24 * 1024)
       cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_keys));
     // 256 threads, 48..57 registers and under 12 KB of shared memory per CTA plus the keys:
@@ -591,18 +657,31 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   if (nblk > 0) {
     dim3 g2(static_cast<unsigned>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta), a.n_groups, a.H);
-    if (a.D == 128)
-      block_scores_kernel<128><<<g2, 256, 0, st>>>(a);
-    else
-      block_scores_kernel<64><<<g2, 256, 0, st>>>(a);
+    if (a.D == 128) {
+      if (mixed)
+        block_scores_kernel<128, true><<<g2, 256, 0, st>>>(a);
+      else
+        block_scores_kernel<128, false><<<g2, 256, 0, st>>>(a);
+    } else {
+      if (mixed)
+        block_scores_kernel<64, true><<<g2, 256, 0, st>>>(a);
+      else
+        block_scores_kernel<64, false><<<g2, 256, 0, st>>>(a);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   const size_t smem = static_cast<size_t>(nblk > 0 ? nblk : 1) * sizeof(uint32_t);
-  if (smem > 40 * 1024)
-    cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   dim3 g3(a.n_groups, a.H);
-  topk_kernel<<<g3, 256, smem, st>>>(a);
+  if (mixed) {
+    if (smem > 40 * 1024)
+      cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    topk_kernel<true><<<g3, 256, smem, st>>>(a);
+  } else {
+    if (smem > 40 * 1024)
+      cudaFuncSetAttribute(topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    topk_kernel<false><<<g3, 256, smem, st>>>(a);
+  }
   return cudaGetLastError();
 }
 
@@ -693,6 +772,6 @@ extern "C" int hsa_select_blocks_noalloc(const void* q, int32_t n_q, int64_t tok
   a.sel_cnt = sel_cnt_dev;
   a.kcap = max_topk;
   a.status = status_dev ? status_dev : reinterpret_cast<int32_t*>(sc);
-  a.barrier = reinterpret_cast<unsigned*>(sc + 16);
+  // (no grid-barrier counter: this entry point runs the three stages as three launches)
   return launch_select(a, st) == cudaSuccess ? HSA_OK : HSA_ERR_CUDA;
 }

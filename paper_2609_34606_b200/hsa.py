@@ -36,7 +36,8 @@ PAGE_TOKENS = 64
 TILE_M = 128
 
 EXPORTS = [
-    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_adaptive",
+    "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_ex",
+    "hsa_select_blocks_adaptive",
     "hsa_select_blocks_noalloc",
     "hsa_forward",
     "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
@@ -50,6 +51,11 @@ class hsa_config(C.Structure):
                 ("max_pages", C.c_int32), ("max_q_tokens", C.c_int32), ("max_topk", C.c_int32),
                 ("lin_mode", C.c_int32), ("gate_act", C.c_int32), ("softmax_scale", C.c_float),
                 ("flags", C.c_uint32), ("lin_rank", C.c_int32), ("lin_seg_tokens", C.c_int32)]
+
+
+class hsa_select_opts(C.Structure):
+    _fields_ = [("inter_block_pages", C.c_int32), ("intra_first_page", C.c_int32),
+                ("intra_budgets_dev", C.c_void_p)]
 
 
 class hsa_sizes(C.Structure):
@@ -74,6 +80,8 @@ def _load() -> C.CDLL:
     lib.hsa_create.argtypes = [C.POINTER(vp), C.POINTER(hsa_config), C.POINTER(hsa_buffers), vp]
     lib.hsa_append_kv.argtypes = [vp, vp, vp, i32, i64, i64, vp]
     lib.hsa_select_blocks.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp, vp]
+    lib.hsa_select_blocks_ex.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, C.POINTER(hsa_select_opts), vp, vp,
+                                         vp]
     lib.hsa_select_blocks_adaptive.argtypes = [vp, vp, i32, i64, i64, i64, i32, C.c_float, C.c_float, i32, vp, vp,
                                                vp, vp]
     lib.hsa_select_blocks_noalloc.argtypes = [vp, i32, i64, i64, i32, i32, vp, i32, i64, i64, i32, C.c_float,
@@ -160,6 +168,16 @@ def hsa_select_blocks(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budg
     _check(_lib.hsa_select_blocks(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
                                   budgets.data_ptr(), int(q_group_tokens), sel_idx.data_ptr(),
                                   sel_cnt.data_ptr(), _stream()), "hsa_select_blocks")
+
+
+def hsa_select_blocks_ex(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budgets: torch.Tensor,
+                         q_group_tokens: int, inter_block_pages: int, intra_first_page: int,
+                         intra_budgets: Optional[torch.Tensor], sel_idx: torch.Tensor, sel_cnt: torch.Tensor) -> None:
+    ts, hs = _thd(q, "q")
+    opts = hsa_select_opts(int(inter_block_pages), int(intra_first_page), _ptr(intra_budgets))
+    _check(_lib.hsa_select_blocks_ex(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
+                                     budgets.data_ptr(), int(q_group_tokens), C.byref(opts), sel_idx.data_ptr(),
+                                     sel_cnt.data_ptr(), _stream()), "hsa_select_blocks_ex")
 
 
 def hsa_select_blocks_adaptive(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, tau_min: float,
@@ -316,6 +334,17 @@ class HSAContext:
         q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
         sel_idx, sel_cnt = sel if sel is not None else self.alloc_selection(q.shape[0], group_tokens)
         hsa_select_blocks(self.ctx, q, q_pos0, causal, budgets, group_tokens, sel_idx, sel_cnt)
+        return sel_idx, sel_cnt
+
+    def select_blocks_ex(self, q: torch.Tensor, budgets: torch.Tensor, inter_block_pages: int = 2,
+                         intra_first_page: int = -1, intra_budgets: Optional[torch.Tensor] = None,
+                         q_pos0: Optional[int] = None, causal: bool = False, group_tokens: int = 0, sel=None):
+        """Selection with coarse inter-chunk blocks (runs of inter_block_pages pages) and single-page
+        intra-chunk blocks from intra_first_page on (see hsa_select_blocks_ex)."""
+        q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
+        sel_idx, sel_cnt = sel if sel is not None else self.alloc_selection(q.shape[0], group_tokens)
+        hsa_select_blocks_ex(self.ctx, q, q_pos0, causal, budgets, group_tokens, inter_block_pages,
+                             intra_first_page, intra_budgets, sel_idx, sel_cnt)
         return sel_idx, sel_cnt
 
     def select_blocks_adaptive(self, q: torch.Tensor, tau_min: float, tau_max: float,

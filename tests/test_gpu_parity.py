@@ -429,3 +429,56 @@ def test_head_adaptive_selection(name, group_tokens, cuda_device):
     out = Hn.f64(ctx.forward(qd, si, sc, group_tokens=group_tokens))
     Hn.assert_close(out, ref["out"], "out")
     ctx.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,causal", [("mid_d128", False), ("mid_mix", False), ("mid_causal", True), ("mid_d64", False)])
+def test_inter_and_intra_chunk_granularity(name, causal, cuda_device):
+    """128-token inter-chunk blocks against the head budgets plus the chunk's own 64-token pages
+    (always on, then with their own budgets); the page lists drive the unchanged forward kernel."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS[name]
+    ctx = Hn.build_context(w, cuda_device, causal=causal)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    Kn, Vn = Hn.f32(K), Hn.f32(V)
+    q = W.gen_query(w)
+    qn, qd = Hn.f32(q), q.to(cuda_device)
+    N = Kn.shape[0]
+    q_pos0 = w.q_pos0
+    p0 = max(0, (N - w.chunk)) // 64            # page that holds the first token of the last chunk
+    budgets = W.gen_budgets(w)
+    intra_b = torch.full((w.H,), 2, dtype=torch.int32)
+
+    def cands_of(pages, ranges):
+        first = {t0 // 64: c for c, (t0, _) in enumerate(ranges)}
+        return sorted({first[p] for p in pages if p in first})
+
+    for inter_pages, first_page, ib in ((2, -1, None), (2, p0, None), (2, p0, intra_b), (1, p0, intra_b)):
+        si, sc = ctx.select_blocks_ex(qd, budgets.to(cuda_device), inter_block_pages=inter_pages,
+                                      intra_first_page=first_page,
+                                      intra_budgets=None if ib is None else ib.to(cuda_device),
+                                      q_pos0=q_pos0, causal=causal)
+        assert ctx.device_status() == 0
+        got = Hn.selection_lists(si, sc)
+        ref, scores = O.select_blocks_mixed(qn, Kn, q_pos0, causal, budgets.tolist(), inter_pages, first_page,
+                                            None if ib is None else ib.tolist())
+        ranges, n_inter = O.mixed_candidates(N, inter_pages, first_page)
+        for h in range(w.H):
+            a, b = got[h][0].tolist(), ref[h][0].tolist()
+            assert a == sorted(set(a))
+            if a != b:   # only candidates whose score ties the weakest selected one may differ
+                ca, cb = cands_of(a, ranges), cands_of(b, ranges)
+                assert len(ca) == len(cb)
+                diff = sorted(set(ca) ^ set(cb))
+                for part in (range(0, n_inter), range(n_inter, len(ranges))):
+                    sel_part = [c for c in cb if c in part]
+                    d_part = [c for c in diff if c in part]
+                    if d_part:
+                        kth = min(scores[h, 0, c] for c in sel_part)
+                        assert all(abs(scores[h, 0, c] - kth) <= Hn.TIE_EPS for c in d_part), (h, d_part)
+        # the forward kernel runs on the page lists as they are
+        rows = W.sample_rows(w, n_random=64).numpy()
+        out = Hn.f64(ctx.forward(qd, si, sc, q_pos0=q_pos0, causal=causal, flags=hsa.HSA_FWD_NO_LINEAR))
+        o_ref = O.sparse_branch(qn, Kn, Vn, got, q_pos0, causal, rows=rows)
+        Hn.assert_close(out[rows], o_ref[rows], "O_sp")
+    ctx.destroy()

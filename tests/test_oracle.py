@@ -370,3 +370,60 @@ def test_adaptive_selection_per_group_gini_is_averaged():
         p = O.block_weights(s[0, g], np.ones(9, bool))
         gs.append(O.gini_of_weights(np.sort(p)[::-1]))
     assert abs(gini[0] - np.mean(gs)) < 1e-14 and len(sel[0]) == 3
+
+
+# ---------------------------------------------------------------- inter- / intra-chunk granularity
+def test_mixed_selection_reduces_to_plain_selection():
+    """One page per inter-chunk block and no intra-chunk region is the plain per-page selection."""
+    q, K = rnd((12, 2, 8), 70), rnd((300, 2, 8), 71)
+    for causal, q_pos0 in ((False, 300), (True, 200)):
+        ref, s_ref = O.select_blocks(q, K, q_pos0, causal, [2, 3])
+        got, s_got = O.select_blocks_mixed(q, K, q_pos0, causal, [2, 3], inter_pages=1, intra_first_page=-1)
+        assert all(np.array_equal(got[h][0], ref[h][0]) for h in range(2))
+        assert np.allclose(s_got, s_ref, rtol=0, atol=1e-14)
+
+
+def test_coarse_block_score_is_token_weighted_mean_of_its_pages():
+    """mean over a 128-token block = (c0 mean0 + c1 mean1) / (c0 + c1): the coarse score follows from
+    the per-page scores and the page token counts (here the last block is one and a bit pages)."""
+    N = 64 * 4 + 64 + 10
+    q, K = rnd((7, 1, 8), 72), rnd((N, 1, 8), 73)
+    page = O.block_scores(q, K)[0, 0]
+    _, s = O.select_blocks_mixed(q, K, N, False, [1], inter_pages=2, intra_first_page=-1)
+    cnt = [O.block_count(b, N) for b in range(O.n_blocks(N))]
+    for c in range(3):
+        b0, b1 = 2 * c, 2 * c + 1
+        want = (cnt[b0] * page[b0] + cnt[b1] * page[b1]) / (cnt[b0] + cnt[b1])
+        assert abs(s[0, 0, c] - want) < 1e-12
+
+
+def test_mixed_selection_brute_force_and_intra_always_on():
+    """Pure-Python loops over tokens: coarse blocks ranked by their own mean key, chunk pages always kept."""
+    N, H, d, Lq = 64 * 5 + 20, 2, 4, 5
+    q, K = rnd((Lq, H, d), 74), rnd((N, H, d), 75)
+    p0 = 4                                    # pages 4 and 5 belong to the current chunk
+    got, _ = O.select_blocks_mixed(q, K, N, False, [1, 2], inter_pages=2, intra_first_page=p0)
+    for h in range(H):
+        qbar = [sum(float(q[i, h, c]) for i in range(Lq)) / Lq for c in range(d)]
+        sc = []
+        for c in range(2):                    # coarse blocks = pages (0,1) and (2,3)
+            toks = range(128 * c, 128 * c + 128)
+            kbar = [sum(float(K[j, h, e]) for j in toks) / 128 for e in range(d)]
+            sc.append(sum(a * b for a, b in zip(qbar, kbar)) / math.sqrt(d))
+        keep = brute.topk_blocks(sc, [True, True], [1, 2][h])
+        pages = sorted(sum(([2 * c, 2 * c + 1] for c in keep), [])) + [4, 5]
+        assert got[h][0].tolist() == pages
+    # an intra-chunk budget selects among the chunk's own pages only, by their own scores
+    got2, s2 = O.select_blocks_mixed(q, K, N, False, [0, 0], inter_pages=2, intra_first_page=p0, intra_budgets=[1, 1])
+    for h in range(H):
+        assert got2[h][0].tolist() == [4 + int(np.argmax(s2[h, 0, 2:]))]
+
+
+def test_mixed_selection_causal_candidates_and_ragged_inter_region():
+    N = 64 * 7
+    q, K = rnd((4, 1, 4), 76), rnd((N, 1, 4), 77)
+    ranges, n_inter = O.mixed_candidates(N, 2, 5)      # 5 history pages -> blocks (0,1), (2,3), (4)
+    assert n_inter == 3 and ranges[:3] == [(0, 128), (128, 256), (256, 320)] and ranges[3:] == [(320, 384), (384, 448)]
+    # last query position 200: candidates are the blocks that start at or before it
+    got, _ = O.select_blocks_mixed(q, K, 197, True, [-1], inter_pages=2, intra_first_page=5)
+    assert got[0][0].tolist() == [0, 1, 2, 3]
