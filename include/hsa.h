@@ -150,18 +150,55 @@ int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stri
  *                       own, outside budgets_dev.
  *   intra_budgets_dev   device int32[H] budgets for those pages, or NULL = every one of them
  *                       (the chunk always attends to itself).
+ *   kv_pages_dev        device int32[n_kv_pages]: ids of the KV pages kept by hsa_retrieve_kv_pages
+ *                       (runs of kv_page_blocks blocks), or NULL for no mask.  An inter-chunk block
+ *                       with a page outside them is no candidate at all: the retrieved pages are
+ *                       the ones that are resident (Section 3.2, "Active KV construction").  The
+ *                       chunk's own pages are never masked.
  * max_topk must hold inter_block_pages * budget + the intra-chunk pages.  opts == NULL is
  * hsa_select_blocks.  Everything else as hsa_select_blocks. */
 typedef struct {
   int32_t inter_block_pages;
   int32_t intra_first_page;
   const int32_t* intra_budgets_dev;
+  const int32_t* kv_pages_dev;
+  int32_t n_kv_pages;
+  int32_t kv_page_blocks;
 } hsa_select_opts;
 int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
                          int64_t head_stride, int64_t q_pos0, int32_t causal,
                          const int32_t* budgets_dev, int32_t q_group_tokens,
                          const hsa_select_opts* opts, int32_t* sel_idx_dev, int32_t* sel_cnt_dev,
                          void* stream);
+
+/* Page-level retrieval of the hierarchical KV cache (Section 3.2, Stage 2).  A KV page is a run of
+ * kv_page_blocks consecutive 64-token blocks of the history (the paper's page of 8 frames x 1560
+ * tokens is 195 blocks).  Its score is alpha_j = Qbar . Kbar_j * scale with the average query of the
+ * chunk and the average key of the page, averaged over the heads (the paper is silent on heads: one
+ * set of pages serves the whole layer); the top_kp best pages (the paper uses K_p = 4; ties to the
+ * lower id) are written in ascending order.
+ *   page_ids_dev   device int32[min(top_kp, pages)] (output); pages = ceil(blocks / kv_page_blocks)
+ *   scores_dev     device fp32[pages] receiving every alpha_j, or NULL
+ *   n_out_host     host int32 receiving min(top_kp, pages) (known without a device read), or NULL
+ * The ids feed hsa_select_opts.kv_pages_dev.  HSA_ERR_UNSUPPORTED above 2048 pages. */
+int hsa_retrieve_kv_pages(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
+                          int64_t head_stride, int32_t kv_page_blocks, int32_t top_kp,
+                          int32_t* page_ids_dev, float* scores_dev, int32_t* n_out_host, void* stream);
+
+/* Tier migration of the hierarchical KV cache (Section 3.2: pages that are not retrieved leave the
+ * GPU for host memory and come back on demand).  The K and V tiles of history blocks
+ * [first_block, first_block + n_blocks) are copied to / from caller-owned host buffers laid out as
+ * [n_blocks][H][64][d] bf16 (pinned memory makes the copies asynchronous), one copy per run of
+ * physically adjacent pages, on the given stream.  The context only tracks residency on the host:
+ * an evicted block keeps its key sum (it still takes part in scoring) but its tiles must be restored
+ * before a forward call selects it -- restrict the selection with kv_pages_dev, or check with
+ * hsa_block_resident.  Appending to a block marks it resident.  HSA_ERR_INVALID_ARG outside the
+ * history. */
+int hsa_evict_blocks(hsa_ctx* ctx, int32_t first_block, int32_t n_blocks, void* host_k, void* host_v,
+                     void* stream);
+int hsa_restore_blocks(hsa_ctx* ctx, int32_t first_block, int32_t n_blocks, const void* host_k,
+                       const void* host_v, void* stream);
+int hsa_block_resident(hsa_ctx* ctx, int32_t block, int32_t* resident_out);
 
 /* Head-adaptive selection (Appendix F, Eq. 12-13): instead of a given budget, each (head, group)
  * keeps the shortest prefix of its blocks, sorted by pooled score, whose softmax mass reaches

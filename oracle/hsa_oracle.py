@@ -176,6 +176,38 @@ def select_blocks(q, K, q_pos0: int, causal: bool, budgets, group_tokens: int = 
 # and that a coarse block is scored by the mean key over all its tokens are
 # this implementation's readings.
 # --------------------------------------------------------------------------
+# --------------------------------------------------------------------------
+# HKV Stage 2, page-level retrieval (Sec. 3.2): a KV page is a run of
+# kv_page_blocks consecutive 64-token blocks (8 frames x 1560 tokens = 195
+# blocks in the paper's setting); its score is
+#     alpha_j = Qbar^T Kbar_j / sqrt(d_k)
+# with the average query of the current chunk and the average key of the
+# page, and the top-K_p pages (K_p = 4 in the paper) are kept.  The paper
+# writes Qbar, Kbar_j in R^{d_k} and is silent on heads: here the score is
+# averaged over the heads, so that one set of pages serves the whole layer
+# (a reading of this implementation).
+# --------------------------------------------------------------------------
+def kv_page_scores(q, K, kv_page_blocks: int, scale: float | None = None):
+    """alpha[j] for every KV page j that holds at least one token."""
+    Lq, H, d = q.shape
+    N = K.shape[0]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    ptok = BLOCK * int(kv_page_blocks)
+    npages = (N + ptok - 1) // ptok
+    qbar = _f64(q).mean(axis=0)                                   # [H, d]
+    alpha = np.zeros(npages)
+    for j in range(npages):
+        kbar = _f64(K[ptok * j:min(N, ptok * (j + 1))]).mean(axis=0)   # [H, d]
+        alpha[j] = float(np.mean(np.sum(qbar * kbar, axis=1))) * scale
+    return alpha
+
+
+def retrieve_kv_pages(q, K, kv_page_blocks: int, top_kp: int, scale: float | None = None):
+    """Ascending ids of the top_kp best-scoring KV pages (ties to the lower id)."""
+    alpha = kv_page_scores(q, K, kv_page_blocks, scale)
+    return select_topk(alpha, np.ones(alpha.size, bool), int(top_kp)), alpha
+
+
 def mixed_candidates(N: int, inter_pages: int, intra_first_page: int):
     """Token ranges [(t0, t1), ...] of the candidates in history order: runs of
     inter_pages pages below intra_first_page (the last run may be short), then
@@ -196,11 +228,15 @@ def mixed_candidates(N: int, inter_pages: int, intra_first_page: int):
 
 def select_blocks_mixed(q, K, q_pos0: int, causal: bool, budgets, inter_pages: int = 2,
                         intra_first_page: int = -1, intra_budgets=None, group_tokens: int = 0,
-                        scale: float | None = None):
+                        scale: float | None = None, kv_pages=None, kv_page_blocks: int = 0):
     """Per (head, group): the budgets[h] best inter-chunk candidates and the
     intra_budgets[h] best intra-chunk candidates (None: all of them), by the
     pooled score mean_q . mean_k(candidate) * scale; ties to the earlier
-    candidate.  Returns (sel, scores): sel[h][g] = ascending int32 page ids,
+    candidate.  kv_pages (with kv_page_blocks): ids of the retrieved KV pages;
+    an inter-chunk candidate with a page outside them is no candidate at all
+    (the retrieved pages are what is resident, Sec. 3.2 "Active KV
+    construction").
+    Returns (sel, scores): sel[h][g] = ascending int32 page ids,
     scores[h, g, c] per candidate."""
     Lq, H, d = q.shape
     N = K.shape[0]
@@ -223,6 +259,12 @@ def select_blocks_mixed(q, K, q_pos0: int, causal: bool, budgets, inter_pages: i
                 cand &= first_tok <= (q_pos0 + e - 1)
             inter = cand.copy()
             inter[n_inter:] = False
+            if kv_pages is not None:
+                allowed = set(int(j) for j in kv_pages)
+                for c in range(n_inter):
+                    first_pg, last_pg = ranges[c][0] // BLOCK, (ranges[c][1] - 1) // BLOCK
+                    if any(pg // int(kv_page_blocks) not in allowed for pg in (first_pg, last_pg)):
+                        inter[c] = False
             intra = cand.copy()
             intra[:n_inter] = False
             chosen = list(select_topk(scores[h, g], inter, int(budgets[h])))

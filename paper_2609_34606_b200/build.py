@@ -9,7 +9,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libhsa.so")
-SOURCES = ["hsa_api.cu", "append.cu", "select.cu", "forward.cu", "linear_causal.cu", "linformer.cu", "linear_only.cu"]
+SOURCES = ["hsa_api.cu", "append.cu", "select.cu", "forward.cu", "linear_causal.cu", "linformer.cu", "linear_only.cu", "retrieve.cu"]
 
 
 def nvcc_path() -> str:

@@ -119,6 +119,8 @@ struct hsa_ctx {
   int nsm;
   CUtensorMap tm_k, tm_v, tm_state, tm_kc, tm_vc, tm_olin;
   int32_t n_segs;  // Linformer: complete segments compressed so far
+  std::vector<int32_t> page_table_host;  // history block -> physical page
+  std::vector<uint8_t> resident;         // per history block: tiles present in the pool (tier migration)
   int last_cuda_error;
 };
 
@@ -215,6 +217,8 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   ctx->last_append = 0;
   ctx->last_cuda_error = 0;
   ctx->n_segs = 0;
+  ctx->page_table_host = pt;
+  ctx->resident.assign(static_cast<size_t>(cfg->max_pages), 1);
   const bool linformer = cfg->lin_mode == HSA_LIN_LINFORMER;
   if (linformer) {
     if (!bufs->kc_pool || !bufs->vc_pool || !bufs->e_k || !bufs->e_v || !aligned(bufs->kc_pool, 256) ||
@@ -342,6 +346,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->n_segs += 1;
   }
+  for (int64_t b = ctx->n_tokens / kBlock; b <= (n1 - 1) / kBlock; ++b) ctx->resident[static_cast<size_t>(b)] = 1;
   ctx->n_tokens = n1;
   ctx->last_append = n_tokens;
   return HSA_OK;
@@ -397,6 +402,12 @@ int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_s
     a.inter_pages = opts->inter_block_pages;
     a.intra_first_page1 = opts->intra_first_page >= 0 ? static_cast<int64_t>(opts->intra_first_page) + 1 : 0;
     a.intra_budgets = opts->intra_budgets_dev;
+    if (opts->kv_pages_dev) {
+      if (opts->n_kv_pages < 0 || opts->n_kv_pages > 64 || opts->kv_page_blocks < 1) return HSA_ERR_INVALID_ARG;
+      a.kv_pages = opts->kv_pages_dev;
+      a.n_kv_pages = opts->n_kv_pages;
+      a.kv_page_blocks = opts->kv_page_blocks;
+    }
   }
   cudaError_t e = launch_select(a, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e);
@@ -577,6 +588,97 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   else
     e = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return HSA_OK;
+}
+
+int hsa_retrieve_kv_pages(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, int64_t head_stride,
+                          int32_t kv_page_blocks, int32_t top_kp, int32_t* page_ids_dev, float* scores_dev,
+                          int32_t* n_out_host, void* stream) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (n_q < 1 || n_q > ctx->cfg.max_q_tokens) return HSA_ERR_INVALID_ARG;
+  if (!tensor_args_ok(ctx, q, tok_stride, head_stride)) return HSA_ERR_INVALID_ARG;
+  if (kv_page_blocks < 1 || top_kp < 0 || top_kp > 64 || !page_ids_dev) return HSA_ERR_INVALID_ARG;
+  const int64_t nblk = (ctx->n_tokens + kBlock - 1) / kBlock;
+  const int64_t n_pages = (nblk + kv_page_blocks - 1) / kv_page_blocks;
+  if (n_pages > 2048) return HSA_ERR_UNSUPPORTED;
+  if (n_out_host) *n_out_host = static_cast<int32_t>(n_pages < top_kp ? n_pages : top_kp);
+  if (n_pages == 0 || top_kp == 0) return HSA_OK;
+  uint8_t* stt = static_cast<uint8_t*>(ctx->buf.state);
+  uint8_t* ws = static_cast<uint8_t*>(ctx->buf.workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SelectArgs sa{};
+  sa.q = static_cast<const __nv_bfloat16*>(q);
+  sa.n_q = n_q;
+  sa.tok_stride = tok_stride;
+  sa.head_stride = head_stride;
+  sa.H = ctx->cfg.num_heads;
+  sa.D = ctx->cfg.head_dim;
+  sa.qpart = reinterpret_cast<float*>(ws + ctx->lay.qpart);
+  cudaError_t e = launch_qsum(sa, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  RetrieveArgs ra{};
+  ra.n_q = n_q;
+  ra.H = sa.H;
+  ra.D = sa.D;
+  ra.max_pages = ctx->cfg.max_pages;
+  ra.n_tokens = ctx->n_tokens;
+  ra.qpart = sa.qpart;
+  ra.ksum = reinterpret_cast<const float*>(stt + ctx->lay.ksum);
+  ra.kv_page_blocks = kv_page_blocks;
+  ra.top_kp = top_kp;
+  ra.scale = ctx->scale;
+  ra.keys = reinterpret_cast<uint32_t*>(ws + ctx->lay.keys);
+  ra.scores_out = scores_dev;
+  ra.page_ids = page_ids_dev;
+  e = launch_retrieve(ra, static_cast<int>(n_pages), st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return HSA_OK;
+}
+
+namespace {
+// Copies the tiles of blocks [b0, b0 + n) between the pools and host buffers, one cudaMemcpyAsync
+// per pool and run of physically adjacent pages.
+int migrate_blocks(hsa_ctx* ctx, int32_t b0, int32_t n, void* host_k, void* host_v, bool to_host, void* stream) {
+  if (!ctx || !host_k || !host_v || b0 < 0 || n < 0) return HSA_ERR_INVALID_ARG;
+  const int64_t nblk = (ctx->n_tokens + kBlock - 1) / kBlock;
+  if (static_cast<int64_t>(b0) + n > nblk) return HSA_ERR_INVALID_ARG;
+  const size_t tile = static_cast<size_t>(ctx->cfg.num_heads) * kBlock * ctx->cfg.head_dim * 2;  // one page, one pool
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* pools[2] = {static_cast<uint8_t*>(ctx->buf.k_pool), static_cast<uint8_t*>(ctx->buf.v_pool)};
+  uint8_t* hosts[2] = {static_cast<uint8_t*>(host_k), static_cast<uint8_t*>(host_v)};
+  int32_t i = 0;
+  while (i < n) {
+    int32_t run = 1;
+    const int32_t p_first = ctx->page_table_host[static_cast<size_t>(b0 + i)];
+    while (i + run < n && ctx->page_table_host[static_cast<size_t>(b0 + i + run)] == p_first + run) ++run;
+    for (int w = 0; w < 2; ++w) {
+      uint8_t* dev = pools[w] + static_cast<size_t>(p_first) * tile;
+      uint8_t* host = hosts[w] + static_cast<size_t>(i) * tile;
+      cudaError_t e = to_host ? cudaMemcpyAsync(host, dev, run * tile, cudaMemcpyDeviceToHost, st)
+                              : cudaMemcpyAsync(dev, host, run * tile, cudaMemcpyHostToDevice, st);
+      if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    i += run;
+  }
+  for (int32_t b = b0; b < b0 + n; ++b) ctx->resident[static_cast<size_t>(b)] = to_host ? 0 : 1;
+  return HSA_OK;
+}
+}  // namespace
+
+int hsa_evict_blocks(hsa_ctx* ctx, int32_t first_block, int32_t n_blocks, void* host_k, void* host_v,
+                     void* stream) {
+  return migrate_blocks(ctx, first_block, n_blocks, host_k, host_v, true, stream);
+}
+
+int hsa_restore_blocks(hsa_ctx* ctx, int32_t first_block, int32_t n_blocks, const void* host_k,
+                       const void* host_v, void* stream) {
+  return migrate_blocks(ctx, first_block, n_blocks, const_cast<void*>(host_k), const_cast<void*>(host_v), false,
+                        stream);
+}
+
+int hsa_block_resident(hsa_ctx* ctx, int32_t block, int32_t* resident_out) {
+  if (!ctx || !resident_out || block < 0 || block >= ctx->cfg.max_pages) return HSA_ERR_INVALID_ARG;
+  *resident_out = ctx->resident[static_cast<size_t>(block)];
   return HSA_OK;
 }
 

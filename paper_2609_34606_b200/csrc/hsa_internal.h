@@ -72,6 +72,22 @@ struct SelectArgs {
   int inter_pages;           // 0 or 1: every page on its own
   int64_t intra_first_page1;  // first intra-chunk page + 1; 0: no intra-chunk region
   const int32_t* intra_budgets;
+  // retrieved KV pages (runs of kv_page_blocks blocks): an inter-chunk candidate with a page outside
+  // them is no candidate (null: no mask)
+  const int32_t* kv_pages;
+  int n_kv_pages, kv_page_blocks;
+};
+
+struct RetrieveArgs {
+  int n_q, H, D, max_pages;
+  int64_t n_tokens;
+  const float* qpart;  // [tiles][H][D] query tile sums
+  const float* ksum;   // [H][max_pages][D]
+  int kv_page_blocks, top_kp;
+  float scale;
+  uint32_t* keys;      // [pages] scratch
+  float* scores_out;   // [pages] or null
+  int32_t* page_ids;   // [min(top_kp, pages)] ascending (output)
 };
 
 struct FwdParams {
@@ -147,6 +163,8 @@ struct AdaptiveArgs {
 };
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st);  // stage 1 alone: query tile sums
+cudaError_t launch_retrieve(const RetrieveArgs& a, int n_pages, cudaStream_t st);
 cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, cudaStream_t st);
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,

@@ -207,7 +207,19 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
     if (lane == 0) {
       const int64_t t0 = static_cast<int64_t>(cand_first_page<MIXED>(cg, c)) * kBlock;
       const int64_t cnt = min64(static_cast<int64_t>(cand_pages<MIXED>(cg, c)) * kBlock, a.n_tokens - t0);
-      keys[c] = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
+      uint32_t key = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
+      if (MIXED && a.kv_pages != nullptr && c < cg.ni) {
+        // every page of the candidate must lie in a retrieved KV page; key 0 marks "no candidate"
+        const int pf = cand_first_page<MIXED>(cg, c), pl = pf + cand_pages<MIXED>(cg, c) - 1;
+        bool in_f = false, in_l = false;
+        for (int i = 0; i < a.n_kv_pages; ++i) {
+          const int kp = a.kv_pages[i];
+          in_f |= (pf / a.kv_page_blocks == kp);
+          in_l |= (pl / a.kv_page_blocks == kp);
+        }
+        if (!(in_f && in_l)) key = 0u;
+      }
+      keys[c] = key;
     }
   }
 }
@@ -235,11 +247,20 @@ struct TopkShared {
 // not they fitted below kcap).  All 256 threads call it; keys live in shared memory.
 template <bool MIXED>
 __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budget, const CandGeom& cg, int c0,
-                                          int32_t* out, int out_pos0, int kcap, TopkShared* sh) {
+                                          int32_t* out, int out_pos0, int kcap, TopkShared* sh, bool masked) {
   int* hist = sh->hist;
   int* warp_sums = sh->warp_sums;
-  if (budget < 0 || budget > n) budget = n;
-  const bool take_all = (budget >= n);
+  // keys equal to 0 are masked-out candidates (no finite score maps to 0): they are never chosen
+  int n_eff = n;
+  if (MIXED && masked) {
+    int my0 = 0, tot0 = 0;
+    for (int b = threadIdx.x; b < n; b += 256) my0 += (keys[b] == 0u);
+    block_exclusive_scan(my0, warp_sums, &tot0);
+    __syncthreads();
+    n_eff = n - tot0;
+  }
+  if (budget < 0 || budget > n_eff) budget = n_eff;
+  const bool take_all = (budget >= n_eff);
   uint32_t thr = 0;
   int need_ties = 0;
   if (!take_all && budget > 0) {
@@ -282,7 +303,7 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
     ties_before = block_exclusive_scan(my_ties, warp_sums, &dummy);
   }
   auto chosen = [&](int b, int& t) -> bool {
-    if (take_all) return true;
+    if (take_all) return !(MIXED && masked) || keys[b] != 0u;
     if (budget == 0) return false;
     const uint32_t k = keys[b];
     if (k == thr) return t++ < need_ties;
@@ -330,10 +351,10 @@ __device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uin
   int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
   // inter-chunk candidates against the head's budget, then intra-chunk ones against theirs
   const int n_inter = min(ncand, cg.ni);
-  int total = topk_range<MIXED>(keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh);
+  int total = topk_range<MIXED>(keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh, a.kv_pages != nullptr);
   if (MIXED && ncand > n_inter)
     total += topk_range<MIXED>(keys + n_inter, ncand - n_inter, a.intra_budgets ? a.intra_budgets[h] : -1, cg, cg.ni, out,
-                        total, a.kcap, sh);
+                        total, a.kcap, sh, false);
   if (threadIdx.x == 0) {
     a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
     if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
@@ -604,9 +625,19 @@ bool coop_info(int* nsm) {
 }
 }  // namespace
 
+cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st) {
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  dim3 g1(n_tiles, a.H);
+  if (a.D == 128)
+    qsum_partial_kernel<128><<<g1, 256, 0, st>>>(a);
+  else
+    qsum_partial_kernel<64><<<g1, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   int nsm = 0;
-  const bool mixed = a.inter_pages > 1 || a.intra_first_page1 > 0;
+  const bool mixed = a.inter_pages > 1 || a.intra_first_page1 > 0 || a.kv_pages != nullptr;
   if (a.barrier && coop_info(&nsm)) {
     // one cooperative launch for all three stages
     const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;

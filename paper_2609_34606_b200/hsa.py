@@ -37,7 +37,8 @@ TILE_M = 128
 
 EXPORTS = [
     "hsa_query_sizes", "hsa_create", "hsa_append_kv", "hsa_select_blocks", "hsa_select_blocks_ex",
-    "hsa_select_blocks_adaptive",
+    "hsa_select_blocks_adaptive", "hsa_retrieve_kv_pages", "hsa_evict_blocks", "hsa_restore_blocks",
+    "hsa_block_resident",
     "hsa_select_blocks_noalloc",
     "hsa_forward",
     "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
@@ -55,7 +56,8 @@ class hsa_config(C.Structure):
 
 class hsa_select_opts(C.Structure):
     _fields_ = [("inter_block_pages", C.c_int32), ("intra_first_page", C.c_int32),
-                ("intra_budgets_dev", C.c_void_p)]
+                ("intra_budgets_dev", C.c_void_p), ("kv_pages_dev", C.c_void_p), ("n_kv_pages", C.c_int32),
+                ("kv_page_blocks", C.c_int32)]
 
 
 class hsa_sizes(C.Structure):
@@ -82,6 +84,10 @@ def _load() -> C.CDLL:
     lib.hsa_select_blocks.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, vp, vp, vp]
     lib.hsa_select_blocks_ex.argtypes = [vp, vp, i32, i64, i64, i64, i32, vp, i32, C.POINTER(hsa_select_opts), vp, vp,
                                          vp]
+    lib.hsa_retrieve_kv_pages.argtypes = [vp, vp, i32, i64, i64, i32, i32, vp, vp, C.POINTER(i32), vp]
+    lib.hsa_evict_blocks.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.hsa_restore_blocks.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.hsa_block_resident.argtypes = [vp, i32, C.POINTER(i32)]
     lib.hsa_select_blocks_adaptive.argtypes = [vp, vp, i32, i64, i64, i64, i32, C.c_float, C.c_float, i32, vp, vp,
                                                vp, vp]
     lib.hsa_select_blocks_noalloc.argtypes = [vp, i32, i64, i64, i32, i32, vp, i32, i64, i64, i32, C.c_float,
@@ -172,12 +178,41 @@ def hsa_select_blocks(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budg
 
 def hsa_select_blocks_ex(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, budgets: torch.Tensor,
                          q_group_tokens: int, inter_block_pages: int, intra_first_page: int,
-                         intra_budgets: Optional[torch.Tensor], sel_idx: torch.Tensor, sel_cnt: torch.Tensor) -> None:
+                         intra_budgets: Optional[torch.Tensor], sel_idx: torch.Tensor, sel_cnt: torch.Tensor,
+                         kv_pages: Optional[torch.Tensor] = None, kv_page_blocks: int = 0) -> None:
     ts, hs = _thd(q, "q")
-    opts = hsa_select_opts(int(inter_block_pages), int(intra_first_page), _ptr(intra_budgets))
+    opts = hsa_select_opts(int(inter_block_pages), int(intra_first_page), _ptr(intra_budgets), _ptr(kv_pages),
+                           0 if kv_pages is None else int(kv_pages.numel()), int(kv_page_blocks))
     _check(_lib.hsa_select_blocks_ex(ctx, q.data_ptr(), q.shape[0], ts, hs, int(q_pos0), int(causal),
                                      budgets.data_ptr(), int(q_group_tokens), C.byref(opts), sel_idx.data_ptr(),
                                      sel_cnt.data_ptr(), _stream()), "hsa_select_blocks_ex")
+
+
+def hsa_retrieve_kv_pages(ctx: int, q: torch.Tensor, kv_page_blocks: int, top_kp: int, page_ids: torch.Tensor,
+                          scores: Optional[torch.Tensor] = None) -> int:
+    """Returns the number of ids written to page_ids (int32, device)."""
+    ts, hs = _thd(q, "q")
+    n = C.c_int32(0)
+    _check(_lib.hsa_retrieve_kv_pages(ctx, q.data_ptr(), q.shape[0], ts, hs, int(kv_page_blocks), int(top_kp),
+                                      page_ids.data_ptr(), _ptr(scores), C.byref(n), _stream()),
+           "hsa_retrieve_kv_pages")
+    return n.value
+
+
+def hsa_evict_blocks(ctx: int, first_block: int, n_blocks: int, host_k: torch.Tensor, host_v: torch.Tensor) -> None:
+    _check(_lib.hsa_evict_blocks(ctx, int(first_block), int(n_blocks), host_k.data_ptr(), host_v.data_ptr(),
+                                 _stream()), "hsa_evict_blocks")
+
+
+def hsa_restore_blocks(ctx: int, first_block: int, n_blocks: int, host_k: torch.Tensor, host_v: torch.Tensor) -> None:
+    _check(_lib.hsa_restore_blocks(ctx, int(first_block), int(n_blocks), host_k.data_ptr(), host_v.data_ptr(),
+                                   _stream()), "hsa_restore_blocks")
+
+
+def hsa_block_resident(ctx: int, block: int) -> bool:
+    r = C.c_int32(0)
+    _check(_lib.hsa_block_resident(ctx, int(block), C.byref(r)), "hsa_block_resident")
+    return bool(r.value)
 
 
 def hsa_select_blocks_adaptive(ctx: int, q: torch.Tensor, q_pos0: int, causal: bool, tau_min: float,
@@ -338,14 +373,38 @@ class HSAContext:
 
     def select_blocks_ex(self, q: torch.Tensor, budgets: torch.Tensor, inter_block_pages: int = 2,
                          intra_first_page: int = -1, intra_budgets: Optional[torch.Tensor] = None,
-                         q_pos0: Optional[int] = None, causal: bool = False, group_tokens: int = 0, sel=None):
+                         q_pos0: Optional[int] = None, causal: bool = False, group_tokens: int = 0, sel=None,
+                         kv_pages: Optional[torch.Tensor] = None, kv_page_blocks: int = 0):
         """Selection with coarse inter-chunk blocks (runs of inter_block_pages pages) and single-page
-        intra-chunk blocks from intra_first_page on (see hsa_select_blocks_ex)."""
+        intra-chunk blocks from intra_first_page on, optionally restricted to the retrieved KV pages
+        (see hsa_select_blocks_ex)."""
         q_pos0 = self.n_tokens if q_pos0 is None else q_pos0
         sel_idx, sel_cnt = sel if sel is not None else self.alloc_selection(q.shape[0], group_tokens)
         hsa_select_blocks_ex(self.ctx, q, q_pos0, causal, budgets, group_tokens, inter_block_pages,
-                             intra_first_page, intra_budgets, sel_idx, sel_cnt)
+                             intra_first_page, intra_budgets, sel_idx, sel_cnt, kv_pages, kv_page_blocks)
         return sel_idx, sel_cnt
+
+    def retrieve_kv_pages(self, q: torch.Tensor, kv_page_blocks: int, top_kp: int = 4, with_scores: bool = False):
+        """Stage-2 page retrieval: (int32 ids of the kept KV pages, ascending[, fp32 score of every page])."""
+        n_pages = (self.n_blocks + kv_page_blocks - 1) // kv_page_blocks
+        ids = torch.zeros(max(1, min(top_kp, n_pages)), dtype=torch.int32, device=self.device)
+        scores = torch.zeros(max(1, n_pages), dtype=torch.float32, device=self.device) if with_scores else None
+        n = hsa_retrieve_kv_pages(self.ctx, q, kv_page_blocks, top_kp, ids, scores)
+        return (ids[:n], scores[:n_pages]) if with_scores else ids[:n]
+
+    def evict_blocks(self, first_block: int, n_blocks: int):
+        """Moves the K / V tiles of the blocks to pinned host memory; returns the two host tensors."""
+        shape = (n_blocks, self.H, PAGE_TOKENS, self.d)
+        hk = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
+        hv = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
+        hsa_evict_blocks(self.ctx, first_block, n_blocks, hk, hv)
+        return hk, hv
+
+    def restore_blocks(self, first_block: int, host_k: torch.Tensor, host_v: torch.Tensor) -> None:
+        hsa_restore_blocks(self.ctx, first_block, host_k.shape[0], host_k, host_v)
+
+    def block_resident(self, block: int) -> bool:
+        return hsa_block_resident(self.ctx, block)
 
     def select_blocks_adaptive(self, q: torch.Tensor, tau_min: float, tau_max: float,
                                q_pos0: Optional[int] = None, causal: bool = False, group_tokens: int = 0):

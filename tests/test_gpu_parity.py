@@ -482,3 +482,70 @@ def test_inter_and_intra_chunk_granularity(name, causal, cuda_device):
         o_ref = O.sparse_branch(qn, Kn, Vn, got, q_pos0, causal, rows=rows)
         Hn.assert_close(out[rows], o_ref[rows], "O_sp")
     ctx.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["mid_d128", "mid_shuffle", "mid_d64"])
+def test_kv_page_retrieval_mask_and_tier_migration(name, cuda_device):
+    """Stage-2 page retrieval against the oracle, the retrieved pages as a candidate mask of the
+    selection, and eviction / restore of blocks to pinned host memory (bit-exact round trip)."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS[name]
+    ctx = Hn.build_context(w, cuda_device)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    Kn, Vn = Hn.f32(K), Hn.f32(V)
+    q = W.gen_query(w)
+    qn, qd = Hn.f32(q), q.to(cuda_device)
+    N = Kn.shape[0]
+    nblk = O.n_blocks(N)
+    kvb = max(2, nblk // 5)                                   # five or six KV pages, the last one short
+    ids, scores = ctx.retrieve_kv_pages(qd, kvb, top_kp=2, with_scores=True)
+    ref_ids, alpha = O.retrieve_kv_pages(qn, Kn, kvb, 2)
+    assert np.allclose(scores.cpu().numpy(), alpha, rtol=1e-5, atol=1e-6)
+    got_ids = ids.cpu().tolist()
+    if got_ids != ref_ids.tolist():                           # only pages that tie the weakest kept one may differ
+        kth = alpha[ref_ids].min()
+        assert all(abs(alpha[j] - kth) <= Hn.TIE_EPS for j in set(got_ids) ^ set(ref_ids.tolist()))
+    assert ctx.retrieve_kv_pages(qd, kvb, top_kp=64).cpu().tolist() == list(range((nblk + kvb - 1) // kvb))
+
+    # the retrieved pages restrict the selection (budgets larger than what they hold included)
+    budgets = torch.tensor([3 if h % 2 == 0 else 10 ** 6 for h in range(w.H)], dtype=torch.int32)
+    for inter_pages in (1, 2):
+        si, sc = ctx.select_blocks_ex(qd, budgets.to(cuda_device), inter_block_pages=inter_pages, kv_pages=ids,
+                                      kv_page_blocks=kvb)
+        got = Hn.selection_lists(si, sc)
+        ref, s = O.select_blocks_mixed(qn, Kn, N, False, budgets.tolist(), inter_pages, -1, None,
+                                       kv_pages=got_ids, kv_page_blocks=kvb)
+        for h in range(w.H):
+            a, b = got[h][0].tolist(), ref[h][0].tolist()
+            assert len(a) == len(b) and all(p // kvb in got_ids for p in a)
+            if a != b:
+                ca, cb = {p // inter_pages for p in a}, {p // inter_pages for p in b}
+                kth = min(s[h, 0, c] for c in cb)
+                assert all(abs(s[h, 0, c] - kth) <= Hn.TIE_EPS for c in ca ^ cb), h
+    assert ctx.device_status() == 0
+
+    # tier migration: evict the blocks outside the retrieved pages, poison their tiles, restore
+    out0 = ctx.forward(qd, si, sc).clone()
+    allsel = Hn.selection_to_device([[np.arange(nblk, dtype=np.int32)] for _ in range(w.H)], ctx.max_topk, cuda_device)
+    full0 = ctx.forward(qd, allsel[0], allsel[1]).clone()
+    evict_page = min(j for j in range((nblk + kvb - 1) // kvb) if j not in got_ids)   # a page that was not kept
+    lo, hi = evict_page * kvb, min(nblk, evict_page * kvb + kvb)
+    if hi > lo:
+        hk, hv = ctx.evict_blocks(lo, hi - lo)
+        torch.cuda.synchronize()
+        assert not ctx.block_resident(lo) and not ctx.block_resident(hi - 1)
+        assert ctx.block_resident(got_ids[0] * kvb)
+        order = W.gen_page_order(w, w.n_blocks)
+        pages = list(range(lo, hi)) if order is None else [int(order[b]) for b in range(lo, hi)]
+        kp = ctx.k_pool.view(torch.bfloat16).view(-1, w.H, 64, w.d)
+        vp = ctx.v_pool.view(torch.bfloat16).view(-1, w.H, 64, w.d)
+        assert torch.equal(hk, kp[pages].cpu()) and torch.equal(hv, vp[pages].cpu())
+        kp[pages] = float("nan")
+        vp[pages] = float("nan")
+        # a selection restricted to the retrieved pages does not touch the evicted tiles
+        assert torch.equal(ctx.forward(qd, si, sc), out0)
+        ctx.restore_blocks(lo, hk, hv)
+        assert ctx.block_resident(lo)
+        assert torch.equal(ctx.forward(qd, allsel[0], allsel[1]), full0)
+    ctx.destroy()

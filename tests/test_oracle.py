@@ -427,3 +427,52 @@ def test_mixed_selection_causal_candidates_and_ragged_inter_region():
     # last query position 200: candidates are the blocks that start at or before it
     got, _ = O.select_blocks_mixed(q, K, 197, True, [-1], inter_pages=2, intra_first_page=5)
     assert got[0][0].tolist() == [0, 1, 2, 3]
+
+
+# ---------------------------------------------------------------- HKV Stage 2 retrieval as a candidate mask
+def test_kv_page_size_from_the_paper():
+    """8 frames of 1560 tokens per KV page (Sec. 3.2) = 195 blocks of 64; 4 pages = 49,920 tokens."""
+    rows = [l.split() for l in open(os.path.join(GOLD, "hkv_active_kv_tokens.txt")) if l[0] != "#"]
+    kp, frames, tpf, total = map(int, rows[0])
+    assert frames * tpf == 195 * O.BLOCK and kp * 195 == O.n_blocks(total)
+
+
+def test_kv_page_retrieval_brute_force_and_reduction():
+    N, H, d, Lq = 64 * 7 + 30, 2, 4, 6
+    q, K = rnd((Lq, H, d), 80), rnd((N, H, d), 81)
+    got, alpha = O.retrieve_kv_pages(q, K, kv_page_blocks=2, top_kp=2)
+    sc = []
+    for j in range(4):                                       # pages of 128 tokens, the last one short
+        toks = range(128 * j, min(N, 128 * j + 128))
+        tot = 0.0
+        for h in range(H):
+            qbar = [sum(float(q[i, h, c]) for i in range(Lq)) / Lq for c in range(d)]
+            kbar = [sum(float(K[t, h, c]) for t in toks) / len(toks) for c in range(d)]
+            tot += sum(a * b for a, b in zip(qbar, kbar))
+        sc.append(tot / H / math.sqrt(d))
+    assert np.allclose(alpha, sc, rtol=0, atol=1e-13)
+    assert got.tolist() == brute.topk_blocks(sc, [True] * 4, 2)
+    # one head, one block per page: the page score is the block score of the plain selection
+    q1, K1 = q[:, :1], K[:, :1]
+    a1 = O.kv_page_scores(q1, K1, 1)
+    assert np.allclose(a1, O.block_scores(q1, K1)[0, 0], rtol=0, atol=1e-14)
+    sel, _ = O.select_blocks(q1, K1, N, False, [3])
+    assert O.retrieve_kv_pages(q1, K1, 1, 3)[0].tolist() == sel[0][0].tolist()
+
+
+def test_retrieved_pages_mask_the_selection():
+    N = 64 * 12
+    q, K = rnd((5, 2, 4), 82), rnd((N, 2, 4), 83)
+    full, _ = O.select_blocks_mixed(q, K, N, False, [3, 3], inter_pages=1)
+    same, _ = O.select_blocks_mixed(q, K, N, False, [3, 3], inter_pages=1, kv_pages=[0, 1, 2, 3], kv_page_blocks=3)
+    assert all(same[h][0].tolist() == full[h][0].tolist() for h in range(2))      # every page retrieved: no mask
+    got, s = O.select_blocks_mixed(q, K, N, False, [3, 5], inter_pages=1, kv_pages=[1, 3], kv_page_blocks=3)
+    allowed = [3, 4, 5, 9, 10, 11]
+    for h in range(2):
+        assert set(got[h][0].tolist()) <= set(allowed)
+        best = sorted(allowed, key=lambda b: (-s[h, 0, b], b))[:[3, 5][h]]
+        assert got[h][0].tolist() == sorted(best)
+    # a budget beyond the retrieved pages takes all of them and nothing else; the chunk's own pages are never masked
+    got2, _ = O.select_blocks_mixed(q, K, N, False, [-1, 99], inter_pages=2, intra_first_page=10,
+                                    kv_pages=[0], kv_page_blocks=3)
+    assert all(got2[h][0].tolist() == [0, 1, 10, 11] for h in range(2))   # block (2, 3) straddles the page end
