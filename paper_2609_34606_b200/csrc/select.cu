@@ -224,6 +224,113 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   }
 }
 
+#ifdef HSA_TIMING
+__device__ long long g_sel_timing[64];
+#define SEL_T(slot)                                              \
+  do {                                                           \
+    if (blockIdx.x == 0 && threadIdx.x == 0) {                   \
+      long long t_;                                              \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));      \
+      g_sel_timing[(slot)] = t_;                                 \
+    }                                                            \
+  } while (0)
+#else
+#define SEL_T(slot) \
+  do {              \
+  } while (0)
+#endif
+
+// Many query groups (per-query-tile selection): one item is a chunk of candidates of one head for
+// ALL groups, so that the key sums are read once; the groups' mean queries are rebuilt eight at a
+// time in shared memory (qs: 8 x D doubles).
+template <int D, bool MIXED>
+__device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chunk, int h, double* qs) {
+  constexpr int GB = 8;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int gtok = a.group_tokens;  // > 0 here, a multiple of the tile height
+  constexpr int PER = D / 32;
+  const CandGeom cg = cand_geom<MIXED>(a);
+  constexpr int NB = kScoreBlocksPerCta / 8;  // candidates per warp
+  constexpr int NP = MIXED ? 2 : 1;
+  double kv[NB][PER];  // key sum of the candidate, widened once (conversions are slow instructions)
+  double inv_cnt[NB];
+  bool masked[NB];
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
+    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+    const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
+    const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      // (lane owns dims lane, lane + 32, ...: conflict-free reads of the mean queries below)
+      const float k0 = np > 0 ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp) * D + e * 32 + lane] : 0.f;
+      const float k1 = (NP > 1 && np > 1) ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp + 1) * D + e * 32 + lane] : 0.f;
+      kv[i][e] = static_cast<double>(k0) + static_cast<double>(k1);
+    }
+    inv_cnt[i] = 1.0 / static_cast<double>(max64(1, min64(static_cast<int64_t>(np) * kBlock,
+                                                          a.n_tokens - static_cast<int64_t>(fp) * kBlock)));
+    masked[i] = false;
+    if (MIXED && a.kv_pages != nullptr && c < cg.ni) {
+      const int pl = fp + np - 1;
+      bool in_f = false, in_l = false;
+      for (int k = 0; k < a.n_kv_pages; ++k) {
+        const int kp = a.kv_pages[k];
+        in_f |= (fp / a.kv_page_blocks == kp);
+        in_l |= (pl / a.kv_page_blocks == kp);
+      }
+      masked[i] = !(in_f && in_l);
+    }
+  }
+  SEL_T(8);
+  for (int g0 = 0; g0 < a.n_groups; g0 += GB) {
+    if (g0 == 0) SEL_T(9);
+    // mean queries of groups g0 .. g0 + 7 (tile sums added in ascending tile order, fp64)
+    constexpr int NV = GB * D / 256;  // values per thread
+    const int tiles_per_group = gtok / kTileM;
+    double sum[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) sum[v] = 0.0;
+    for (int tt = 0; tt < tiles_per_group; ++tt) {
+      float part[NV];  // independent loads first, then the adds
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int idx = threadIdx.x + 256 * v;
+        const int g = g0 + idx / D, col = idx % D;
+        const int t = g * tiles_per_group + tt;
+        part[v] = (g < a.n_groups && t * kTileM < a.n_q) ? __ldcg(&a.qpart[(static_cast<size_t>(t) * a.H + h) * D + col]) : 0.f;
+      }
+#pragma unroll
+      for (int v = 0; v < NV; ++v) sum[v] += static_cast<double>(part[v]);
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int idx = threadIdx.x + 256 * v;
+      const int g = g0 + idx / D;
+      const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
+      qs[idx] = g < a.n_groups ? sum[v] * (static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo)) : 0.0;
+    }
+    __syncthreads();
+    if (g0 == 0) SEL_T(10);
+    for (int gi = 0; gi < GB && g0 + gi < a.n_groups; ++gi) {
+      uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g0 + gi) * a.max_pages;
+#pragma unroll
+      for (int i = 0; i < NB; ++i) {
+        const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+        if (c >= cg.nc) continue;  // warp-uniform
+        double dot = 0.0;
+#pragma unroll
+        for (int e = 0; e < PER; ++e)
+          dot += qs[gi * D + e * 32 + lane] * kv[i][e];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (lane == 0) keys[c] = masked[i] ? 0u : order_key(static_cast<float>(dot * inv_cnt[i]));
+      }
+    }
+    __syncthreads();
+    if (g0 == 0) SEL_T(11);
+  }
+}
+
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   __shared__ double qs[D + 256];  // mean query, then the per-way partial sums
@@ -400,28 +507,39 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctr, unsigned target, int
   __syncthreads();
 }
 
+
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
   extern __shared__ uint32_t fused_keys[];
   __shared__ __align__(16) unsigned char scratch[256 / (D / 8) * D * 4];  // tile-sum partials / mean query
   __shared__ TopkShared sh;
+  SEL_T(0);
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
     qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
   }
+  SEL_T(1);
   grid_barrier(bar_ctr, bar_base + gridDim.x, a.status);
-  for (int it = blockIdx.x; it < n_chunks * a.n_groups * a.H; it += gridDim.x) {
-    const int chunk = it % n_chunks, gh = it / n_chunks;
-    scores_item<D, MIXED>(a, chunk, gh % a.n_groups, gh / a.n_groups, reinterpret_cast<double*>(scratch));
-    __syncthreads();
+  SEL_T(2);
+  if (a.n_groups > 1) {
+    for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x)
+      scores_item_groups<D, MIXED>(a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
+  } else {
+    for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x) {
+      scores_item<D, MIXED>(a, it % n_chunks, 0, it / n_chunks, reinterpret_cast<double*>(scratch));
+      __syncthreads();
+    }
   }
+  SEL_T(3);
   grid_barrier(bar_ctr, bar_base + 2 * gridDim.x, a.status);
+  SEL_T(4);
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
     topk_item<MIXED>(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
     __syncthreads();
-  }
+    SEL_T(5);
+}
 }
 
 // ---------------------------------------------------------------------------------------
@@ -624,6 +742,14 @@ bool coop_info(int* nsm) {
   return cached_coop != 0 && cached_sm > 0;
 }
 }  // namespace
+
+#ifdef HSA_TIMING
+}  // namespace hsa
+extern "C" int hsa_debug_read_sel_timing(long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, hsa::g_sel_timing, sizeof(long long) * n));
+}
+namespace hsa {
+#endif
 
 cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st) {
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
