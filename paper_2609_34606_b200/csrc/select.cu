@@ -240,36 +240,55 @@ __device__ long long g_sel_timing[64];
   } while (0)
 #endif
 
-// Many query groups (per-query-tile selection): one item is a chunk of candidates of one head for
-// ALL groups, so that the key sums are read once; the groups' mean queries are rebuilt eight at a
-// time in shared memory (qs: 8 x D doubles).
+// Many query groups (per-query-tile selection): the scores of one head are a small matrix product
+//   scores[g][c] = sum_e qbar[g][e] * ksum[c][e]
+// and plain fp64 arithmetic is a slow pipe on this GPU, so it runs on the fp64 tensor-core path
+// (mma.sync m8n8k4).  One item is a chunk of 32 candidates of one head for ALL groups, so that the
+// key sums are read once: warp w owns candidates 8 (w & 3) .. + 7 (their key sums sit in registers as
+// the B fragments of all k-steps) and rows 8 (w >> 2) .. + 7 of each batch of 16 groups, whose mean
+// queries are rebuilt in shared memory (qs: 16 rows of D + 4 doubles; the pad keeps the fragment
+// loads at the two wavefronts a 256-byte access needs anyway).
+constexpr int kGroupBatch = 16;
+
+__device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1)
+               : "d"(a), "d"(b));
+}
+
 template <int D, bool MIXED>
 __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chunk, int h, double* qs) {
-  constexpr int GB = 8;
+  constexpr int GB = kGroupBatch, PITCH = D + 4, KS = D / 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens;  // > 0 here, a multiple of the tile height
-  constexpr int PER = D / 32;
   const CandGeom cg = cand_geom<MIXED>(a);
-  constexpr int NB = kScoreBlocksPerCta / 8;  // candidates per warp
-  constexpr int NP = MIXED ? 2 : 1;
-  double kv[NB][PER];  // key sum of the candidate, widened once (conversions are slow instructions)
-  double inv_cnt[NB];
-  bool masked[NB];
-#pragma unroll
-  for (int i = 0; i < NB; ++i) {
-    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+  const int c0 = chunk * kScoreBlocksPerCta + 8 * (warp & 3);  // this warp's eight candidates
+  // B fragments: element (k = lane % 4, n = lane / 4) of every k-step = key sum of candidate
+  // c0 + lane / 4 at dims 4 kk + lane % 4 (a coarse candidate's two pages are added here)
+  float kb[KS];
+  {
+    const int c = c0 + (lane >> 2);
     const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
     const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
+    const float* k0 = a.ksum + (static_cast<size_t>(h) * a.max_pages + fp) * D + (lane & 3);
 #pragma unroll
-    for (int e = 0; e < PER; ++e) {
-      // (lane owns dims lane, lane + 32, ...: conflict-free reads of the mean queries below)
-      const float k0 = np > 0 ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp) * D + e * 32 + lane] : 0.f;
-      const float k1 = (NP > 1 && np > 1) ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp + 1) * D + e * 32 + lane] : 0.f;
-      kv[i][e] = static_cast<double>(k0) + static_cast<double>(k1);
+    for (int kk = 0; kk < KS; ++kk) {
+      float v = np > 0 ? k0[4 * kk] : 0.f;
+      if (MIXED && np > 1) v += k0[D + 4 * kk];
+      kb[kk] = v;
     }
-    inv_cnt[i] = 1.0 / static_cast<double>(max64(1, min64(static_cast<int64_t>(np) * kBlock,
+  }
+  // the two candidates of this lane's accumulator columns: token counts and mask
+  double inv_cnt[2];
+  bool masked[2];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int c = c0 + 2 * (lane & 3) + t;
+    const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
+    const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
+    inv_cnt[t] = 1.0 / static_cast<double>(max64(1, min64(static_cast<int64_t>(np) * kBlock,
                                                           a.n_tokens - static_cast<int64_t>(fp) * kBlock)));
-    masked[i] = false;
+    masked[t] = false;
     if (MIXED && a.kv_pages != nullptr && c < cg.ni) {
       const int pl = fp + np - 1;
       bool in_f = false, in_l = false;
@@ -278,15 +297,13 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
         in_f |= (fp / a.kv_page_blocks == kp);
         in_l |= (pl / a.kv_page_blocks == kp);
       }
-      masked[i] = !(in_f && in_l);
+      masked[t] = !(in_f && in_l);
     }
   }
-  SEL_T(8);
+  const int tiles_per_group = gtok / kTileM;
   for (int g0 = 0; g0 < a.n_groups; g0 += GB) {
-    if (g0 == 0) SEL_T(9);
-    // mean queries of groups g0 .. g0 + 7 (tile sums added in ascending tile order, fp64)
+    // mean queries of groups g0 .. g0 + 15 (tile sums added in ascending tile order, fp64)
     constexpr int NV = GB * D / 256;  // values per thread
-    const int tiles_per_group = gtok / kTileM;
     double sum[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) sum[v] = 0.0;
@@ -305,29 +322,28 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int idx = threadIdx.x + 256 * v;
-      const int g = g0 + idx / D;
+      const int gi = idx / D, g = g0 + gi;
       const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
-      qs[idx] = g < a.n_groups ? sum[v] * (static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo)) : 0.0;
+      qs[gi * PITCH + idx % D] = g < a.n_groups ? sum[v] * (static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo)) : 0.0;
     }
     __syncthreads();
-    if (g0 == 0) SEL_T(10);
-    for (int gi = 0; gi < GB && g0 + gi < a.n_groups; ++gi) {
-      uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g0 + gi) * a.max_pages;
+    const int row0 = 8 * (warp >> 2);  // this warp's eight rows of the batch
+    if (g0 + row0 < a.n_groups && c0 < cg.nc) {  // warp-uniform
+      // A fragment: element (m = lane / 4, k = lane % 4) of every k-step
+      const double* arow = qs + (row0 + (lane >> 2)) * PITCH + (lane & 3);
+      double d0 = 0.0, d1 = 0.0;
 #pragma unroll
-      for (int i = 0; i < NB; ++i) {
-        const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
-        if (c >= cg.nc) continue;  // warp-uniform
-        double dot = 0.0;
-#pragma unroll
-        for (int e = 0; e < PER; ++e)
-          dot += qs[gi * D + e * 32 + lane] * kv[i][e];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        if (lane == 0) keys[c] = masked[i] ? 0u : order_key(static_cast<float>(dot * inv_cnt[i]));
+      for (int kk = 0; kk < KS; ++kk) dmma_m8n8k4(d0, d1, arow[4 * kk], static_cast<double>(kb[kk]));
+      // accumulator: row lane / 4 (group), columns 2 (lane % 4) and + 1 (candidates)
+      const int g = g0 + row0 + (lane >> 2);
+      if (g < a.n_groups) {
+        uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
+        const int c = c0 + 2 * (lane & 3);
+        if (c < cg.nc) keys[c] = masked[0] ? 0u : order_key(static_cast<float>(d0 * inv_cnt[0]));
+        if (c + 1 < cg.nc) keys[c + 1] = masked[1] ? 0u : order_key(static_cast<float>(d1 * inv_cnt[1]));
       }
     }
     __syncthreads();
-    if (g0 == 0) SEL_T(11);
   }
 }
 
@@ -511,7 +527,10 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctr, unsigned target, int
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
   extern __shared__ uint32_t fused_keys[];
-  __shared__ __align__(16) unsigned char scratch[256 / (D / 8) * D * 4];  // tile-sum partials / mean query
+  // tile-sum partials / mean query / (many groups) a batch of mean queries
+  constexpr int kGroupBytes = kGroupBatch * (D + 4) * 8;
+  constexpr int kScratch = kGroupBytes > 256 / (D / 8) * D * 4 ? kGroupBytes : 256 / (D / 8) * D * 4;
+  __shared__ __align__(16) unsigned char scratch[kScratch];
   __shared__ TopkShared sh;
   SEL_T(0);
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
