@@ -332,8 +332,8 @@ def bench_ours(args, rank: int, world: int):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{w.name}: H={w.H} d={w.d} chunk={w.Lq} history={w.N} tokens "
                                    f"({w.n_blocks} blocks of 64) top-{w.topk} blocks/head",
-                       "step": "restore the 9-chunk running state (S, z) + hsa_append_kv + hsa_select_blocks + "
-                               "hsa_forward",
+                       "step": f"restore the {w.n_chunks - 1}-chunk running state (S, z) + hsa_append_kv + "
+                               "hsa_select_blocks + hsa_forward",
                        "launch": (f"CUDA graphs: the timed loop replays a graph of {2 * RING} consecutive steps "
                                   "(single-step graphs for the remainder)"
                                   if args.launch == "graph" else "eager: every call issued from the host"),

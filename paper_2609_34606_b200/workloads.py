@@ -117,7 +117,8 @@ def gen_kv_chunk(w: Workload, c: int, layer: int = 0):
     k = torch.randn(w.chunk, w.H, w.d, generator=_gen(_tensor_seed(w, 1, c, layer)))
     v = torch.randn(w.chunk, w.H, w.d, generator=_gen(_tensor_seed(w, 2, c, layer)))
     if w.mixture:
-        mu = segment_means(w)[c // w.seg_chunks]
+        means = segment_means(w)
+        mu = means[min(c // w.seg_chunks, means.shape[0] - 1)]  # chunks past the history: last segment
         k = mu[None] + w.sigma * k
     return k.to(torch.bfloat16), v.to(torch.bfloat16)
 
