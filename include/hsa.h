@@ -83,6 +83,9 @@ typedef struct {
   uint32_t flags;         /* HSA_CFG_* bits                                                    */
   int32_t lin_rank;       /* HSA_LIN_LINFORMER: projection rank r, a multiple of 128 (else 0)         */
   int32_t lin_seg_tokens; /* HSA_LIN_LINFORMER: segment length L; every append must be exactly L      */
+  int32_t split_blocks;   /* a (query tile, head) with more selected blocks than this is split over
+                             several CTAs whose partial results the last one to finish merges
+                             (0 -> 256; only matters when max_topk exceeds it)                     */
 } hsa_config;
 
 typedef struct {

@@ -64,6 +64,7 @@ struct Smem {
 
 struct Bars {
   uint64_t q_full;
+  int ticket;  // split tiles: arrival number of this CTA among the parts of its (tile, head)
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[kSBufs];
   uint64_t p_full[kSBufs];
@@ -186,7 +187,8 @@ __device__ __forceinline__ void init_barriers(Bars* bars) {
 
 }  // namespace
 
-template <int D>
+// SPLIT: compiled with the split-tile path (grid z > 1); the plain kernel carries none of it
+template <int D, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v,
@@ -208,6 +210,25 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int32_t* sel = p.sel_idx + (static_cast<size_t>(h) * p.n_groups + g) * p.kcap;
   int cnt = p.do_sparse ? p.sel_cnt[static_cast<size_t>(h) * p.n_groups + g] : 0;
   cnt = max(0, min(cnt, min(p.kcap, p.n_blocks)));  // never more blocks than the history holds
+  // A long list is split over the CTAs (tile, head, 0 .. nsplit - 1): each takes a run of whole
+  // two-page steps; CTAs beyond nsplit leave before they set anything up.
+  int nsplit = 1;
+  const int part = blockIdx.z;
+  if (SPLIT && gridDim.z > 1) {
+    const int steps_total = (cnt + 1) / 2;
+    const int split_steps = p.split_blocks / 2;
+    nsplit = min(static_cast<int>(gridDim.z), max(1, (steps_total + split_steps - 1) / split_steps));
+    const int steps_per = (steps_total + nsplit - 1) / nsplit;
+    if (steps_per > 0) nsplit = (steps_total + steps_per - 1) / steps_per;  // no empty part
+    if (part >= nsplit) return;
+    if (nsplit > 1) {
+      const int b_lo = 2 * part * steps_per;
+      const int b_hi = min(cnt, 2 * (part + 1) * steps_per);
+      sel += b_lo;
+      cnt = b_hi - b_lo;
+    }
+  }
+  const int slot = (tile * p.H + h) * static_cast<int>(gridDim.z) + part;  // this CTA's partial-result slot
   const int nsteps = (cnt + 1) / 2;
 
   if (threadIdx.x == 0) {
@@ -686,8 +707,67 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         lsum += stats[(gg * 128 + r) * 4 + 0];
         den += stats[(gg * 128 + r) * 4 + 1];
       }
-      const float inv_l = (nsteps > 0 && lsum > 0.f) ? 1.f / lsum : 0.f;
+      float inv_l = (nsteps > 0 && lsum > 0.f) ? 1.f / lsum : 0.f;
       const bool has_o = nsteps > 0;
+      // Split tile: every part dumps its unnormalised accumulator with the row sums and the
+      // exponent references, then takes a ticket; the part that draws the last ticket merges all of
+      // them (its own included) in the epilogue below, the others write no output.  Only the attempt
+      // that stands (no redo pending) takes part.
+      const bool final_attempt = safe || bars->redo == 0;
+      bool do_output = final_attempt;
+      float pf[SPLIT ? kFwdSplitMax : 1];  // merge factors 2^(ref_p - max ref) of the parts (split tiles only)
+      if (SPLIT && nsplit > 1 && final_attempt) {
+        if (ok) {
+          float* po = p.part_o + (static_cast<size_t>(slot) * kTileM + r) * D + cbase;
+#pragma unroll 1
+          for (int c0 = 0; c0 < HC; c0 += 16) {
+            uint32_t oa[16];
+            tmem_ld16(o_tmem + cbase + c0, oa);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+              *reinterpret_cast<float4*>(po + c0 + i) =
+                  make_float4(__uint_as_float(oa[i]), __uint_as_float(oa[i + 1]), __uint_as_float(oa[i + 2]),
+                              __uint_as_float(oa[i + 3]));
+          }
+          if (grp == 0) {
+            p.part_l[static_cast<size_t>(slot) * kTileM + r] = lsum;
+            p.part_ref[static_cast<size_t>(slot) * kTileM + r] = t_ref;
+          }
+          __threadfence();
+        }
+        named_bar_sync(3, 128 * kGroups);
+        if (warp == 4 && lane == 0) {
+          int32_t* tk = p.part_ticket + tile * p.H + h;
+          const int t = ok ? atomicAdd(tk, 1) : -1;
+          if (t == nsplit - 1) *tk = 0;  // the counter is back at zero for the next launch
+          bars->ticket = t;
+        }
+        named_bar_sync(3, 128 * kGroups);
+        do_output = bars->ticket == nsplit - 1;
+        if (do_output) {
+          __threadfence();
+          // common reference R = largest reference among the parts that saw a key for this row
+          const size_t s0 = static_cast<size_t>(slot - part) * kTileM + r;
+          float rmax = -INFINITY;
+          for (int q = 0; q < nsplit; ++q)
+            if (__ldcg(&p.part_l[s0 + static_cast<size_t>(q) * kTileM]) > 0.f)
+              rmax = fmaxf(rmax, __ldcg(&p.part_ref[s0 + static_cast<size_t>(q) * kTileM]));
+          float ltot = 0.f;
+#pragma unroll
+          for (int q = 0; q < (SPLIT ? kFwdSplitMax : 1); ++q) {
+            pf[q] = 0.f;
+            if (q < nsplit) {
+              const float lq = __ldcg(&p.part_l[s0 + static_cast<size_t>(q) * kTileM]);
+              if (lq > 0.f) {
+                pf[q] = ex2(__ldcg(&p.part_ref[s0 + static_cast<size_t>(q) * kTileM]) - rmax);
+                ltot = fmaf(lq, pf[q], ltot);
+              }
+            }
+          }
+          inv_l = ltot > 0.f ? 1.f / ltot : 0.f;
+        }
+      }
       if (ok && p.do_linear && epi) {
         ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
         tc_fence_after();
@@ -697,7 +777,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // branch has not looked at Q at all: its TMA load may still be in flight and must land first.
       if (ok && epi && nsteps == 0 && !p.do_linear)
         ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
-      if (ok && epi) {  // warp-uniform: the TMEM loads below are warp-collective
+      if (ok && epi && do_output) {  // warp-uniform: the TMEM loads below are warp-collective
         const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
         float lin_den = den;
         const float* lnum = nullptr;
@@ -719,7 +799,30 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
           uint32_t oa[16], ln[16];
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 0);
-          if (has_o) tmem_ld16(o_tmem + c0, oa);
+          if (SPLIT && nsplit > 1) {
+            // merged accumulator: sum over the parts of factor * partial, from the dumps
+            float acc[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+            const float* po = p.part_o + (static_cast<size_t>(slot - part) * kTileM + r) * D + c0;
+#pragma unroll
+            for (int q = 0; q < (SPLIT ? kFwdSplitMax : 1); ++q) {
+              if (q < nsplit && pf[q] != 0.f) {
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                  const float4 v = __ldcg(reinterpret_cast<const float4*>(po + static_cast<size_t>(q) * kTileM * D + i));
+                  acc[i] = fmaf(pf[q], v.x, acc[i]);
+                  acc[i + 1] = fmaf(pf[q], v.y, acc[i + 1]);
+                  acc[i + 2] = fmaf(pf[q], v.z, acc[i + 2]);
+                  acc[i + 3] = fmaf(pf[q], v.w, acc[i + 3]);
+                }
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) oa[i] = __float_as_uint(acc[i]);
+          } else if (has_o) {
+            tmem_ld16(o_tmem + c0, oa);
+          }
           if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
           tc_wait_ld();
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 1);
@@ -794,7 +897,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // (rows past the end of the chunk are clipped by the tensor map)
       fence_proxy_async_smem();
       named_bar_sync(2, 128 * kGroups);
-      if (ok && warp == 4) {
+      if (ok && do_output && warp == 4) {
         if (elect_one_sync()) {
           for (int dh = 0; dh < DH; ++dh) tma_store_3d(&tm_out, smem + L::kQ + dh * L::kHalf, dh * 64, h, row0);
           tma_store_commit();
@@ -821,22 +924,37 @@ extern "C" int hsa_debug_read_timing(long long* host_out, int n) {
 #endif
 
 cudaError_t forward_init() {
-  cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128>,
+  cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kTotal);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(hsa_forward_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Smem<64>::kTotal);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(hsa_forward_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Smem<128>::kTotal);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(hsa_forward_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Smem<64>::kTotal);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(hsa_forward_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Smem<64>::kTotal);
+  return e;
 }
 
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                            const CUtensorMap& tm_v, const CUtensorMap& tm_state, const CUtensorMap& tm_out,
                            cudaStream_t st) {
   const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
-  dim3 grid(n_tiles, p.H);
-  if (D == 128)
-    hsa_forward_kernel<128><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
-  else
-    hsa_forward_kernel<64><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+  dim3 grid(n_tiles, p.H, p.max_splits > 1 ? p.max_splits : 1);
+  const bool split = p.max_splits > 1;
+  if (D == 128) {
+    if (split)
+      hsa_forward_kernel<128, true><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+    else
+      hsa_forward_kernel<128, false><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+  } else {
+    if (split)
+      hsa_forward_kernel<64, true><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+    else
+      hsa_forward_kernel<64, false><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+  }
   return cudaGetLastError();
 }
 

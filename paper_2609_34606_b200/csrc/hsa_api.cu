@@ -38,7 +38,9 @@ struct Layout {
   // state
   size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
   // workspace
-  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ad_w, ad_idx, ad_gini, ad_wsum, ws_total;
+  size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ad_w, ad_idx, ad_gini, ad_wsum,
+      part_o, part_l, part_ref, part_ticket, ws_total;
+  int fwd_splits, split_blocks;
   // Linformer
   size_t n_cpages, cpool;
 };
@@ -59,6 +61,7 @@ bool config_ok(const hsa_config* c) {
   }
   if (c->gate_act != 0 && c->gate_act != 1) return false;
   if (!(c->softmax_scale >= 0.f)) return false;
+  if (c->split_blocks < 0) return false;
   if ((c->flags & HSA_CFG_ADAPTIVE) && c->max_pages > 8192) return false;
   return true;
 }
@@ -99,6 +102,18 @@ Layout make_layout(const hsa_config* c) {
     L.csel = o;   o = align_up(o + H * L.n_cpages * 4, 256);
     L.ccnt = o;   o = align_up(o + H * 4, 256);
     L.olin = o;   o = align_up(o + static_cast<size_t>(c->max_q_tokens) * H * D * 2, 256);
+  }
+  // split tiles of the forward kernel
+  L.split_blocks = c->split_blocks > 0 ? c->split_blocks : 256;
+  L.split_blocks += L.split_blocks & 1;  // whole two-page steps
+  L.fwd_splits = (c->max_topk + L.split_blocks - 1) / L.split_blocks;
+  if (L.fwd_splits > kFwdSplitMax) L.fwd_splits = kFwdSplitMax;
+  if (L.fwd_splits > 1) {
+    const size_t slots = tiles * H * static_cast<size_t>(L.fwd_splits);
+    L.part_o = o;      o = align_up(o + slots * kTileM * D * 4, 256);
+    L.part_l = o;      o = align_up(o + slots * kTileM * 4, 256);
+    L.part_ref = o;    o = align_up(o + slots * kTileM * 4, 256);
+    L.part_ticket = o; o = align_up(o + tiles * H * 4, 256);
   }
   L.ws_total = o;
   return L;
@@ -238,6 +253,9 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   uint8_t* ws = static_cast<uint8_t*>(bufs->workspace);
   e = cudaMemcpy(ws + ctx->lay.page_table, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(ws + ctx->lay.status, 0, 16);
+  if (e == cudaSuccess && ctx->lay.fwd_splits > 1)
+    e = cudaMemset(ws + ctx->lay.part_ticket, 0,
+                   static_cast<size_t>((cfg->max_q_tokens + kTileM - 1) / kTileM) * cfg->num_heads * 4);
   if (e == cudaSuccess) e = cudaMemset(bufs->state, 0, ctx->lay.state_total);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = forward_init();
@@ -530,6 +548,15 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   p.do_linear = do_linear;
   p.do_sparse = do_sparse;
   p.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
+  p.max_splits = 1;
+  if (do_sparse && ctx->lay.fwd_splits > 1) {
+    p.max_splits = ctx->lay.fwd_splits;
+    p.split_blocks = ctx->lay.split_blocks;
+    p.part_o = reinterpret_cast<float*>(ws + ctx->lay.part_o);
+    p.part_l = reinterpret_cast<float*>(ws + ctx->lay.part_l);
+    p.part_ref = reinterpret_cast<float*>(ws + ctx->lay.part_ref);
+    p.part_ticket = reinterpret_cast<int32_t*>(ws + ctx->lay.part_ticket);
+  }
   if (causal_lin) {
     CausalLinArgs c{};
     c.q = static_cast<const __nv_bfloat16*>(q);
@@ -577,6 +604,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     p1.scale_log2 = p.scale_log2;
     p1.do_linear = 0;
     p1.do_sparse = 1;
+    p1.max_splits = 1;
     p1.status = p.status;
     cudaError_t e1 = launch_forward(p1, D, tm_q, ctx->tm_kc, ctx->tm_vc, ctx->tm_state, tm_olin, st);
     if (e1 != cudaSuccess) return cuda_fail(ctx, e1);

@@ -11,6 +11,7 @@ namespace hsa {
 constexpr int kBlock = HSA_PAGE_TOKENS;  // tokens per KV block = tokens per page
 constexpr int kTileM = 128;              // query rows per work item of the forward kernel
 constexpr int kStateSplitMax = 16;       // token-axis splits of the state update (per head)
+constexpr int kFwdSplitMax = 16;         // CTAs a long (query tile, head) of the forward kernel is split over
 
 __host__ __device__ inline int64_t min64(int64_t a, int64_t b) { return a < b ? a : b; }
 __host__ __device__ inline int64_t max64(int64_t a, int64_t b) { return a > b ? a : b; }
@@ -115,6 +116,14 @@ struct FwdParams {
   const float* lin_num;  // causal intra-chunk partials [n_q][H][D] (or null)
   const float* lin_den;  // [n_q][H]
   const __nv_bfloat16* ext_lin;  // linear-branch output computed elsewhere, [n_q][H][D] (or null)
+  // split tiles: a (tile, head) with more than split_blocks selected blocks runs as several CTAs
+  // (grid z = max_splits); each dumps its unnormalised O, row sums and exponent references, the last
+  // one to take a ticket merges them and writes the output
+  int max_splits, split_blocks;
+  float* part_o;         // [tiles][H][max_splits][128][D]
+  float* part_l;         // [tiles][H][max_splits][128]
+  float* part_ref;       // [tiles][H][max_splits][128]
+  int32_t* part_ticket;  // [tiles][H], zero between launches
   int32_t* status;
 };
 

@@ -51,7 +51,8 @@ class hsa_config(C.Structure):
     _fields_ = [("num_heads", C.c_int32), ("head_dim", C.c_int32), ("page_tokens", C.c_int32),
                 ("max_pages", C.c_int32), ("max_q_tokens", C.c_int32), ("max_topk", C.c_int32),
                 ("lin_mode", C.c_int32), ("gate_act", C.c_int32), ("softmax_scale", C.c_float),
-                ("flags", C.c_uint32), ("lin_rank", C.c_int32), ("lin_seg_tokens", C.c_int32)]
+                ("flags", C.c_uint32), ("lin_rank", C.c_int32), ("lin_seg_tokens", C.c_int32),
+                ("split_blocks", C.c_int32)]
 
 
 class hsa_select_opts(C.Structure):
@@ -305,13 +306,13 @@ class HSAContext:
                  lin_mode: int = HSA_LIN_STATE, gate_act: int = 0, softmax_scale: float = 0.0,
                  causal: bool = False, page_order: Optional[torch.Tensor] = None,
                  device: str | torch.device = "cuda:0", adaptive: bool = False, lin_rank: int = 0, lin_seg_tokens: int = 0,
-                 e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None):
+                 e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None, split_blocks: int = 0):
         self.device = torch.device(device)
         self.H, self.d = H, d
         self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
         self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
                               softmax_scale, (HSA_CFG_CAUSAL if causal else 0) | (HSA_CFG_ADAPTIVE if adaptive else 0),
-                              lin_rank, lin_seg_tokens)
+                              lin_rank, lin_seg_tokens, split_blocks)
         self.sizes = hsa_query_sizes(self.cfg)
         with torch.cuda.device(self.device):
             mk = lambda n: torch.empty(max(n, 16), dtype=torch.uint8, device=self.device)

@@ -549,3 +549,41 @@ def test_kv_page_retrieval_mask_and_tier_migration(name, cuda_device):
         assert ctx.block_resident(lo)
         assert torch.equal(ctx.forward(qd, allsel[0], allsel[1]), full0)
     ctx.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,causal", [("mid_d128", False), ("mid_mix", False), ("mid_causal", True), ("mid_d64", False)])
+def test_long_lists_split_over_ctas_and_merged(name, causal, cuda_device):
+    """A (query tile, head) whose list is longer than split_blocks runs as several CTAs; the last
+    one to finish merges their partial accumulators.  With a small split_blocks every tile of these
+    workloads is split (lists of unequal lengths per head, odd block counts, a partial last block),
+    and the result must match the oracle and the unsplit kernel."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS[name]
+    q = W.gen_query(w)
+    qn, qd = Hn.f32(q), q.to(cuda_device)
+    outs = {}
+    for sb in (0, 6):
+        ctx = Hn.build_context(w, cuda_device, causal=causal, split_blocks=sb)
+        K, V = Hn.append_history(ctx, w, cuda_device)
+        nblk = ctx.n_blocks
+        # head h keeps every block but the first h (so the heads differ in length and in parity)
+        sel = [[np.arange(min(h, nblk - 1), nblk, dtype=np.int32)] for h in range(w.H)]
+        si, sc = Hn.selection_to_device(sel, ctx.max_topk, cuda_device)
+        for flags in (0, hsa.HSA_FWD_NO_LINEAR):
+            for rep in range(3):                       # tickets must be back at zero after each launch
+                out = ctx.forward(qd, si, sc, q_pos0=w.q_pos0, causal=causal, flags=flags)
+                assert ctx.device_status() == 0
+                if rep == 0:
+                    outs[(sb, flags)] = out.clone()
+                else:
+                    assert torch.equal(out, outs[(sb, flags)])
+        if sb:
+            Kn, Vn = Hn.f32(K), Hn.f32(V)
+            ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, causal, sel, linear_form="state")
+            Hn.assert_close(Hn.f64(outs[(sb, hsa.HSA_FWD_NO_LINEAR)]), ref["O_sp"], "O_sp")
+            Hn.assert_close(Hn.f64(outs[(sb, 0)]), ref["out"], "out")
+        ctx.destroy()
+    for flags in (0, hsa.HSA_FWD_NO_LINEAR):
+        d = (outs[(6, flags)].float() - outs[(0, flags)].float()).abs().max()
+        assert float(d) <= 2e-2
