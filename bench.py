@@ -373,6 +373,88 @@ def bench_ours(args, rank: int, world: int):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- rollout (cfg5)
+def bench_rollout(args, rank: int, world: int):
+    """Full-stack rollout: `layers` contexts, n_chunks chunks; per chunk and layer append the chunk,
+    select, forward (the history grows, so the calls are issued one by one: no graph fits).  Inputs
+    rotate over a ring of 8 (q, k, v) triples per layer generated on the device (seeded N(0,1))."""
+    from paper_2609_34606_b200 import hsa
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = W.WORKLOADS[args.workload]
+    layers = args.layers or w.layers
+    RR = 8
+    ctxs = [hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=w.Lq, max_topk=w.topk, device=dev)
+            for _ in range(layers)]
+    g = torch.Generator(device=dev)
+    ring = []
+    for layer in range(layers):
+        g.manual_seed(4_000_000 + 1000 * layer + rank)
+        ring.append([[torch.randn(w.Lq, w.H, w.d, device=dev, generator=g).to(torch.bfloat16) for _ in range(3)]
+                     for _ in range(RR)])
+    outs = [torch.empty(w.Lq, w.H, w.d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    budgets = W.gen_budgets(w).to(dev)
+    sels = [c.alloc_selection(w.Lq) for c in ctxs]
+
+    def rollout(n_chunks, evs=None):
+        for c in range(n_chunks):
+            if evs is not None:
+                evs[c].record()
+            for layer, ctx in enumerate(ctxs):
+                q, k, v = ring[layer][c % RR]
+                ctx.append_kv(k, v)
+                ctx.select_blocks(q, budgets, sel=sels[layer])
+                ctx.forward(q, sels[layer][0], sels[layer][1], out=outs[layer & 1])
+        if evs is not None:
+            evs[n_chunks].record()
+
+    def reset():
+        for ctx in ctxs:
+            ctx.rewind(0)
+            ctx.state.zero_()
+
+    rollout(3)                    # warm-up
+    torch.cuda.synchronize()
+    assert all(c.device_status() == 0 for c in ctxs)
+    sampler = ClockSampler(dev)
+    runs = []
+    for rep_i in range(2):        # the second rollout shows the run-to-run spread
+        reset()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(w.n_chunks + 1)]
+        torch.cuda.synchronize()
+        t0 = time.time()
+        rollout(w.n_chunks, evs)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        per_chunk = [evs[c].elapsed_time(evs[c + 1]) for c in range(w.n_chunks)]
+        runs.append({"ms_total": evs[0].elapsed_time(evs[-1]), "wall": (t0, t1), "per_chunk": per_chunk})
+    time.sleep(0.2)
+    clocks = sampler.summary(runs[0]["wall"][0], runs[1]["wall"][1])
+    sampler.stop()
+    status = max(c.device_status() for c in ctxs)
+    # work model: 64 full blocks per head from the first chunk on (a chunk alone is 73 blocks)
+    fl = step_flops(w, [w.topk * 64] * w.H)
+    steps = w.n_chunks * layers
+    best = min(runs, key=lambda r: r["ms_total"])
+    ms_step = best["ms_total"] / steps
+    pc = best["per_chunk"]
+    print(json.dumps({
+        "metric": METRIC, "value": fl["total"] / (ms_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1,
+        "steps": steps, "warmup": 3 * layers, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: rollout of {w.n_chunks} chunks x {layers} layers, H={w.H} d={w.d} "
+                               f"chunk={w.Lq}, top-{w.topk} blocks/head, history grows to {w.n_chunks * w.chunk} tokens",
+                   "step": "hsa_append_kv + hsa_select_blocks + hsa_forward of one layer for one chunk",
+                   "launch": "eager: every call issued from the host (the history grows every step)",
+                   "l2": f"{layers} layers x {RR} rotating (q,k,v) triples, pools {layers * 2 * w.n_blocks * w.H * 64 * w.d * 2 / 1e9:.0f} GB"},
+        "rollout_ms": [r["ms_total"] for r in runs],
+        "ms_per_chunk_all_layers": {"first": pc[0], "median": sorted(pc)[len(pc) // 2], "last": pc[-1]},
+        "flops_per_step": fl["total"], "clocks": clocks, "gpu_launches": 4 * steps, "device_status": status}),
+        flush=True)
+    for c in ctxs:
+        c.destroy()
+
+
 # ----------------------------------------------------------------------------- oracle (CPU)
 def oracle_step(w: W.Workload, data, rows):
     """One bounded oracle step: block selection over the full history, then both branches and the
@@ -450,6 +532,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--cpu-rows", type=int, default=4680)
+    ap.add_argument("--layers", type=int, default=0, help="rollout workloads: number of layers (0 = the workload's)")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="how the timed steps are issued: replayed CUDA graphs (default) or call by call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -461,6 +544,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         bench_reference(args, rank, world)
+    elif W.WORKLOADS[args.workload].layers > 1:
+        if rank == 0:
+            bench_rollout(args, rank, world)
     else:
         bench_ours(args, rank, world)
 
