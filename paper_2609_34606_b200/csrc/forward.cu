@@ -794,10 +794,40 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             (wr && p.ext_lin) ? p.ext_lin + (static_cast<size_t>(row) * p.H + h) * D : nullptr;
         const int g_ds = static_cast<int>(p.g_ds);
         const bool sig = p.gate_act == 1;
+        // (decided from the launch parameters, not from this thread's pointers: the branch holds
+        // warp-collective TMEM loads and must not diverge inside a warp)
+        const bool plain = !p.g_lin && !p.g_sp && !(p.do_linear && p.lin_num != nullptr) && !p.ext_lin &&
+                           !(SPLIT && nsplit > 1);
+        if (plain) {
+          // no gates, no causal partials, no external linear output, no merge: 32 columns per trip
+          const float il = has_o ? inv_l : 0.f, id = p.do_linear ? inv_den : 0.f;
+#pragma unroll 1
+          for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
+            uint32_t oa[32], ln[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) oa[i] = ln[i] = 0u;
+            if (has_o) tmem_ld32(o_tmem + c0, oa);
+            if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
+            tc_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+              pk[i >> 1] = pack_bf16(fmaf(__uint_as_float(oa[i]), il, __uint_as_float(ln[i]) * id),
+                                     fmaf(__uint_as_float(oa[i + 1]), il, __uint_as_float(ln[i + 1]) * id));
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const int cc = (c0 >> 3) + q4;  // 16-byte chunk of the row
+              *reinterpret_cast<uint4*>(smem + L::kQ + (cc >> 3) * L::kHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) =
+                  make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
+            }
+          }
+        }
         // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
 #pragma unroll 1
-        for (int c0 = cbase; c0 < cbase + HC; c0 += 16) {
+        for (int c0 = cbase; c0 < (plain ? cbase : cbase + HC); c0 += 16) {
           uint32_t oa[16], ln[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) oa[i] = ln[i] = 0u;
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 0);
           if (SPLIT && nsplit > 1) {
             // merged accumulator: sum over the parts of factor * partial, from the dumps
@@ -826,6 +856,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
           tc_wait_ld();
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 1);
+          uint32_t packed[8];
+          {
           // gate weights and causal partials are fetched under ONE branch each per trip (a branch
           // per element costs far more than the arithmetic it guards)
           float wl[16], ws[16], ladd[16];
@@ -867,7 +899,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               ladd[8 + 2 * i + 1] = f1.y;
             }
           }
-          uint32_t packed[8];
 #pragma unroll
           for (int i = 0; i < 16; i += 2) {
             float res[2];
@@ -879,6 +910,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               res[e] = fmaf(wl[i + e], olin, ws[i + e] * osp);
             }
             packed[i >> 1] = pack_bf16(res[0], res[1]);
+          }
           }
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 2);
           // stage the row into the Q tile's shared memory (dead by now; each thread touches only
