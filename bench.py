@@ -33,9 +33,9 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_34606_b200 import workloads as W  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one hsa_forward_kernel<128> launch on cfg2, from the
-# ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.44 MB + 0.58 MB)
-NCU_TRAFFIC_BYTES = {"cfg2": 41.02e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one hsa_forward_kernel<128, false> launch on cfg2, from
+# the ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.42 MB + 0.69 MB)
+NCU_TRAFFIC_BYTES = {"cfg2": 41.11e6}
 METRIC = "hsa_effective_tflops"
 UNIT = "TFLOP/s"
 RING = 4  # distinct (q, k, v, out) input sets rotated between steps (> L2 in total)
@@ -353,7 +353,7 @@ def bench_ours(args, rank: int, world: int):
                     "h2d_bytes_per_step": 3 * w.Lq * w.H * w.d * 2, "d2h_bytes_per_step": w.Lq * w.H * w.d * 2},
             "gpu_launches": 4 * K,  # append_fused, state_reduce, select_fused, hsa_forward per step
             "device_status": status,
-            "roofline": {"kernel": "hsa_forward_kernel<128>", "bound": "tensor", "achieved": fwd_tf,
+            "roofline": {"kernel": "hsa_forward_kernel<128, false>", "bound": "tensor", "achieved": fwd_tf,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tf / peaks["bf16_tflops"],
                          "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": by["forward"],
                          "peak_source": peaks["source"] + " (burst)",
