@@ -84,6 +84,9 @@ static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory sl
 #ifndef HSA_INTERLEAVE
 #define HSA_INTERLEAVE 8
 #endif
+#ifndef HSA_CONTINUOUS
+#define HSA_CONTINUOUS 8
+#endif
 #ifdef HSA_TIMING
 __device__ long long g_hsa_timing[4096];
 #define HSA_T(slot)                                                      \
@@ -611,6 +614,34 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           ++tok_i;
         }
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 3);
+#if HSA_CONTINUOUS
+        if (nchunks == 4 && !need_mask) {
+          // full, unmasked step (the usual case): ONE software pipeline over the 128 columns --
+          // scale-and-shift of column i, exponential of column i - LAG, row sum and bf16 pack of
+          // column i - 2 LAG -- that does not drain at the chunk boundaries; the TMEM load of the next
+          // chunk is issued when the pipeline enters a chunk, the P store when it leaves one
+          constexpr int LAG = HSA_CONTINUOUS;
+          float y[128];
+          uint32_t pk[2][16];
+#pragma unroll
+          for (int i = 0; i < 128 + 2 * LAG; ++i) {
+            if (i < 128) {
+              if ((i & 31) == 0) {
+                tc_wait_ld();
+                if (i + 32 < 128) tmem_ld32(s_tmem + i + 32, cbuf[((i >> 5) + 1) & 1]);
+              }
+              y[i] = fmaf(__uint_as_float(cbuf[(i >> 5) & 1][i & 31]), sl2, nt);
+            }
+            if (i >= LAG && i - LAG < 128) y[i - LAG] = ex2v(y[i - LAG]);
+            if (i >= 2 * LAG && i - 2 * LAG < 128) {
+              const int k = i - 2 * LAG;
+              acc[k & 3] += y[k];
+              if (k & 1) pk[(k >> 5) & 1][(k & 31) >> 1] = pack_bf16(y[k - 1], y[k]);
+              if ((k & 31) == 31) tmem_st16(s_tmem + 16 * (k >> 5), pk[(k >> 5) & 1]);
+            }
+          }
+        } else
+#endif
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           if (c < nchunks) {
