@@ -523,6 +523,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (!ok) break;
         tc_fence_after();
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 1);
+        uint32_t cbuf[2][32];  // two 32-column chunks of the score row in flight
+        // the first chunk is requested at once: its latency runs under the bookkeeping below
+        // (the steps that look for the row maximum first issue their own loads)
+        const bool early_ld = !(safe || j == 0);
+        if (early_ld) tmem_ld32(s_tmem, cbuf[0]);
         const int npg = min(2, cnt - 2 * j);
         const int n = npg * kBlock;
         if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
@@ -535,7 +540,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
           lim1 = npg > 1 ? static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk1) * kBlock))) : 0;
         }
-        uint32_t cbuf[2][32];  // two 32-column chunks of the score row in flight
         const int nchunks = n / 32;
         if (safe || j == 0) {
           // the reference needs the row maximum first: a pass over the score row in chunks
@@ -607,7 +611,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // the previous P chunk run under the arithmetic of the current one
         const float nt = -t_ref;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
-        tmem_ld32(s_tmem, cbuf[0]);
+        if (!early_ld) tmem_ld32(s_tmem, cbuf[0]);
         if (kTokens && !safe) {
           ok = __all_sync(0xffffffffu, wait_bar(&bars->tok[grp], tok_i & 1, bars, p.status));
           if (!ok) break;
