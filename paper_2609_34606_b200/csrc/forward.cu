@@ -88,10 +88,15 @@ static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory sl
 #define HSA_CONTINUOUS 8
 #endif
 #ifdef HSA_TIMING
+#ifndef HSA_T_BX
+#define HSA_T_BX 0
+#define HSA_T_BY 0
+#endif
 __device__ long long g_hsa_timing[4096];
+__device__ long long g_cta_t[8192];
 #define HSA_T(slot)                                                      \
   do {                                                                   \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && (slot) < 4096) \
+    if (blockIdx.x == HSA_T_BX && blockIdx.y == HSA_T_BY && lane == 0 && (slot) < 4096) \
       g_hsa_timing[(slot)] = clock64();                                  \
   } while (0)
 #else
@@ -134,6 +139,10 @@ __device__ __forceinline__ float ex2v(float x) {
   float y;
   asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// phi(x) = elu(x) + 1 = max(x, 0) + exp(min(x, 0))
+__device__ __forceinline__ float phi_elu1(float x) {
+  return fmaxf(x, 0.f) + ex2(fminf(x, 0.f) * 1.4426950408889634f);
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float m;
@@ -207,6 +216,15 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp == 4) HSA_T(3000);
+#ifdef HSA_TIMING
+  if (threadIdx.x == 0) {
+    g_cta_t[(blockIdx.y * gridDim.x + blockIdx.x) * 3] = globaltimer_ns();
+    uint32_t smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    g_cta_t[(blockIdx.y * gridDim.x + blockIdx.x) * 3 + 2] = smid;
+    g_cta_t[4096 + (blockIdx.y * gridDim.x + blockIdx.x) * 2] = clock64();
+  }
+#endif
   const int tile = blockIdx.x, h = blockIdx.y;
   const int row0 = tile * kTileM;
   const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
@@ -467,13 +485,14 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       constexpr int HC = D / 2;
       const bool epi = grp < 2;
       const int cbase = (grp & 1) * HC;
-      float den_part = 0.f;
+      float den_part = 0.f, den_part2 = 0.f;
       uint32_t fr[HC / 2];
       if (ok && p.do_linear && epi) {
         // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
         // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
         // and kept in registers until the epilogue
         ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
+        if (quad == 0) HSA_T(3012 + grp);
         const uint8_t* qrow = smem + L::kQ + r * 128;
         const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
 #pragma unroll
@@ -483,21 +502,20 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
           const int dh = cc >> 3, ch = cc & 7;
           const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
-          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float2 f = __bfloat1622float2(q2[i]);
-            const float a0 = f.x > 0.f ? f.x + 1.f : __expf(f.x);
-            const float a1 = f.y > 0.f ? f.y + 1.f : __expf(f.y);
-            const __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
-            fr[c16 * 4 + i] = *reinterpret_cast<const uint32_t*>(&pk);
-            const float2 rr = __bfloat1622float2(pk);  // the rounded values the MMA will see
-            den_part = fmaf(rr.x, z[2 * i], den_part);
-            den_part = fmaf(rr.y, z[2 * i + 1], den_part);
+            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
+            fr[c16 * 4 + i] = pk;
+            // the denominator uses the rounded values the MMA will see
+            den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
+            den_part2 = fmaf(__uint_as_float(pk & 0xffff0000u), z[2 * i + 1], den_part2);
           }
         }
+        den_part += den_part2;
       }
 
+      if (quad == 0) HSA_T(3014 + grp);
       // block ids of the next step are fetched one step ahead, off the critical path
       int nb0 = 0, nb1 = 0;
       if (first < nsteps) {
@@ -978,6 +996,12 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   }
 
   if (warp == 4) HSA_T(3010);
+#ifdef HSA_TIMING
+  if (threadIdx.x == 0) {
+    g_cta_t[(blockIdx.y * gridDim.x + blockIdx.x) * 3 + 1] = globaltimer_ns();
+    g_cta_t[4096 + (blockIdx.y * gridDim.x + blockIdx.x) * 2 + 1] = clock64();
+  }
+#endif
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
@@ -985,6 +1009,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 }
 
 #ifdef HSA_TIMING
+extern "C" int hsa_debug_read_cta_times(long long* host_out, int n) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_cta_t, sizeof(long long) * n));
+}
 extern "C" int hsa_debug_read_timing(long long* host_out, int n) {
   return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_hsa_timing, sizeof(long long) * n));
 }
