@@ -592,36 +592,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       constexpr int HC = D / 2;
       const bool epi = grp < 2;
       const int cbase = (grp & 1) * HC;
-      float den_part = 0.f, den_part2 = 0.f;
-      uint32_t fr[HC / 2];
-      if (ok && p.do_linear && epi) {
-        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
-        // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
-        // and kept in registers until the epilogue
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, ic & 1, bars, p.status));
-        if (quad == 0) HSA_T(3012 + grp);
-        const uint8_t* qrow = smem + L::kQ + r * 128;
-        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
-#pragma unroll
-        for (int c16 = 0; c16 < HC / 8; ++c16) {
-          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
-          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
-          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
-          const int dh = cc >> 3, ch = cc & 7;
-          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
-          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
-            fr[c16 * 4 + i] = pk;
-            // the denominator uses the rounded values the MMA will see
-            den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
-            den_part2 = fmaf(__uint_as_float(pk & 0xffff0000u), z[2 * i + 1], den_part2);
-          }
-        }
-        den_part += den_part2;
-      }
-
       if (quad == 0) HSA_T(3014 + grp);
       // block ids of the next step are fetched one step ahead, off the critical path
       int nb0 = 0, nb1 = 0;
@@ -839,6 +809,38 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 5);
       }
 
+      // ---- linear branch operands (Q is still in shared memory: the next item's tile is requested only
+      //      after phi(Q) has been handed over)
+      float den_part = 0.f, den_part2 = 0.f;
+      uint32_t fr[HC / 2];
+      if (ok && p.do_linear && epi) {
+        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
+        // MMA) and the partial denominator phi(q) . z -- after the group's last step, while the
+        // tensor pipe finishes the item's last products
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, ic & 1, bars, p.status));
+        if (quad == 0) HSA_T(3012 + grp);
+        const uint8_t* qrow = smem + L::kQ + r * 128;
+        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
+#pragma unroll
+        for (int c16 = 0; c16 < HC / 8; ++c16) {
+          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
+          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
+          const int dh = cc >> 3, ch = cc & 7;
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
+          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
+            fr[c16 * 4 + i] = pk;
+            // the denominator uses the rounded values the MMA will see
+            den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
+            den_part2 = fmaf(__uint_as_float(pk & 0xffff0000u), z[2 * i + 1], den_part2);
+          }
+        }
+        den_part += den_part2;
+      }
+
       // ---------------------------------------------------------------- epilogue
       // (this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D))
       if (ok && nsteps > 0) {
@@ -928,10 +930,14 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           inv_l = ltot > 0.f ? 1.f / ltot : 0.f;
         }
       }
-      if (ok && p.do_linear && epi) {
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, ic & 1, bars, p.status));
-        tc_fence_after();
-      }
+      // the linear numerator is final once the MMA lane's commit has arrived
+      auto wait_lin = [&]() {
+        if (ok && p.do_linear && epi) {
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, ic & 1, bars, p.status));
+          tc_fence_after();
+        }
+      };
+      if (!(epi && do_output)) wait_lin();
       if (quad == 0) HSA_T(3006 + grp);
       // The output tile is staged in the V stage that held the last step's values (the state
       // halves, if any, sit in the other two): free since the last P V, and not loaded again before
@@ -959,28 +965,46 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const bool plain = !p.g_lin && !p.g_sp && !(p.do_linear && p.lin_num != nullptr) && !p.ext_lin &&
                            !(SPLIT && nsplit > 1);
         if (plain) {
-          // no gates, no causal partials, no external linear output, no merge: 32 columns per trip
+          // no gates, no causal partials, no external linear output, no merge.  The sparse part is
+          // read and scaled first, while the tensor pipe still works on the linear numerator.
           const float il = has_o ? inv_l : 0.f, id = p.do_linear ? inv_den : 0.f;
-#pragma unroll 1
-          for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
-            uint32_t oa[32], ln[32];
+          float osp[HC];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) oa[i] = ln[i] = 0u;
-            if (has_o) tmem_ld32(o_tmem + c0, oa);
-            if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
-            tc_wait_ld();
+          for (int c0 = 0; c0 < HC; c0 += 32) {
+            uint32_t oa[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) oa[i] = 0u;
+            if (has_o) {
+              tmem_ld32(o_tmem + cbase + c0, oa);
+              tc_wait_ld();
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) osp[c0 + i] = __uint_as_float(oa[i]) * il;
+          }
+          wait_lin();
+#pragma unroll
+          for (int c0 = 0; c0 < HC; c0 += 32) {
+            uint32_t ln[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ln[i] = 0u;
+            if (p.do_linear) {
+              tmem_ld32(tmem + lane_off + kColLin + cbase + c0, ln);
+              tc_wait_ld();
+            }
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2)
-              pk[i >> 1] = pack_bf16(fmaf(__uint_as_float(oa[i]), il, __uint_as_float(ln[i]) * id),
-                                     fmaf(__uint_as_float(oa[i + 1]), il, __uint_as_float(ln[i + 1]) * id));
+              pk[i >> 1] = pack_bf16(fmaf(__uint_as_float(ln[i]), id, osp[c0 + i]),
+                                     fmaf(__uint_as_float(ln[i + 1]), id, osp[c0 + i + 1]));
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
-              const int cc = (c0 >> 3) + q4;  // 16-byte chunk of the row
+              const int cc = ((cbase + c0) >> 3) + q4;  // 16-byte chunk of the row
               *reinterpret_cast<uint4*>(stage_out + (cc >> 3) * L::kHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) =
                   make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
             }
           }
+        } else {
+          wait_lin();
         }
         // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
 #pragma unroll 1
