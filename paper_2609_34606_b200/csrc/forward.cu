@@ -1,10 +1,6 @@
 // hsa_forward kernel for sm_100a.
 //
-// Work items are (128-row query tile, head) pairs.  The plain kernel is persistent: one CTA per SM
-// takes the items b, b + gridDim.x, ... and the barriers, rings and score buffers run on from item
-// to item, so that the Q tile, the first K steps and the first Q K^T of the next item are
-// requested / issued under the epilogue of the current one.  The split kernel (long lists) has one
-// CTA per (tile, head, part).  384 threads in three warpgroups:
+// One CTA per (128-row query tile, head), 384 threads in three warpgroups:
 //   warp 0       TMA producer: Q tile, then the selected K/V pages gathered through the page
 //                table (two 64-token pages = 128 keys per step) into two 3-stage rings, then the
 //                hi/lo halves of the linear state; also owns the TMEM allocation
@@ -61,9 +57,9 @@ struct Smem {
   static constexpr int kQ = 0;
   static constexpr int kK = kTile;
   static constexpr int kV = kTile + kStages * kTile;
+  static constexpr int kStats = kK;  // float[2][128][4], reuses K stage 0 once the loop is over
   static constexpr int kBars = kTile + 2 * kStages * kTile;
-  static constexpr int kBarBytes = 3072;         // barriers and per-row values
-  static constexpr int kTotal = kBars + kBarBytes;  // the dynamic shared memory must start on a 1 KB boundary
+  static constexpr int kTotal = kBars + 1024 + 1024;  // barriers + per-row reference, + slack
 };
 
 struct Bars {
@@ -78,19 +74,18 @@ struct Bars {
   uint64_t tok[2];  // exponential-phase token: the two softmax groups take turns on the SFU
   uint64_t lin_a_full;
   uint64_t lin_done;
-  uint64_t final_known;  // the MMA lane has seen the last P of the item: `final` is valid
-  uint64_t o_free;       // both groups have read the accumulators of the item out of TMEM
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile int redo;
-  volatile int final;    // this attempt's result stands (no safe pass follows)
-  float mref[128];       // per-row exponent reference (log2 domain) of the fast pass
-  float2 stat[2][128];   // per group and row: partial row sum, partial linear denominator
+  float mref[128];  // per-row exponent reference (log2 domain) of the fast pass
 };
-static_assert(sizeof(Bars) <= 3072, "barrier block must fit its shared-memory slot");
+static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory slot");
 
 #ifndef HSA_INTERLEAVE
 #define HSA_INTERLEAVE 8
+#endif
+#ifndef HSA_PDL
+#define HSA_PDL 1
 #endif
 #ifndef HSA_CONTINUOUS
 #define HSA_CONTINUOUS 8
@@ -200,8 +195,6 @@ __device__ __forceinline__ void init_barriers(Bars* bars) {
   mbar_init(&bars->tok[1], 128);
   mbar_init(&bars->lin_a_full, 256);
   mbar_init(&bars->lin_done, 1);
-  mbar_init(&bars->final_known, 1);
-  mbar_init(&bars->o_free, 128 * kGroups);
   bars->redo = 0;
   fence_mbar_init();
 }
@@ -217,61 +210,45 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_out, const FwdParams p) {
   using L = Smem<D>;
   constexpr int DH = D / 64;  // 64-element (128-byte) slabs per row
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  uint8_t* smem = smem_raw;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
   Bars* bars = reinterpret_cast<Bars*>(smem + L::kBars);
+  float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][l, den, -, -]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp == 4) HSA_T(3000);
-  if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled tiles need the 1 KB boundary
-    if (threadIdx.x == 0) atomicCAS(p.status, 0, kDevBounds);
-    return;
-  }
-  // Work items are (tile, head) pairs, tile fastest.  The plain kernel is persistent: CTA b takes the
-  // items b, b + gridDim.x, ... one after the other, so that the set-up, the first loads and the
-  // first Q K^T of an item run under the epilogue of the item before it.  The split kernel keeps
-  // one item per CTA: grid (tile, head, part).
-  const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
-  const int n_items = n_tiles * p.H;
-  const int item0 = SPLIT ? static_cast<int>(blockIdx.y) * n_tiles + static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
-  const int item_stride = SPLIT ? n_items : static_cast<int>(gridDim.x);
-  const int part = SPLIT ? static_cast<int>(blockIdx.z) : 0;
-  const int nparts = SPLIT ? static_cast<int>(gridDim.z) : 1;
-  struct Item {
-    int tile, h, row0, cnt, nsteps, nsplit;
-    const int32_t* sel;
-  };
-  auto get_item = [&](int item) -> Item {
-    Item I;
-    I.tile = item % n_tiles;
-    I.h = item / n_tiles;
-    I.row0 = I.tile * kTileM;
-    const int g = p.group_tokens > 0 ? I.row0 / p.group_tokens : 0;
-    I.sel = p.sel_idx + (static_cast<size_t>(I.h) * p.n_groups + g) * p.kcap;
-    int cnt = p.do_sparse ? p.sel_cnt[static_cast<size_t>(I.h) * p.n_groups + g] : 0;
-    cnt = max(0, min(cnt, min(p.kcap, p.n_blocks)));  // never more blocks than the history holds
-    // A long list is split over the CTAs (tile, head, 0 .. nsplit - 1): each takes a run of whole
-    // two-page steps; CTAs beyond nsplit leave before they set anything up.
-    I.nsplit = 1;
-    if (SPLIT && nparts > 1) {
-      const int steps_total = (cnt + 1) / 2;
-      const int split_steps = p.split_blocks / 2;
-      int nsplit = min(nparts, max(1, (steps_total + split_steps - 1) / split_steps));
-      const int steps_per = (steps_total + nsplit - 1) / nsplit;
-      if (steps_per > 0) nsplit = (steps_total + steps_per - 1) / steps_per;  // no empty part
-      I.nsplit = nsplit;
-      if (nsplit > 1 && part < nsplit) {
-        const int b_lo = 2 * part * steps_per;
-        const int b_hi = min(cnt, 2 * (part + 1) * steps_per);
-        I.sel += b_lo;
-        cnt = b_hi - b_lo;
-      }
+#if HSA_PDL
+  // launched with programmatic stream serialization: this grid may be scheduled while the kernel
+  // before it (block selection) is still draining; nothing of that kernel's output is read above
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int row0 = tile * kTileM;
+  const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
+  const int32_t* sel = p.sel_idx + (static_cast<size_t>(h) * p.n_groups + g) * p.kcap;
+  int cnt = p.do_sparse ? p.sel_cnt[static_cast<size_t>(h) * p.n_groups + g] : 0;
+  cnt = max(0, min(cnt, min(p.kcap, p.n_blocks)));  // never more blocks than the history holds
+  // A long list is split over the CTAs (tile, head, 0 .. nsplit - 1): each takes a run of whole
+  // two-page steps; CTAs beyond nsplit leave before they set anything up.
+  int nsplit = 1;
+  const int part = blockIdx.z;
+  if (SPLIT && gridDim.z > 1) {
+    const int steps_total = (cnt + 1) / 2;
+    const int split_steps = p.split_blocks / 2;
+    nsplit = min(static_cast<int>(gridDim.z), max(1, (steps_total + split_steps - 1) / split_steps));
+    const int steps_per = (steps_total + nsplit - 1) / nsplit;
+    if (steps_per > 0) nsplit = (steps_total + steps_per - 1) / steps_per;  // no empty part
+    if (part >= nsplit) return;
+    if (nsplit > 1) {
+      const int b_lo = 2 * part * steps_per;
+      const int b_hi = min(cnt, 2 * (part + 1) * steps_per);
+      sel += b_lo;
+      cnt = b_hi - b_lo;
     }
-    I.cnt = cnt;
-    I.nsteps = (cnt + 1) / 2;
-    return I;
-  };
-  if (SPLIT && part >= get_item(item0).nsplit) return;
+  }
+  const int slot = (tile * p.H + h) * static_cast<int>(gridDim.z) + part;  // this CTA's partial-result slot
+  const int nsteps = (cnt + 1) / 2;
 
   if (threadIdx.x == 0) {
     bars->abort_flag = 0;
@@ -305,56 +282,33 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     return true;
   };
 
-  // Running counters, the same in every role: K / score steps and V steps (the state halves count
-  // as two) since the barriers were last initialised, and items since then.  Ring stage, score
-  // buffer and barrier parity of a step all follow from them, so the rings run on across items.
-  int G = 0, Gv = 0, ic = 0;
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    // one lane of warp 0 and one of warp 1 do the issuing; elected once, because they carry state
-    // from item to item
-    const bool leader = elect_one_sync();
-    if (warp == 0 && leader) {
-      tma_prefetch_desc(&tm_q);
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-    }
-    // what the tail of the previous item has already done for this one (plain kernel only)
-    int pre_k = -1;       // producer: Q requested and this many K steps; -1: nothing
-    bool pre_qk = false;  // MMA lane: the first Q K^T are issued
-#pragma unroll 1
-    for (int item = item0; item < n_items; item += item_stride) {
-    const Item I = get_item(item);
-    const int h = I.h, row0 = I.row0, cnt = I.cnt, nsteps = I.nsteps;
-    const int32_t* sel = I.sel;
-    safe = false;
 #pragma unroll 1
     for (int attempt = 0; attempt < 2; ++attempt) {
     if (warp == 0) {
       // ================================================================= TMA producer
-      if (leader) {
-        auto load_q = [&](int xh, int xrow0) {
-          mbar_expect_tx(&bars->q_full, L::kTile);
-          for (int dh = 0; dh < DH; ++dh)
-            tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, xh, xrow0);
-        };
-        if (pre_k < 0) load_q(h, row0);
+      if (elect_one_sync()) {
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        mbar_expect_tx(&bars->q_full, L::kTile);
+        for (int dh = 0; dh < DH; ++dh)
+          tma_load_3d(smem + L::kQ + dh * L::kHalf, &tm_q, &bars->q_full, dh * 64, h, row0);
         bool ok = true;
-        int armed_k = 0, armed_v = 0;  // loads issued per ring in this attempt, for the drain on abort
-        // step j of the item (xsel, xcnt, xh), whose steps start at gbase in its ring
-        auto load_kv = [&](const int32_t* xsel, int xcnt, int xh, int gbase, int j, bool is_k) -> bool {
-          auto page_row = [&](int idx) -> int32_t {
-            int blk = xsel[idx];
-            if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
-              atomicCAS(p.status, 0, kDevBounds);
-              blk = 0;
-            }
-            return (p.page_table[blk] * p.H + xh) * kBlock;
-          };
-          const int gj = gbase + j;
-          const int s = gj % kStages;
-          const uint32_t ph = (gj / kStages) & 1;
-          const int npg = min(2, xcnt - 2 * j);
+        int armed_k = 0, armed_v = 0;  // loads issued per ring, for the drain on abort
+        auto page_row = [&](int idx) -> int32_t {
+          int blk = sel[idx];
+          if (blk < 0 || blk >= p.n_blocks) {  // never follow a bad index into the pool
+            atomicCAS(p.status, 0, kDevBounds);
+            blk = 0;
+          }
+          return (p.page_table[blk] * p.H + h) * kBlock;
+        };
+        auto load_kv = [&](int j, bool is_k) -> bool {
+          const int s = j % kStages;
+          const uint32_t ph = (j / kStages) & 1;
+          const int npg = min(2, cnt - 2 * j);
           uint64_t* full = is_k ? &bars->k_full[s] : &bars->v_full[s];
           uint64_t* empty = is_k ? &bars->k_empty[s] : &bars->v_empty[s];
           uint8_t* dst = smem + (is_k ? L::kK : L::kV) + s * L::kTile;
@@ -373,20 +327,18 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           return true;
         };
         // K runs three steps ahead of V: the scores of step j+3 are issued right after P V of j
-        for (int j = max(pre_k, 0); j < min(kSBufs, nsteps) && ok; ++j) ok = load_kv(sel, cnt, h, G, j, true);
-        if (pre_k > 0) armed_k = pre_k;
-        pre_k = -1;
+        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = load_kv(j, true);
 #pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
-          ok = load_kv(sel, cnt, h, Gv, j, false);
-          if (ok && j + kSBufs < nsteps) ok = load_kv(sel, cnt, h, G, j + kSBufs, true);
+          ok = load_kv(j, false);
+          if (ok && j + kSBufs < nsteps) ok = load_kv(j + kSBufs, true);
         }
         if (ok && p.do_linear) {
           // hi and lo halves of the D x D state ride the V ring as two more "steps"
           for (int hl = 0; hl < 2 && ok; ++hl) {
-            const int gj = Gv + nsteps + hl;
-            const int s = gj % kStages;
-            const uint32_t ph = (gj / kStages) & 1;
+            const int j = nsteps + hl;
+            const int s = j % kStages;
+            const uint32_t ph = (j / kStages) & 1;
             ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
             if (!ok) break;
             const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
@@ -398,62 +350,33 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             ++armed_v;
           }
         }
-        // the Q tile has landed before the item ends (a tile without any step never looks at it)
-        if (ok) ok = wait_bar(&bars->q_full, ic & 1, bars, p.status);
-        if (!SPLIT && ok && item + item_stride < n_items) {
-          // Next item: once this one's scores are all consumed (and phi(Q) is taken), the Q tile and
-          // the K ring are free, so its Q and first K steps are requested under the epilogue.
-          ok = wait_bar(&bars->final_known, ic & 1, bars, p.status);
-          if (ok && p.do_linear) ok = wait_bar(&bars->lin_a_full, ic & 1, bars, p.status);
-          if (ok && bars->final) {
-            const Item N = get_item(item + item_stride);
-            load_q(N.h, N.row0);
-            pre_k = 0;
-            for (int j = 0; j < min(kSBufs, N.nsteps) && ok; ++j) {
-              ok = load_kv(N.sel, N.cnt, N.h, G + nsteps, j, true);
-              if (ok) ++pre_k;
-            }
-          }
-        }
         if (!ok) {
           // drain: let every copy already issued land before the CTA's shared memory goes away
-          mbar_wait(&bars->q_full, ic & 1, 1u << 16);
-          for (int i = 0; i < 2; ++i) {
-            const int arms = i == 0 ? armed_k : armed_v;
-            for (int a = max(0, arms - kStages); a < arms; ++a) {  // the last loads of each stage
-              const int gj = (i == 0 ? G : Gv) + a;
-              mbar_wait(i == 0 ? &bars->k_full[gj % kStages] : &bars->v_full[gj % kStages], (gj / kStages) & 1, 1u << 16);
-            }
-          }
-          if (pre_k >= 0) {  // requests made for the next item
-            mbar_wait(&bars->q_full, (ic + 1) & 1, 1u << 16);
-            for (int a = 0; a < pre_k; ++a) {
-              const int gj = G + nsteps + a;
-              mbar_wait(&bars->k_full[gj % kStages], (gj / kStages) & 1, 1u << 16);
+          for (int s = 0; s < kStages; ++s) {
+            for (int i = 0; i < 2; ++i) {
+              const int arms = i == 0 ? armed_k : armed_v;
+              uint64_t* bar = i == 0 ? &bars->k_full[s] : &bars->v_full[s];
+              const int last = ((arms - 1 - s) / kStages) * kStages + s;  // last step armed on s
+              if (arms > s) mbar_wait(bar, (last / kStages) & 1, 1u << 16);
             }
           }
         }
       }
     } else if (warp == 1) {
       // ================================================================= MMA issuer
-      if (leader) {
+      if (elect_one_sync()) {
         constexpr uint32_t kHiSw = desc_hi_sw128(1024);
         const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::kQ), 16);
-        bool ok = true;
-        if (!pre_qk) {
-          ok = wait_bar(&bars->q_full, ic & 1, bars, p.status);
-          tc_fence_after();
-        }
+        bool ok = wait_bar(&bars->q_full, 0, bars, p.status);
+        tc_fence_after();
         HSA_T(3011);
-        // scores of step j of an item with xcnt pages whose steps start at gbase
-        auto issue_qk = [&](int xcnt, int gbase, int j) -> bool {
-          const int gj = gbase + j;
-          const int s = gj % kStages;
-          if (!wait_bar(&bars->k_full[s], (gj / kStages) & 1, bars, p.status)) return false;
+        auto issue_qk = [&](int j) -> bool {
+          const int s = j % kStages;
+          if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
           tc_fence_after();
           const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::kK + s * L::kTile), 16);
-          const uint32_t d_tmem = tmem + kColS + 128 * (gj % kSBufs);
-          if (xcnt - 2 * j >= 2) {
+          const uint32_t d_tmem = tmem + kColS + 128 * (j % kSBufs);
+          if (cnt - 2 * j >= 2) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 0, 0);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
@@ -469,21 +392,19 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
           }
           tc_commit(&bars->k_empty[s]);
-          tc_commit(&bars->s_full[gj % kSBufs]);
+          tc_commit(&bars->s_full[j % kSBufs]);
           return true;
         };
-        if (!pre_qk)
-          for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = issue_qk(cnt, G, j);
-        pre_qk = false;
+        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = issue_qk(j);
 #pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
-          const int s = (Gv + j) % kStages;
-          const int b = (G + j) % kSBufs;
+          const int s = j % kStages;
+          const int b = j % kSBufs;
           HSA_T(2048 + j * 8 + 0);
-          ok = wait_bar(&bars->p_full[b], ((G + j) / kSBufs) & 1, bars, p.status);
+          ok = wait_bar(&bars->p_full[b], (j / kSBufs) & 1, bars, p.status);
           if (!ok) break;
           HSA_T(2048 + j * 8 + 1);
-          ok = wait_bar(&bars->v_full[s], ((Gv + j) / kStages) & 1, bars, p.status);
+          ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
           if (!ok) break;
           tc_fence_after();
           HSA_T(2048 + j * 8 + 2);
@@ -505,21 +426,16 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           HSA_T(2048 + j * 8 + 3);
           // the scores of step j+3 overwrite the P just consumed: issued after the P V above,
           // the tensor pipe runs them in order
-          if (j + kSBufs < nsteps) ok = issue_qk(cnt, G, j + kSBufs);
+          if (j + kSBufs < nsteps) ok = issue_qk(j + kSBufs);
           HSA_T(2048 + j * 8 + 4);
         }
-        if (ok) {
-          tc_commit(&bars->o_done);
-          // every P of the item has been seen, so every step has had its say on the safe pass
-          bars->final = (safe || bars->redo == 0) ? 1 : 0;
-          mbar_arrive(&bars->final_known);
-        }
+        if (ok) tc_commit(&bars->o_done);
         if (ok && p.do_linear) {
-          ok = wait_bar(&bars->lin_a_full, ic & 1, bars, p.status);
+          ok = wait_bar(&bars->lin_a_full, 0, bars, p.status);
           for (int hl = 0; hl < 2 && ok; ++hl) {
-            const int gj = Gv + nsteps + hl;
-            const int s = gj % kStages;
-            ok = wait_bar(&bars->v_full[s], (gj / kStages) & 1, bars, p.status);
+            const int j = nsteps + hl;
+            const int s = j % kStages;
+            ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
             if (!ok) break;
             tc_fence_after();
             constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
@@ -532,38 +448,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           if (ok) tc_commit(&bars->lin_done);
         }
-        if (!SPLIT && ok && item + item_stride < n_items && bars->final) {
-          // Next item: its first scores are issued as soon as the groups have read this item's
-          // accumulators out of TMEM (the linear branch borrows two score buffers), so that they
-          // are ready when the groups come out of the epilogue.
-          ok = wait_bar(&bars->o_free, ic & 1, bars, p.status);
-          if (ok) ok = wait_bar(&bars->q_full, (ic + 1) & 1, bars, p.status);
-          tc_fence_after();
-          const Item N = get_item(item + item_stride);
-          for (int j = 0; j < min(kSBufs, N.nsteps) && ok; ++j) ok = issue_qk(N.cnt, G + nsteps, j);
-          pre_qk = ok;
-        }
       }
     }
       if (!end_of_attempt()) break;
       safe = true;
-      G = Gv = ic = 0;  // the barriers were initialised again
-    }
-    G += nsteps;
-    Gv += nsteps + (p.do_linear ? 2 : 0);
-    ++ic;
-    if (bars->abort_flag) break;
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(HSA_SMREGS));
-    int mc = 0;  // exponent references published so far (one per item that ran a fast pass with steps)
-#pragma unroll 1
-    for (int item = item0; item < n_items; item += item_stride) {
-    const Item I = get_item(item);
-    const int tile = I.tile, h = I.h, row0 = I.row0, cnt = I.cnt, nsteps = I.nsteps, nsplit = I.nsplit;
-    const int32_t* sel = I.sel;
-    const int slot = (tile * p.H + h) * nparts + part;  // this CTA's partial-result slot
-    safe = false;
 #pragma unroll 1
     for (int attempt = 0; attempt < 2; ++attempt) {
       // ================================================================= softmax groups + epilogue
@@ -592,6 +483,36 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       constexpr int HC = D / 2;
       const bool epi = grp < 2;
       const int cbase = (grp & 1) * HC;
+      float den_part = 0.f, den_part2 = 0.f;
+      uint32_t fr[HC / 2];
+      if (ok && p.do_linear && epi) {
+        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
+        // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
+        // and kept in registers until the epilogue
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
+        if (quad == 0) HSA_T(3012 + grp);
+        const uint8_t* qrow = smem + L::kQ + r * 128;
+        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
+#pragma unroll
+        for (int c16 = 0; c16 < HC / 8; ++c16) {
+          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
+          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
+          const int dh = cc >> 3, ch = cc & 7;
+          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
+          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
+            fr[c16 * 4 + i] = pk;
+            // the denominator uses the rounded values the MMA will see
+            den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
+            den_part2 = fmaf(__uint_as_float(pk & 0xffff0000u), z[2 * i + 1], den_part2);
+          }
+        }
+        den_part += den_part2;
+      }
+
       if (quad == 0) HSA_T(3014 + grp);
       // block ids of the next step are fetched one step ahead, off the critical path
       int nb0 = 0, nb1 = 0;
@@ -611,10 +532,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           nb0 = sel[2 * (j + stride)];
           nb1 = (2 * (j + stride) + 1 < cnt) ? sel[2 * (j + stride) + 1] : 0;
         }
-        const int b = (G + j) % kSBufs;
+        const int b = j % kSBufs;
         const uint32_t s_tmem = tmem + lane_off + kColS + 128 * b;
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 0);
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], ((G + j) / kSBufs) & 1, bars, p.status));
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], (j / kSBufs) & 1, bars, p.status));
         if (!ok) break;
         tc_fence_after();
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 1);
@@ -677,7 +598,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
             if (j > 0) {
               // O must be quiescent: the previous P V has to be complete before it is rescaled
-              ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (G + j - 1) & 1, bars, p.status));
+              ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (j - 1) & 1, bars, p.status));
               if (!ok) break;
               tc_fence_after();
               if (__any_sync(0xffffffffu, factor != 1.f)) {
@@ -697,7 +618,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
         } else if (j < kGroups) {
           // first step of groups 1 and 2 in the fast pass: take the reference group 0 fixed
-          ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready, mc & 1, bars, p.status));
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready, 0, bars, p.status));
           if (!ok) break;
           t_ref = bars->mref[r];
         }
@@ -809,42 +730,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 5);
       }
 
-      // ---- linear branch operands (Q is still in shared memory: the next item's tile is requested only
-      //      after phi(Q) has been handed over)
-      float den_part = 0.f, den_part2 = 0.f;
-      uint32_t fr[HC / 2];
-      if (ok && p.do_linear && epi) {
-        // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
-        // MMA) and the partial denominator phi(q) . z -- after the group's last step, while the
-        // tensor pipe finishes the item's last products
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, ic & 1, bars, p.status));
-        if (quad == 0) HSA_T(3012 + grp);
-        const uint8_t* qrow = smem + L::kQ + r * 128;
-        const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
-#pragma unroll
-        for (int c16 = 0; c16 < HC / 8; ++c16) {
-          const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
-          const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
-          const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
-          const int dh = cc >> 3, ch = cc & 7;
-          const uint4 raw = *reinterpret_cast<const uint4*>(qrow + dh * L::kHalf + ((ch ^ (r & 7)) << 4));
-          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
-            fr[c16 * 4 + i] = pk;
-            // the denominator uses the rounded values the MMA will see
-            den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
-            den_part2 = fmaf(__uint_as_float(pk & 0xffff0000u), z[2 * i + 1], den_part2);
-          }
-        }
-        den_part += den_part2;
-      }
-
       // ---------------------------------------------------------------- epilogue
       // (this group's columns of the output row: group 0 -> [0, D/2), group 1 -> [D/2, D))
       if (ok && nsteps > 0) {
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, ic & 1, bars, p.status));
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
         tc_fence_after();
       }
       if (quad == 0) HSA_T(3002 + grp);
@@ -859,15 +748,15 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mbar_arrive(&bars->lin_a_full);
       }
       // publish this group's partial row sum and denominator, then read the other group's
-      bars->stat[grp][r] = make_float2(l, den_part);
+      stats[(grp * 128 + r) * 4 + 0] = l;
+      stats[(grp * 128 + r) * 4 + 1] = den_part;
       if (quad == 0) HSA_T(3004 + grp);
       named_bar_sync(1, 128 * kGroups);
       float lsum = 0.f, den = 0.f;
 #pragma unroll
       for (int gg = 0; gg < kGroups; ++gg) {
-        const float2 st = bars->stat[gg][r];
-        lsum += st.x;
-        den += st.y;
+        lsum += stats[(gg * 128 + r) * 4 + 0];
+        den += stats[(gg * 128 + r) * 4 + 1];
       }
       float inv_l = (nsteps > 0 && lsum > 0.f) ? 1.f / lsum : 0.f;
       const bool has_o = nsteps > 0;
@@ -930,19 +819,15 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           inv_l = ltot > 0.f ? 1.f / ltot : 0.f;
         }
       }
-      // the linear numerator is final once the MMA lane's commit has arrived
-      auto wait_lin = [&]() {
-        if (ok && p.do_linear && epi) {
-          ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, ic & 1, bars, p.status));
-          tc_fence_after();
-        }
-      };
-      if (!(epi && do_output)) wait_lin();
+      if (ok && p.do_linear && epi) {
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
+        tc_fence_after();
+      }
       if (quad == 0) HSA_T(3006 + grp);
-      // The output tile is staged in the V stage that held the last step's values (the state
-      // halves, if any, sit in the other two): free since the last P V, and not loaded again before
-      // the next item, which starts after the store below has read it.
-      uint8_t* stage_out = smem + L::kV + ((Gv + nsteps + 2) % kStages) * L::kTile;
+      // The output tile is staged in the Q tile's shared memory.  A tile with no step and no linear
+      // branch has not looked at Q at all: its TMA load may still be in flight and must land first.
+      if (ok && epi && nsteps == 0 && !p.do_linear)
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
       if (ok && epi && do_output) {  // warp-uniform: the TMEM loads below are warp-collective
         const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
         float lin_den = den;
@@ -965,46 +850,28 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const bool plain = !p.g_lin && !p.g_sp && !(p.do_linear && p.lin_num != nullptr) && !p.ext_lin &&
                            !(SPLIT && nsplit > 1);
         if (plain) {
-          // no gates, no causal partials, no external linear output, no merge.  The sparse part is
-          // read and scaled first, while the tensor pipe still works on the linear numerator.
+          // no gates, no causal partials, no external linear output, no merge: 32 columns per trip
           const float il = has_o ? inv_l : 0.f, id = p.do_linear ? inv_den : 0.f;
-          float osp[HC];
+#pragma unroll 1
+          for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
+            uint32_t oa[32], ln[32];
 #pragma unroll
-          for (int c0 = 0; c0 < HC; c0 += 32) {
-            uint32_t oa[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) oa[i] = 0u;
-            if (has_o) {
-              tmem_ld32(o_tmem + cbase + c0, oa);
-              tc_wait_ld();
-            }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) osp[c0 + i] = __uint_as_float(oa[i]) * il;
-          }
-          wait_lin();
-#pragma unroll
-          for (int c0 = 0; c0 < HC; c0 += 32) {
-            uint32_t ln[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) ln[i] = 0u;
-            if (p.do_linear) {
-              tmem_ld32(tmem + lane_off + kColLin + cbase + c0, ln);
-              tc_wait_ld();
-            }
+            for (int i = 0; i < 32; ++i) oa[i] = ln[i] = 0u;
+            if (has_o) tmem_ld32(o_tmem + c0, oa);
+            if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
+            tc_wait_ld();
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2)
-              pk[i >> 1] = pack_bf16(fmaf(__uint_as_float(ln[i]), id, osp[c0 + i]),
-                                     fmaf(__uint_as_float(ln[i + 1]), id, osp[c0 + i + 1]));
+              pk[i >> 1] = pack_bf16(fmaf(__uint_as_float(oa[i]), il, __uint_as_float(ln[i]) * id),
+                                     fmaf(__uint_as_float(oa[i + 1]), il, __uint_as_float(ln[i + 1]) * id));
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
-              const int cc = ((cbase + c0) >> 3) + q4;  // 16-byte chunk of the row
-              *reinterpret_cast<uint4*>(stage_out + (cc >> 3) * L::kHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) =
+              const int cc = (c0 >> 3) + q4;  // 16-byte chunk of the row
+              *reinterpret_cast<uint4*>(smem + L::kQ + (cc >> 3) * L::kHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) =
                   make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
             }
           }
-        } else {
-          wait_lin();
         }
         // rolled on purpose: 16 columns per trip keeps this once-per-tile code small
 #pragma unroll 1
@@ -1097,11 +964,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           }
           if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 2);
-          // stage the row (each thread touches only its own) in the 128-byte-swizzled layout the
-          // output tensor map expects
+          // stage the row into the Q tile's shared memory (dead by now; each thread touches only
+          // its own row) in the 128-byte-swizzled layout the output tensor map expects
           {
             const int cc = c0 >> 3;  // 16-byte chunk of the row
-            uint8_t* srow = stage_out + (cc >> 3) * L::kHalf + r * 128;
+            uint8_t* srow = smem + L::kQ + (cc >> 3) * L::kHalf + r * 128;
             *reinterpret_cast<uint4*>(srow + (((cc & 7) ^ (r & 7)) << 4)) =
                 make_uint4(packed[0], packed[1], packed[2], packed[3]);
             *reinterpret_cast<uint4*>(srow + ((((cc + 1) & 7) ^ (r & 7)) << 4)) =
@@ -1109,16 +976,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
         }
       }
-      // the accumulators of this item have been read: the tensor pipe may start on the next item
-      tc_fence_before();
-      mbar_arrive(&bars->o_free);
       // both epilogue groups have staged their columns: one elected thread stores the tile
       // (rows past the end of the chunk are clipped by the tensor map)
       fence_proxy_async_smem();
       named_bar_sync(2, 128 * kGroups);
       if (ok && do_output && warp == 4) {
         if (elect_one_sync()) {
-          for (int dh = 0; dh < DH; ++dh) tma_store_3d(&tm_out, stage_out + dh * L::kHalf, dh * 64, h, row0);
+          for (int dh = 0; dh < DH; ++dh) tma_store_3d(&tm_out, smem + L::kQ + dh * L::kHalf, dh * 64, h, row0);
           tma_store_commit();
           tma_store_wait_read();  // the tile must stay in shared memory until it has been read
         }
@@ -1126,13 +990,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       if (quad == 0) HSA_T(3008 + grp);
       if (!end_of_attempt()) break;
       safe = true;
-      G = Gv = ic = mc = 0;  // the barriers were initialised again
-    }
-    if (nsteps > 0 && !safe) ++mc;  // group 0 published a reference in the fast pass
-    G += nsteps;
-    Gv += nsteps + (p.do_linear ? 2 : 0);
-    ++ic;
-    if (bars->abort_flag) break;
     }
   }
 
@@ -1149,14 +1006,8 @@ extern "C" int hsa_debug_read_timing(long long* host_out, int n) {
 }
 #endif
 
-static int g_fwd_sms = 0;  // SMs of the device: the persistent kernel runs one CTA on each
-
 cudaError_t forward_init() {
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_fwd_sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(hsa_forward_kernel<128, false>,
+  cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kTotal);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(hsa_forward_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1174,23 +1025,24 @@ cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q, c
                            const CUtensorMap& tm_v, const CUtensorMap& tm_state, const CUtensorMap& tm_out,
                            cudaStream_t st) {
   const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
+  dim3 grid(n_tiles, p.H, p.max_splits > 1 ? p.max_splits : 1);
   const bool split = p.max_splits > 1;
-  // split: one CTA per (tile, head, part); plain: one persistent CTA per SM over the (tile, head) items
-  const int n_items = n_tiles * p.H;
-  dim3 grid(n_tiles, p.H, p.max_splits);
-  if (!split) grid = dim3(n_items < g_fwd_sms ? n_items : (g_fwd_sms > 0 ? g_fwd_sms : 1), 1, 1);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = D == 128 ? Smem<128>::kTotal : Smem<64>::kTotal;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = HSA_PDL ? 1 : 0;
   if (D == 128) {
-    if (split)
-      hsa_forward_kernel<128, true><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
-    else
-      hsa_forward_kernel<128, false><<<grid, kThreads, Smem<128>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
-  } else {
-    if (split)
-      hsa_forward_kernel<64, true><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
-    else
-      hsa_forward_kernel<64, false><<<grid, kThreads, Smem<64>::kTotal, st>>>(tm_q, tm_k, tm_v, tm_state, tm_out, p);
+    if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, true>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
+    return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, false>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
   }
-  return cudaGetLastError();
+  if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, true>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
+  return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, false>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
 }
 
 }  // namespace hsa
