@@ -38,7 +38,6 @@ namespace {
 #define HSA_SMREGS 224
 #endif
 constexpr int kGroups = HSA_GROUPS;  // softmax groups; group g takes the KV steps j = g (mod kGroups)
-constexpr bool kTokens = false;       // serialise the groups' exponential phases (2 groups only)
 constexpr int kThreads = 128 + 128 * kGroups;
 constexpr int kStages = 3;   // K ring and V ring depth
 constexpr int kSBufs = 3;    // score buffers in TMEM
@@ -71,7 +70,6 @@ struct Bars {
   uint64_t pv_done;
   uint64_t o_done;
   uint64_t mref_ready;
-  uint64_t tok[2];  // exponential-phase token: the two softmax groups take turns on the SFU
   uint64_t lin_a_full;
   uint64_t lin_done;
   uint32_t tmem_base;
@@ -151,27 +149,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
   return m;
 }
-__device__ __forceinline__ uint64_t pack2(float a, float b) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-// (a0, a1) * s2 + t2 on the packed fp32 pipe
-__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, uint64_t s2,
-                                      uint64_t t2) {
-  uint64_t d;
-  const uint64_t a = pack2(a0, a1);
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(s2), "l"(t2));
-  unpack2(d, d0, d1);
-}
-__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
@@ -191,8 +168,6 @@ __device__ __forceinline__ void init_barriers(Bars* bars) {
   mbar_init(&bars->pv_done, 1);
   mbar_init(&bars->o_done, 1);
   mbar_init(&bars->mref_ready, 128);  // group 0 publishes the per-row reference
-  mbar_init(&bars->tok[0], 128);
-  mbar_init(&bars->tok[1], 128);
   mbar_init(&bars->lin_a_full, 256);
   mbar_init(&bars->lin_done, 1);
   bars->redo = 0;
@@ -520,11 +495,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         nb0 = sel[2 * first];
         nb1 = (2 * first + 1 < cnt) ? sel[2 * first + 1] : 0;
       }
-      // fast pass: the two groups alternate on the exponential phase.  Both are bound by the same
-      // SFU pipe there, so running the phases one after the other costs nothing and lets each
-      // group's loads, stores and barrier traffic hide under the other's exponentials.
-      if (kTokens && !safe && grp == 1) mbar_arrive(&bars->tok[0]);
-      int tok_i = 0;
 #pragma unroll 1
       for (int j = first; j < nsteps; j += stride) {
         int blk0 = nb0, blk1 = nb1;
@@ -628,11 +598,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const float nt = -t_ref;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
         if (!early_ld) tmem_ld32(s_tmem, cbuf[0]);
-        if (kTokens && !safe) {
-          ok = __all_sync(0xffffffffu, wait_bar(&bars->tok[grp], tok_i & 1, bars, p.status));
-          if (!ok) break;
-          ++tok_i;
-        }
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 3);
 #if HSA_CONTINUOUS
         if (nchunks == 4 && !need_mask) {
@@ -674,7 +639,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               for (int i = 0; i < 32; ++i)
                 if (i >= lim) x[i] = 0xff800000u;  // -inf
             }
-#if HSA_INTERLEAVE
             // software pipeline over the chunk's 32 columns: scale-and-shift of column i, the
             // exponential of column i - LAG and the row sum / bf16 pack of column i - LAG - LAG2 are
             // issued next to each other, so that the FMA-pipe work fills the issue slots between
@@ -693,25 +657,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (k & 1) pk[k >> 1] = pack_bf16(y[k - 1], y[k]);
               }
             }
-#else
-            // stage by stage over the whole chunk, so that 32 independent operations of each kind
-            // are in flight: scale-and-shift, exponential, row sum, bf16 pack
-            float y[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = fmaf(__uint_as_float(x[i]), sl2, nt);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = ex2(y[i]);
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              acc[0] += y[i];
-              acc[1] += y[i + 1];
-              acc[2] += y[i + 2];
-              acc[3] += y[i + 3];
-            }
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) pk[i >> 1] = pack_bf16(y[i], y[i + 1]);
-#endif
             tmem_st16(s_tmem + 16 * c, pk);
             if (quad == 0) HSA_T(3100 + grp * 256 + (j / kGroups) * 8 + c);
           }
@@ -722,7 +667,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           // a weight far above the fixed reference: finite here, but the tile is redone safely
           if (!safe && !(lstep <= kRedoSum)) bars->redo = 1;
         }
-        if (kTokens && !safe) mbar_arrive(&bars->tok[grp ^ 1]);
         if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 4);
         tc_wait_st();
         tc_fence_before();
