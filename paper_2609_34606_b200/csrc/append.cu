@@ -305,6 +305,9 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
 
   // the reduction kernel behind this one may be scheduled early; it waits for this grid itself
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // this grid is itself launched as a programmatic dependent: whatever ran before it in the stream
+  // (the forward kernel of the layer before, a copy) is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const int h = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -590,8 +593,17 @@ cudaError_t launch_append(const AppendArgs& a_in, const AppendMaps* maps, cudaSt
     const int per = (nb + a.nsplit - 1) / a.nsplit;
     a.nsplit = (nb + per - 1) / per;  // no empty CTAs
     dim3 grid(a.nsplit, a.H);
-    append_fused_kernel<<<grid, kAfThreads, kAfSmem, st>>>(a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kAfThreads);
+    cfg.dynamicSmemBytes = kAfSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, append_fused_kernel, a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
     if (e != cudaSuccess) return e;
   } else {
     dim3 gridA(static_cast<unsigned>(b1 - b0 + 1), a.H);
