@@ -533,6 +533,8 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsi
   __shared__ __align__(16) unsigned char scratch[kScratch];
   __shared__ TopkShared sh;
   SEL_T(0);
+  // launched as a programmatic dependent: the kernel before this one is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
@@ -815,7 +817,21 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
       if (e0 != cudaSuccess) return e0;
     }
     void* params[3] = {&aa, &ctr, &base};
-    cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(256), params, smem_keys, st);
+    // cooperative (all CTAs co-resident: they meet at two grid barriers) and a programmatic
+    // dependent of the kernel before it (its launch overlaps that kernel's tail)
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem_keys;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelExC(&cfg, fn, params);
     if (a.bar_host) {
       a.bar_host->valid = (e == cudaSuccess);
       a.bar_host->total = base + 2 * grid;
