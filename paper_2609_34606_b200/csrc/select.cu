@@ -153,18 +153,19 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   {
     // 256 / D threads per column, each summing an interleaved subset of the tile partials with
-    // up to 16 loads in flight; the subsets are then added in a fixed order
+    // up to 20 loads in flight (one round trip for a chunk of up to 40 tiles at head_dim 128); the subsets are then added in a fixed order
     constexpr int WAYS = 256 / D;
+    constexpr int kInFlight = 20;
     const int col = threadIdx.x % D, way = threadIdx.x / D;
     const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
     double s = 0.0;
-    for (int t0 = tile_lo + way; t0 < tile_hi; t0 += 16 * WAYS) {
-      float v[16];
+    for (int t0 = tile_lo + way; t0 < tile_hi; t0 += kInFlight * WAYS) {
+      float v[kInFlight];
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
+      for (int i = 0; i < kInFlight; ++i)
         v[i] = (t0 + i * WAYS < tile_hi) ? __ldcg(&a.qpart[(static_cast<size_t>(t0 + i * WAYS) * a.H + h) * D + col]) : 0.f;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) s += static_cast<double>(v[i]);
+      for (int i = 0; i < kInFlight; ++i) s += static_cast<double>(v[i]);
     }
     double* part = qs + D;  // [WAYS][D]
     part[way * D + col] = s;
