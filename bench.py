@@ -34,8 +34,8 @@ sys.path.insert(0, ROOT)
 from paper_2609_34606_b200 import workloads as W  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one hsa_forward_kernel<128, false> launch on cfg2, from
-# the ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.42 MB + 0.69 MB)
-NCU_TRAFFIC_BYTES = {"cfg2": 41.11e6}
+# the ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.43 MB + 0.77 MB)
+NCU_TRAFFIC_BYTES = {"cfg2": 41.20e6}
 METRIC = "hsa_effective_tflops"
 UNIT = "TFLOP/s"
 RING = 4  # distinct (q, k, v, out) input sets rotated between steps (> L2 in total)
@@ -164,7 +164,7 @@ def bench_ours(args, rank: int, world: int):
     budgets = W.gen_budgets(w).to(dev)
     sel = ctx.alloc_selection(w.Lq)
 
-    def step(i, ev=None, from_host=False):
+    def step(i, ev=None, from_host=False, with_forward=True):
         q, k, v, out = devs[i % RING]
         if from_host:
             hq, hk, hv, hout = host[i % RING]
@@ -183,7 +183,8 @@ def bench_ours(args, rank: int, world: int):
         ctx.select_blocks(q, budgets, sel=sel)
         if ev:
             ev[2].record()
-        ctx.forward(q, sel[0], sel[1], out=out)
+        if with_forward:
+            ctx.forward(q, sel[0], sel[1], out=out)
         if ev:
             ev[3].record()
         if from_host:
@@ -249,6 +250,12 @@ def bench_ours(args, rank: int, world: int):
             "forward": time_graph(capture(fwd(0), NK), NK),
             "linear_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_SPARSE), NK), NK),
             "sparse_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_LINEAR), NK), NK)}
+    # the forward call inside the step: a graph of the same steps without it, subtracted from the full
+    # one below (the kernel with its launch gap, behind the selection kernel and with the L2 contents
+    # a step leaves; a kernel replayed on its own sees its pages in L2 and comes out a little faster)
+    GSn = 2 * RING
+    ms_step_no_fwd = time_graph(capture(lambda i: step(i, with_forward=False), GSn), GSn)
+    ms_step_graph = time_graph(capture(step, GSn), GSn)
     step(0)  # leaves the context as a full step does
 
     # the timed loop: K steps, as replays of a graph that holds GS steps plus single-step graphs for
@@ -297,7 +304,7 @@ def bench_ours(args, rank: int, world: int):
             print(json.dumps({"profile_run": True, "launch": args.launch, "steps": K, "ms_per_step": ms_total / K,
                               "eager_ms_per_step": ms_eager,
                               "eager_stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
-                              "kernel_ms": kern}))
+                              "kernel_ms": kern, "forward_in_step_ms": ms_step_graph - ms_step_no_fwd}))
         ctx.destroy()
         return
     # end-to-end through the same API with host buffers: every step copies its inputs from pinned
@@ -389,6 +396,9 @@ def bench_ours(args, rank: int, world: int):
                          "peak_source": peaks["source"] + " (burst)",
                          "frac_of_sustained": fwd_tf / peaks["bf16_tflops_sustained"],
                          "timing": "average duration of the call replayed from CUDA graphs, CUDA events",
+                         "in_step_ms": ms_step_graph - ms_step_no_fwd,
+                         "frac_in_step": tf(fl["forward"], ms_step_graph - ms_step_no_fwd) / peaks["bf16_tflops"],
+                         "in_step_timing": "graph of 8 steps minus the same graph without the forward call, per step",
                          "append_hbm_frac": by["append"] / kern["append"] / 1e6 / peaks["hbm_gbs"],
                          "select_hbm_frac": by["select"] / kern["select"] / 1e6 / peaks["hbm_gbs"],
                          "linear_only_hbm_frac": (2 * w.Lq * w.H * w.d * 2 + w.H * w.d * w.d * 4) / ms_lin_only
