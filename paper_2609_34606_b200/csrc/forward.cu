@@ -82,6 +82,9 @@ static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory sl
 #ifndef HSA_INTERLEAVE
 #define HSA_INTERLEAVE 8
 #endif
+#ifndef HSA_L2AHEAD
+#define HSA_L2AHEAD 1
+#endif
 #ifndef HSA_PDL
 #define HSA_PDL 1
 #endif
@@ -335,6 +338,22 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               if (arms > s) mbar_wait(bar, (last / kStages) & 1, 1u << 16);
             }
           }
+        }
+      }
+    } else if (HSA_L2AHEAD && warp == 2 && attempt == 0) {
+      // ================================================================= L2 look-ahead
+      // The tiles of a (head, group) walk through the same list at about the same time.  Each of
+      // them asks a slice of the list (entries tile-in-group, + tiles-per-group, ...) into L2 when
+      // it starts, so that between them the whole list is on its way long before the rings reach it.
+      if (!SPLIT && p.k_pool != nullptr && elect_one_sync()) {  // (split tiles: measured slower with it)
+        const int n_tiles = static_cast<int>(gridDim.x);
+        const int tpg = p.group_tokens > 0 ? max(1, p.group_tokens / kTileM) : n_tiles;  // tiles per group
+        for (int e = kStages * 2 + tile % tpg; e < cnt; e += tpg) {
+          const int blk = sel[e];
+          if (blk < 0 || blk >= p.n_blocks) continue;
+          const size_t off = (static_cast<size_t>(p.page_table[blk]) * p.H + h) * (kBlock * D * 2);
+          bulk_prefetch_l2(p.k_pool + off, kBlock * D * 2);
+          bulk_prefetch_l2(p.v_pool + off, kBlock * D * 2);
         }
       }
     } else if (warp == 1) {

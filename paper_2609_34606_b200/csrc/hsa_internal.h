@@ -125,6 +125,9 @@ struct FwdParams {
   float* part_ref;       // [tiles][H][max_splits][128]
   int32_t* part_ticket;  // [tiles][H], zero between launches
   int32_t* status;
+  // L2 look-ahead of the page gather: the pools themselves (null: none)
+  const uint8_t* k_pool;
+  const uint8_t* v_pool;
 };
 
 struct CausalLinArgs {
