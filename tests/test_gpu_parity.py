@@ -587,3 +587,45 @@ def test_long_lists_split_over_ctas_and_merged(name, causal, cuda_device):
     for flags in (0, hsa.HSA_FWD_NO_LINEAR):
         d = (outs[(6, flags)].float() - outs[(0, flags)].float()).abs().max()
         assert float(d) <= 2e-2
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["mid_d128", "mid_mix"])
+def test_step_replayed_from_a_cuda_graph_is_bit_identical(name, cuda_device):
+    """append + select + forward captured in one CUDA graph (the cooperative launch and the
+    programmatic-dependent launches are ordinary graph nodes) and replayed three times give exactly
+    what the same calls give when they are issued one by one."""
+    w = W.WORKLOADS[name]
+    ctx = Hn.build_context(w, cuda_device, max_topk=max(w.n_blocks, 1))
+    Hn.append_history(ctx, w, cuda_device, n_chunks=w.n_chunks - 1)
+    k, v = (t.to(cuda_device) for t in W.gen_kv_chunk(w, w.n_chunks - 1))
+    q = W.gen_query(w).to(cuda_device)
+    budgets = W.gen_budgets(w).to(cuda_device)
+    n0 = ctx.n_tokens
+    state0, ksum0 = ctx.state.clone(), ctx.ksum.clone()
+
+    def step(sel, out):
+        ctx.state.copy_(state0)
+        ctx.ksum.copy_(ksum0)
+        ctx.rewind(n0)
+        ctx.append_kv(k, v)
+        ctx.select_blocks(q, budgets, sel=sel)
+        ctx.forward(q, sel[0], sel[1], out=out)
+
+    sel_e, out_e = ctx.alloc_selection(w.Lq), torch.zeros_like(q)
+    step(sel_e, out_e)
+    torch.cuda.synchronize()
+    state_e = ctx.state.clone()
+    sel_g, out_g = ctx.alloc_selection(w.Lq), torch.zeros_like(q)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step(sel_g, out_g)
+    for _ in range(3):
+        out_g.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        assert torch.equal(sel_g[1], sel_e[1]) and torch.equal(sel_g[0], sel_e[0])
+        assert torch.equal(out_g.view(torch.int16), out_e.view(torch.int16))
+        assert torch.equal(ctx.state, state_e)
+    assert ctx.n_tokens == n0 + w.chunk
