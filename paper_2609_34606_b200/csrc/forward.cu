@@ -6,8 +6,11 @@
 //                hi/lo halves of the linear state; also owns the TMEM allocation
 //   warp 1       tcgen05.mma issuer: S = Q K^T three steps ahead, O += P V with P read from
 //                TMEM, then the linear numerator phi(Q) S
+//   warp 2       (one lane, once) asks a slice of the group's block list into L2 ahead of the rings
 //   warps 4..11  two softmax groups of four warps: group g takes the KV steps j = g (mod 2);
 //                one query row per thread
+// The kernel is launched as a programmatic dependent of the kernel before it (block selection)
+// and waits for it on entry.
 // TMEM: O (128 fp32 columns) | three S buffers (128 columns each); P overwrites the first 64
 // columns of its S buffer as packed bf16.  With three score buffers the tensor pipe never waits
 // for a softmax group: Q K^T of step j+3 is issued right after P V of step j.
