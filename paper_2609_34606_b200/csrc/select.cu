@@ -145,13 +145,15 @@ __device__ __forceinline__ int cand_visible(const CandGeom& g, int64_t p_last) {
 // ---------------------------------------------------------------------------------------
 constexpr int kScoreBlocksPerCta = 32;
 
+// rebuild = false: qs[0, D) still holds the mean query of this (group, head) from the item before
 template <int D, bool MIXED>
-__device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs) {
+__device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs,
+                                            bool rebuild = true) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
   const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  {
+  if (rebuild) {
     // 256 / D threads per column, each summing an interleaved subset of the tile partials with
     // up to 20 loads in flight (one round trip for a chunk of up to 40 tiles at head_dim 128); the subsets are then added in a fixed order
     constexpr int WAYS = 256 / D;
@@ -549,8 +551,16 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsi
     for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x)
       scores_item_groups<D, MIXED>(a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
   } else {
-    for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x) {
-      scores_item<D, MIXED>(a, it % n_chunks, 0, it / n_chunks, reinterpret_cast<double*>(scratch));
+    // a CTA takes a run of consecutive (head, chunk) items: the mean query of a head is rebuilt
+    // from the tile partials only when the run enters the head
+    const int n_items = n_chunks * a.H;
+    const int per = (n_items + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    const int it0 = static_cast<int>(blockIdx.x) * per, it1 = min(n_items, it0 + per);
+    int h_cur = -1;
+    for (int it = it0; it < it1; ++it) {
+      const int h = it / n_chunks;
+      scores_item<D, MIXED>(a, it % n_chunks, 0, h, reinterpret_cast<double*>(scratch), h != h_cur);
+      h_cur = h;
       __syncthreads();
     }
   }
