@@ -264,6 +264,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   };
 
   if (warp < 4) {
+    // Register budget: the CTA is allocated 168 x 384 registers.  The 128 threads here give back
+    // 168 - 56 each (14336), exactly what the 256 softmax threads take to reach 224 (HSA_SMREGS);
+    // a split that asks for more than is given back would block at setmaxnreg.inc for ever.
+    static_assert(128 * (168 - 56) >= 256 * (HSA_SMREGS - 168), "setmaxnreg.inc would never be satisfied");
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
 #pragma unroll 1
     for (int attempt = 0; attempt < 2; ++attempt) {
