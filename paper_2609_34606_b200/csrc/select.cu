@@ -435,24 +435,37 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
     if (k == thr) return t++ < need_ties;
     return k > thr;
   };
+  // first walk: which of this thread's candidates are chosen (kept as a bit mask while the range
+  // has at most 32 candidates) and how many pages they hold; second walk, after the scan: emit
   int my_pages = 0;
+  uint32_t picked = 0;
+  const bool use_mask = per <= 32;
   {
     int t = ties_before;
     for (int b = lo; b < hi; ++b)
-      if (chosen(b, t)) my_pages += cand_pages<MIXED>(cg, c0 + b);
+      if (chosen(b, t)) {
+        my_pages += cand_pages<MIXED>(cg, c0 + b);
+        picked |= 1u << ((b - lo) & 31);
+      }
   }
   int total = 0;
   int pos = out_pos0 + block_exclusive_scan(my_pages, warp_sums, &total);
-  {
-    int t = ties_before;
-    for (int b = lo; b < hi; ++b) {
-      if (chosen(b, t)) {
-        const int fp = cand_first_page<MIXED>(cg, c0 + b);
-        const int np = cand_pages<MIXED>(cg, c0 + b);
-        for (int pg = 0; pg < np; ++pg, ++pos)
-          if (pos < kcap) out[pos] = fp + pg;
-      }
+  auto emit = [&](int b) {
+    const int fp = cand_first_page<MIXED>(cg, c0 + b);
+    const int np = cand_pages<MIXED>(cg, c0 + b);
+    for (int pg = 0; pg < np; ++pg, ++pos)
+      if (pos < kcap) out[pos] = fp + pg;
+  };
+  if (use_mask) {
+    while (picked) {
+      const int i = __ffs(picked) - 1;
+      picked &= picked - 1;
+      emit(lo + i);
     }
+  } else {
+    int t = ties_before;
+    for (int b = lo; b < hi; ++b)
+      if (chosen(b, t)) emit(b);
   }
   __syncthreads();  // hist / warp_sums are reused by the next call
   return total;
