@@ -152,7 +152,6 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
-  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
   if (rebuild) {
     // 256 / D threads per column, each summing an interleaved subset of the tile partials with
     // up to 20 loads in flight (one round trip for a chunk of up to 40 tiles at head_dim 128); the subsets are then added in a fixed order
@@ -422,8 +421,24 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
   // index-ordered compaction: thread t owns the contiguous range [t*per, t*per+per)
   const int per = (n + 255) / 256;
   const int lo = min(n, static_cast<int>(threadIdx.x) * per), hi = min(n, lo + per);
+  const bool use_mask = per <= 32;  // the thread's range fits a 32-bit mask: ONE walk over the keys
   int ties_before = 0, dummy;
-  if (!take_all && budget > 0) {
+  uint32_t gt = 0, eq = 0;  // candidates above the threshold / equal to it, as bits of the range
+  if (use_mask) {
+    for (int b = lo; b < hi; ++b) {
+      const uint32_t k = keys[b];
+      const uint32_t bit = 1u << (b - lo);
+      if (take_all) {
+        if (!(MIXED && masked) || k != 0u) gt |= bit;
+      } else if (budget > 0) {
+        if (k > thr)
+          gt |= bit;
+        else if (k == thr)
+          eq |= bit;
+      }
+    }
+    if (!take_all && budget > 0) ties_before = block_exclusive_scan(__popc(eq), warp_sums, &dummy);
+  } else if (!take_all && budget > 0) {
     int my_ties = 0;
     for (int b = lo; b < hi; ++b) my_ties += (keys[b] == thr);
     ties_before = block_exclusive_scan(my_ties, warp_sums, &dummy);
@@ -435,18 +450,28 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
     if (k == thr) return t++ < need_ties;
     return k > thr;
   };
-  // first walk: which of this thread's candidates are chosen (kept as a bit mask while the range
-  // has at most 32 candidates) and how many pages they hold; second walk, after the scan: emit
+  // which of this thread's candidates are chosen and how many pages they hold; after the scan: emit
   int my_pages = 0;
   uint32_t picked = 0;
-  const bool use_mask = per <= 32;
-  {
+  if (use_mask) {
+    // ties at the threshold go to the lowest indices: this thread's ties rank ties_before, + 1, ...
+    int allow = need_ties - ties_before;
+    uint32_t e = eq;
+    while (allow > 0 && e) {
+      picked |= e & (0u - e);
+      e &= e - 1;
+      --allow;
+    }
+    picked |= gt;
+    if (!MIXED) {
+      my_pages = __popc(picked);
+    } else {
+      for (uint32_t m = picked; m; m &= m - 1) my_pages += cand_pages<MIXED>(cg, c0 + lo + __ffs(m) - 1);
+    }
+  } else {
     int t = ties_before;
     for (int b = lo; b < hi; ++b)
-      if (chosen(b, t)) {
-        my_pages += cand_pages<MIXED>(cg, c0 + b);
-        picked |= 1u << ((b - lo) & 31);
-      }
+      if (chosen(b, t)) my_pages += cand_pages<MIXED>(cg, c0 + b);
   }
   int total = 0;
   int pos = out_pos0 + block_exclusive_scan(my_pages, warp_sums, &total);
