@@ -365,6 +365,7 @@ struct TopkShared {
   int warp_sums[8];
   uint32_t prefix;
   int krem;
+  int exact;  // radix select: the bin just chosen holds exactly the keys still to take
 };
 
 // The `budget` largest keys of keys[0, n) (ties at the threshold to the lower index), emitted in
@@ -408,11 +409,15 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
       if (above < krem && above + mine >= krem) {                     // exactly one thread
         sh->prefix = prefix | (static_cast<uint32_t>(bin) << shift);
         sh->krem = krem - above;  // still to take among keys matching the longer prefix
+        sh->exact = (above + mine == krem);
       }
       __syncthreads();
       prefix = sh->prefix;
       krem = sh->krem;
       mask |= 255u << shift;
+      // every key of the chosen bin is wanted: the prefix with zero low bits is a threshold that
+      // all of them reach, and krem (their number) covers the ones that equal it exactly
+      if (sh->exact) break;
     }
     thr = prefix;
     need_ties = krem;
