@@ -629,3 +629,42 @@ def test_step_replayed_from_a_cuda_graph_is_bit_identical(name, cuda_device):
         assert torch.equal(out_g.view(torch.int16), out_e.view(torch.int16))
         assert torch.equal(ctx.state, state_e)
     assert ctx.n_tokens == n0 + w.chunk
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_rep,budget", [(40, 7), (300, 129), (600, 1), (600, 599)])
+def test_selection_exact_ties_go_to_the_lower_block_index(n_rep, budget, cuda_device):
+    """A history made of one 64-token block repeated n_rep times, followed by one distinct block:
+    the repeated blocks have bit-identical pooled scores, so the budget cuts through a group of exact
+    ties, which must go to the lower block indices (in every thread's range of the compaction, with
+    one key per thread and with several).  Checked against the oracle's selection as well."""
+    from paper_2609_34606_b200 import hsa
+    H, d = 2, 128
+    gen = torch.Generator().manual_seed(1234 + n_rep)
+    blk_k = torch.randn(64, H, d, generator=gen).to(torch.bfloat16)
+    blk_v = torch.randn(64, H, d, generator=gen).to(torch.bfloat16)
+    last_k = (torch.randn(64, H, d, generator=gen) * 3).to(torch.bfloat16)
+    last_v = torch.randn(64, H, d, generator=gen).to(torch.bfloat16)
+    K = torch.cat([blk_k.repeat(n_rep, 1, 1), last_k], 0)
+    V = torch.cat([blk_v.repeat(n_rep, 1, 1), last_v], 0)
+    n_blocks = n_rep + 1
+    step = 64 * 50  # tokens per append
+    ctx = hsa.HSAContext(H, d, max_pages=n_blocks, max_q_tokens=step, max_topk=n_blocks, device=cuda_device)
+    for t0 in range(0, K.shape[0], step):
+        ctx.append_kv(K[t0:t0 + step].to(cuda_device), V[t0:t0 + step].to(cuda_device))
+    q = torch.randn(200, H, d, generator=gen).to(torch.bfloat16)
+    budgets = torch.tensor([budget, budget + 1], dtype=torch.int32)
+    si, sc = ctx.select_blocks(q.to(cuda_device), budgets.to(cuda_device))
+    assert ctx.device_status() == 0
+    got = Hn.selection_lists(si, sc)
+    ref, scores = O.select_blocks(Hn.f64(q), Hn.f64(K), K.shape[0], False, budgets.numpy())
+    for h in range(H):
+        b = int(budgets[h])
+        s = scores[h, 0]
+        assert np.all(s[:n_rep] == s[0]), "the repeated blocks must tie exactly in the oracle too"
+        # the distinct block either beats the ties or not; the rest of the budget is the lowest indices
+        want = [n_rep] if s[n_rep] > s[0] else []
+        want = sorted(list(range(b - len(want))) + want)
+        assert got[h][0].tolist() == want
+        assert ref[h][0].tolist() == want
+    ctx.destroy()
