@@ -16,8 +16,8 @@
 // for a softmax group: Q K^T of step j+3 is issued right after P V of step j.
 //
 // Both groups accumulate into ONE O.  That needs a common exponent reference per row, so in the
-// normal ("fast") pass the reference is fixed once: the row maximum of the first step plus a
-// headroom of 2^20.  Every later weight is exp2(s - ref) with no running maximum and no rescale.
+// normal ("fast") pass the reference is fixed once: the row maximum over the first 32 keys of the
+// first step (all of its keys when the step is masked) plus a headroom of 2^20.  Every later weight is exp2(s - ref) with no running maximum and no rescale.
 // fp32 / bf16 carry the same relative precision at any magnitude, so the result equals the
 // usual online softmax as long as no weight overflows; a step whose weights exceed 2^27 sets a
 // flag and the tile is redone in a "safe" pass: one group, classic online softmax with lazy
@@ -556,12 +556,15 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (safe || j == 0) {
           // the reference needs the row maximum first: a pass over the score row in chunks
           float mxa = -INFINITY, mxb = -INFINITY;
+          // (the fixed reference of the fast pass only has to be near the row maximum: an unmasked
+          // first step takes it from its first 32 columns)
+          const int nmax = (safe || need_mask) ? nchunks : 1;
           tmem_ld32(s_tmem, cbuf[0]);
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            if (c < nchunks) {
+            if (c < nmax) {
               tc_wait_ld();
-              if (c + 1 < nchunks) tmem_ld32(s_tmem + 32 * (c + 1), cbuf[(c + 1) & 1]);
+              if (c + 1 < nmax) tmem_ld32(s_tmem + 32 * (c + 1), cbuf[(c + 1) & 1]);
               uint32_t(&x)[32] = cbuf[c & 1];
               if (need_mask) {
                 const int lim = ((c >> 1) ? lim1 : lim0) - (c & 1) * 32;
