@@ -305,9 +305,11 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
 
   // the reduction kernel behind this one may be scheduled early; it waits for this grid itself
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // this grid is itself launched as a programmatic dependent: whatever ran before it in the stream
-  // (the forward kernel of the layer before, a copy) is complete from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // This grid is itself launched as a programmatic dependent: it may be scheduled while the kernel
+  // before it in the stream (the forward kernel of the layer before) is still finishing.  The
+  // set-up below touches nothing of that kernel's; every thread waits for its end (wait_prior)
+  // before the first load of the inputs is issued and before the CTA-wide barrier.
+  auto wait_prior = [] { asm volatile("griddepcontrol.wait;" ::: "memory"); };
 
   const int h = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -340,6 +342,7 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
     }
     bars->abort_flag = 0;
     fence_mbar_init();
+    wait_prior();
     // the first ring fill starts before the rest of the CTA is set up
     for (int bi = 0; bi < nblk && bi < kAfDepth; ++bi) issue_loads(bi);
     tma_prefetch_desc(&tm_kpool);
@@ -352,6 +355,7 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
   // bf16 1.0 everywhere: under any swizzle the tile reads as all ones
   for (int i = threadIdx.x; i < kAfOnes / 4; i += kAfThreads) reinterpret_cast<uint32_t*>(ones)[i] = 0x3F803F80u;
   fence_proxy_async_smem();
+  wait_prior();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();

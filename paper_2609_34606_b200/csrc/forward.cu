@@ -199,9 +199,26 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp == 4) HSA_T(3000);
+  // barriers, TMEM allocation and the CTA-wide barrier that publishes them
+  auto setup = [&]() {
+    if (threadIdx.x == 0) {
+      bars->abort_flag = 0;
+      init_barriers(bars);
+    }
+    if (warp == 0) {
+      tmem_alloc(&bars->tmem_base, kTmemCols);
+      tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  };
+  // Launched with programmatic stream serialization: this grid may be scheduled while the kernel
+  // before it (block selection) is still extracting its lists.  Nothing of that kernel's output is
+  // read before the wait; the plain kernel does its set-up first, under that kernel's tail (a split
+  // CTA may still leave without any set-up, so it sets up after it has seen its list).
+  if (!SPLIT) setup();
 #if HSA_PDL
-  // launched with programmatic stream serialization: this grid may be scheduled while the kernel
-  // before it (block selection) is still draining; nothing of that kernel's output is read above
   asm volatile("griddepcontrol.wait;" ::: "memory");
 #endif
   const int tile = blockIdx.x, h = blockIdx.y;
@@ -231,17 +248,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   const int slot = (tile * p.H + h) * static_cast<int>(gridDim.z) + part;  // this CTA's partial-result slot
   const int nsteps = (cnt + 1) / 2;
 
-  if (threadIdx.x == 0) {
-    bars->abort_flag = 0;
-    init_barriers(bars);
-  }
-  if (warp == 0) {
-    tmem_alloc(&bars->tmem_base, kTmemCols);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
+  if (SPLIT) setup();
   const uint32_t tmem = bars->tmem_base;
   if (warp == 4) HSA_T(3001);
 

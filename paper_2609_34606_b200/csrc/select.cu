@@ -610,6 +610,10 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsi
   SEL_T(3);
   grid_barrier(bar_ctr, bar_base + 2 * gridDim.x, a.status);
   SEL_T(4);
+  // Only a few CTAs have a list to extract; the others leave now.  The kernel behind this one
+  // (launched as a programmatic dependent, it waits for this grid's end before it reads a list)
+  // may take their places and do its set-up meanwhile.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
     topk_item<MIXED>(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
     __syncthreads();
