@@ -227,7 +227,11 @@ int hsa_select_blocks_adaptive(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t
  * process exits.
  *   ksum_dev                  device fp32 [H][ksum_head_stride_blocks][d]: per-(head, block) key
  *                             sums as hsa_append_kv maintains them (see hsa_state_layout)
- *   status_dev                device int32 status word, or NULL to use one inside the scratch
+ *   status_dev                device int32 status word (zeroed by the caller) that receives
+ *                             HSA_ERR_DEVICE_BOUNDS when a list had to be cut at max_topk; with NULL
+ *                             the flag goes to a word inside the scratch that no entry point reads,
+ *                             i.e. a cut list is then not reported: pass a word when max_topk may
+ *                             be smaller than a budget
  * Limits (HSA_ERR_OUT_OF_PAGES beyond them): ceil(n_q/128) * H * d <= 131072,
  * H * ksum_head_stride_blocks <= 131072, ceil(n_tokens/64) <= 51200.
  * It calls no allocator (no cudaMalloc / cudaFree, no library routine that allocates).  The first
@@ -273,8 +277,21 @@ int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens);
  * S fp32 [H][d][d], z fp32 [H][d], key sums fp32 [H][max_pages][d]. */
 int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksum);
 
-/* Synchronises the device, reads and clears the status word: HSA_OK or a DEVICE_* code. */
+/* Synchronises the device, reads and clears the status word: HSA_OK or a DEVICE_* code.
+ * After HSA_ERR_DEVICE_TIMEOUT the selection written by the call that timed out has every count
+ * set to zero (a forward call on it computes the linear branch alone), and this call also puts
+ * the selection kernel's grid barrier back to its initial state, so the next call starts clean. */
 int hsa_device_status(hsa_ctx* ctx, int32_t* status_out);
+
+/* Bound, in nanoseconds, of a wait at the grid barrier of the selection kernel (the one place
+ * where CTAs wait for each other; default 2e9).  When it runs out the kernel ends, the status word
+ * holds HSA_ERR_DEVICE_TIMEOUT and the call's selection is empty.  wait_ns > 0. */
+int hsa_set_wait_limit_ns(hsa_ctx* ctx, uint64_t wait_ns);
+
+/* Byte offsets inside the workspace, for tests and monitoring: the int32 status word, and the
+ * two uint32 words {arrive count, generation} of the selection kernel's grid barrier (both are
+ * zero whenever no selection kernel is running). */
+int hsa_workspace_layout(hsa_ctx* ctx, size_t* off_status, size_t* off_barrier);
 
 /* Synchronises the device, reads and clears a counter: the number of (query tile, head) work
  * items since the last read whose softmax had to be redone with a running maximum because a

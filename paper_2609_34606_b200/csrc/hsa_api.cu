@@ -124,7 +124,7 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 }  // namespace
 
 struct hsa_ctx {
-  hsa::GridBarrierHost select_bar;  // running total of the selection kernel's grid-barrier counter
+  unsigned long long wait_ns;  // bound of the selection kernel's grid-barrier waits
   hsa_config cfg;
   hsa_buffers buf;
   Layout lay;
@@ -232,6 +232,7 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   ctx->last_append = 0;
   ctx->last_cuda_error = 0;
   ctx->n_segs = 0;
+  ctx->wait_ns = 2000000000ull;
   ctx->page_table_host = pt;
   ctx->resident.assign(static_cast<size_t>(cfg->max_pages), 1);
   const bool linformer = cfg->lin_mode == HSA_LIN_LINFORMER;
@@ -415,7 +416,7 @@ int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_s
   a.kcap = ctx->cfg.max_topk;
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   a.barrier = reinterpret_cast<unsigned*>(ws + ctx->lay.status + 8);
-  a.bar_host = &ctx->select_bar;
+  a.wait_ns = ctx->wait_ns;
   if (opts) {
     a.inter_pages = opts->inter_block_pages;
     a.intra_first_page1 = opts->intra_first_page >= 0 ? static_cast<int64_t>(opts->intra_first_page) + 1 : 0;
@@ -738,6 +739,19 @@ int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksu
   return HSA_OK;
 }
 
+int hsa_workspace_layout(hsa_ctx* ctx, size_t* off_status, size_t* off_barrier) {
+  if (!ctx) return HSA_ERR_INVALID_ARG;
+  if (off_status) *off_status = ctx->lay.status;
+  if (off_barrier) *off_barrier = ctx->lay.status + 8;
+  return HSA_OK;
+}
+
+int hsa_set_wait_limit_ns(hsa_ctx* ctx, uint64_t wait_ns) {
+  if (!ctx || wait_ns == 0) return HSA_ERR_INVALID_ARG;
+  ctx->wait_ns = wait_ns;
+  return HSA_OK;
+}
+
 int hsa_device_status(hsa_ctx* ctx, int32_t* status_out) {
   if (!ctx || !status_out) return HSA_ERR_INVALID_ARG;
   cudaError_t e = cudaDeviceSynchronize();
@@ -746,6 +760,8 @@ int hsa_device_status(hsa_ctx* ctx, int32_t* status_out) {
   int32_t v = 0;
   e = cudaMemcpy(&v, ws + ctx->lay.status, 4, cudaMemcpyDeviceToHost);
   if (e == cudaSuccess && v != 0) e = cudaMemset(ws + ctx->lay.status, 0, 4);
+  // a grid barrier that ran out leaves its arrive count behind: both of its words start over
+  if (e == cudaSuccess && v == HSA_ERR_DEVICE_TIMEOUT) e = cudaMemset(ws + ctx->lay.status + 8, 0, 8);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   *status_out = v;
   return HSA_OK;

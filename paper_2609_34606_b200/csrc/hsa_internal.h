@@ -42,12 +42,6 @@ struct AppendArgs {
   int32_t* status;  // device status word
 };
 
-// Host-side view of a grid-barrier arrive counter that is never cleared between launches.
-struct GridBarrierHost {
-  unsigned total = 0;  // value the device counter reaches once every launch so far has finished
-  bool valid = false;  // false: the device counter has to be cleared before the next launch
-};
-
 struct SelectArgs {
   const __nv_bfloat16* q;
   int n_q;
@@ -66,8 +60,9 @@ struct SelectArgs {
   int32_t* sel_cnt;
   int kcap;
   int32_t* status;
-  unsigned* barrier;  // grid-barrier arrive counter for the single-launch path (null: three launches)
-  GridBarrierHost* bar_host;  // host-side running total of that counter (null: cleared per launch)
+  unsigned* barrier;  // grid barrier of the single-launch path: {arrive count, generation}, both zero
+                      // when no launch is in flight (null: three launches)
+  unsigned long long wait_ns;  // bound of a wait at that barrier
   // candidate geometry: pages before the first intra-chunk page are selected in runs of inter_pages pages against
   // budgets[], the pages from it on one by one against intra_budgets[] (null: all of them)
   int inter_pages;           // 0 or 1: every page on its own

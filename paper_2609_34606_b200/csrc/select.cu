@@ -226,21 +226,6 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   }
 }
 
-#ifdef HSA_TIMING
-__device__ long long g_sel_timing[64];
-#define SEL_T(slot)                                              \
-  do {                                                           \
-    if (blockIdx.x == 0 && threadIdx.x == 0) {                   \
-      long long t_;                                              \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));      \
-      g_sel_timing[(slot)] = t_;                                 \
-    }                                                            \
-  } while (0)
-#else
-#define SEL_T(slot) \
-  do {              \
-  } while (0)
-#endif
 
 // Many query groups (per-query-tile selection): the scores of one head are a small matrix product
 //   scores[g][c] = sum_e qbar[g][e] * ksum[c][e]
@@ -538,58 +523,80 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------
-// The three stages in ONE cooperative launch (one CTA per SM, all co-resident): query tile sums,
-// grid barrier, scores, grid barrier, top-k.  Saves two launches and their drain / ramp-up.
-// The barrier is an arrive counter in global memory (cleared by the host before the launch)
-// that one thread per CTA polls with a time bound; on expiry the CTA records a timeout in the
-// status word and carries on, so the kernel always terminates.
+// The three stages in ONE cooperative launch (all CTAs co-resident): query tile sums, grid
+// barrier, scores, grid barrier, top-k.  Saves two launches and their drain / ramp-up.
+//
+// The grid barrier lives entirely on the device: two words in the workspace, an arrive count and
+// a generation.  A CTA reads the generation, arrives, and waits for the generation to change; the
+// last CTA to arrive puts the count back to zero and advances the generation.  Nothing depends on
+// host-side bookkeeping, so a launch captured in a CUDA graph behaves the same on every replay,
+// in any order with other launches.  The wait is bounded (wait_ns): on expiry the CTA records a
+// timeout in the status word and the kernel ends with every list of the call counted as empty.
+// The host clears the two words when it reads that status (hsa_device_status).
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void grid_barrier(unsigned* ctr, unsigned target, int32_t* status) {
+__device__ __forceinline__ bool grid_barrier(unsigned* bar, int32_t* status, unsigned long long wait_ns) {
+  __shared__ int bar_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
+    int ok = 1;
+    unsigned gen;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(bar + 1) : "memory");
     __threadfence();
-    atomicAdd(ctr, 1u);
-    unsigned long long t0 = 0;
-    for (unsigned i = 0;; ++i) {
-      unsigned v;
-      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-      if (static_cast<int32_t>(v - target) >= 0) break;  // the counter only grows; wrap-safe
-      if ((i & 63u) == 63u) {
-        unsigned long long now;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-        if (t0 == 0) t0 = now;
-        if (now - t0 > 2000000000ull) {
-          atomicCAS(status, 0, kDevTimeout);
-          break;
+    const unsigned arrived = atomicAdd(bar, 1u);
+    if (arrived == gridDim.x - 1) {
+      bar[0] = 0u;  // ordered before the new generation by the release below
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(bar + 1), "r"(gen + 1u) : "memory");
+    } else {
+      unsigned long long t0 = 0;
+      for (unsigned i = 0;; ++i) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar + 1) : "memory");
+        if (v != gen) break;
+        if ((i & 63u) == 63u) {
+          unsigned long long now;
+          asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+          if (t0 == 0) t0 = now;
+          // another CTA gave up already, or this one has waited long enough
+          if (*reinterpret_cast<volatile int32_t*>(status) == kDevTimeout || now - t0 > wait_ns) {
+            atomicCAS(status, 0, kDevTimeout);
+            ok = 0;
+            break;
+          }
         }
       }
     }
     __threadfence();
+    bar_ok = ok;
   }
   __syncthreads();
+  return bar_ok != 0;
 }
 
-
 template <int D, bool MIXED>
-__global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsigned* bar_ctr, unsigned bar_base) {
+__global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   extern __shared__ uint32_t fused_keys[];
   // tile-sum partials / mean query / (many groups) a batch of mean queries
   constexpr int kGroupBytes = kGroupBatch * (D + 4) * 8;
   constexpr int kScratch = kGroupBytes > 256 / (D / 8) * D * 4 ? kGroupBytes : 256 / (D / 8) * D * 4;
   __shared__ __align__(16) unsigned char scratch[kScratch];
   __shared__ TopkShared sh;
-  SEL_T(0);
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
+  // a barrier that ran out: no list of this call can be trusted, every one is counted as empty
+  auto give_up = [&]() {
+    for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x)
+      if (threadIdx.x == 0) a.sel_cnt[it] = 0;  // it = h * n_groups + g
+  };
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
     qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
   }
-  SEL_T(1);
-  grid_barrier(bar_ctr, bar_base + gridDim.x, a.status);
-  SEL_T(2);
+  if (!grid_barrier(a.barrier, a.status, a.wait_ns)) {
+    give_up();
+    return;
+  }
   if (a.n_groups > 1) {
     for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x)
       scores_item_groups<D, MIXED>(a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
@@ -607,9 +614,10 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsi
       __syncthreads();
     }
   }
-  SEL_T(3);
-  grid_barrier(bar_ctr, bar_base + 2 * gridDim.x, a.status);
-  SEL_T(4);
+  if (!grid_barrier(a.barrier, a.status, a.wait_ns)) {
+    give_up();
+    return;
+  }
   // Only a few CTAs have a list to extract; the others leave now.  The kernel behind this one
   // (launched as a programmatic dependent, it waits for this grid's end before it reads a list)
   // may take their places and do its set-up meanwhile.
@@ -617,8 +625,7 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a, unsi
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
     topk_item<MIXED>(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
     __syncthreads();
-    SEL_T(5);
-}
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -822,13 +829,6 @@ bool coop_info(int* nsm) {
 }
 }  // namespace
 
-#ifdef HSA_TIMING
-}  // namespace hsa
-extern "C" int hsa_debug_read_sel_timing(long long* host_out, int n) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, hsa::g_sel_timing, sizeof(long long) * n));
-}
-namespace hsa {
-#endif
 
 cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st) {
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
@@ -848,7 +848,6 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
     const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;
     const size_t smem_keys = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
     SelectArgs aa = a;
-    unsigned* ctr = a.barrier;
     const void* fn = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(select_fused_kernel<128, true>)
                                          : reinterpret_cast<const void*>(select_fused_kernel<128, false>))
                                 : (mixed ? reinterpret_cast<const void*>(select_fused_kernel<64, true>)
@@ -864,17 +863,7 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
       per_sm = occ < 3 ? occ : 3;
     }
     const unsigned grid = static_cast<unsigned>(nsm * per_sm);
-    // The arrive counter only grows: each launch adds 2 * grid to it, and the host keeps the
-    // running total so that no clearing launch is needed.  Without a host total (or after a
-    // failed launch) the counter is cleared on the stream first.
-    unsigned base = 0;
-    if (a.bar_host && a.bar_host->valid) {
-      base = a.bar_host->total;
-    } else {
-      cudaError_t e0 = cudaMemsetAsync(a.barrier, 0, sizeof(unsigned), st);
-      if (e0 != cudaSuccess) return e0;
-    }
-    void* params[3] = {&aa, &ctr, &base};
+    void* params[1] = {&aa};
     // cooperative (all CTAs co-resident: they meet at two grid barriers) and a programmatic
     // dependent of the kernel before it (its launch overlaps that kernel's tail)
     cudaLaunchConfig_t cfg{};
@@ -889,12 +878,7 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelExC(&cfg, fn, params);
-    if (a.bar_host) {
-      a.bar_host->valid = (e == cudaSuccess);
-      a.bar_host->total = base + 2 * grid;
-    }
-    return e;
+    return cudaLaunchKernelExC(&cfg, fn, params);
   }
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   dim3 g1(n_tiles, a.H);

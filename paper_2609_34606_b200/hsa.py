@@ -41,7 +41,8 @@ EXPORTS = [
     "hsa_block_resident",
     "hsa_select_blocks_noalloc",
     "hsa_forward",
-    "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_device_status", "hsa_safe_pass_tiles",
+    "hsa_get_info", "hsa_rewind", "hsa_state_layout", "hsa_workspace_layout", "hsa_set_wait_limit_ns",
+    "hsa_device_status", "hsa_safe_pass_tiles",
     "hsa_last_cuda_error",
     "hsa_destroy", "hsa_status_string",
 ]
@@ -99,6 +100,8 @@ def _load() -> C.CDLL:
     lib.hsa_rewind.argtypes = [vp, i64]
     lib.hsa_state_layout.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t),
                                      C.POINTER(C.c_size_t)]
+    lib.hsa_workspace_layout.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    lib.hsa_set_wait_limit_ns.argtypes = [vp, C.c_uint64]
     lib.hsa_device_status.argtypes = [vp, C.POINTER(i32)]
     lib.hsa_safe_pass_tiles.argtypes = [vp, C.POINTER(i64)]
     lib.hsa_last_cuda_error.argtypes = [vp]
@@ -277,6 +280,16 @@ def hsa_state_layout(ctx: int) -> Tuple[int, int, int]:
     return a.value, b.value, c.value
 
 
+def hsa_workspace_layout(ctx: int) -> Tuple[int, int]:
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(_lib.hsa_workspace_layout(ctx, C.byref(a), C.byref(b)), "hsa_workspace_layout")
+    return a.value, b.value
+
+
+def hsa_set_wait_limit_ns(ctx: int, wait_ns: int) -> None:
+    _check(_lib.hsa_set_wait_limit_ns(ctx, int(wait_ns)), "hsa_set_wait_limit_ns")
+
+
 def hsa_device_status(ctx: int) -> int:
     s = C.c_int32()
     _check(_lib.hsa_device_status(ctx, C.byref(s)), "hsa_device_status")
@@ -431,6 +444,14 @@ class HSAContext:
 
     def device_status(self) -> int:
         return hsa_device_status(self.ctx)
+
+    def set_wait_limit_ns(self, wait_ns: int) -> None:
+        hsa_set_wait_limit_ns(self.ctx, wait_ns)
+
+    def barrier_words(self) -> torch.Tensor:
+        """uint32-as-int32 view [2] of the selection kernel's grid barrier {arrive count, generation}."""
+        off = hsa_workspace_layout(self.ctx)[1]
+        return self.workspace[off:off + 8].view(torch.int32)
 
     def safe_pass_tiles(self) -> int:
         return hsa_safe_pass_tiles(self.ctx)

@@ -591,44 +591,112 @@ def test_long_lists_split_over_ctas_and_merged(name, causal, cuda_device):
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("name", ["mid_d128", "mid_mix"])
-def test_step_replayed_from_a_cuda_graph_is_bit_identical(name, cuda_device):
-    """append + select + forward captured in one CUDA graph (the cooperative launch and the
-    programmatic-dependent launches are ordinary graph nodes) and replayed three times give exactly
-    what the same calls give when they are issued one by one."""
+def test_steps_replayed_from_cuda_graphs_are_bit_identical(name, cuda_device):
+    """append + select + forward captured in CUDA graphs (the cooperative launch and the
+    programmatic-dependent launches are ordinary graph nodes) give exactly what the same calls give
+    issued one by one -- with a different query chunk in the captured buffer at every replay (so a
+    stage of the selection kernel that ran ahead of its grid barrier would read the previous
+    replay's sums), two graphs captured one after the other and replayed out of capture order, two
+    selection calls per graph, and eager calls in between."""
     w = W.WORKLOADS[name]
     ctx = Hn.build_context(w, cuda_device, max_topk=max(w.n_blocks, 1))
     Hn.append_history(ctx, w, cuda_device, n_chunks=w.n_chunks - 1)
     k, v = (t.to(cuda_device) for t in W.gen_kv_chunk(w, w.n_chunks - 1))
-    q = W.gen_query(w).to(cuda_device)
+    qs = [W.gen_query(w, step=i).to(cuda_device) for i in range(4)]
     budgets = W.gen_budgets(w).to(cuda_device)
     n0 = ctx.n_tokens
     state0, ksum0 = ctx.state.clone(), ctx.ksum.clone()
 
-    def step(sel, out):
+    def step(q, sel, out, scratch_sel):
         ctx.state.copy_(state0)
         ctx.ksum.copy_(ksum0)
         ctx.rewind(n0)
         ctx.append_kv(k, v)
-        ctx.select_blocks(q, budgets, sel=sel)
+        ctx.select_blocks(out, budgets, sel=scratch_sel)   # a selection on other data first: its sums
+        ctx.select_blocks(q, budgets, sel=sel)              # and keys are what a missed barrier would reuse
         ctx.forward(q, sel[0], sel[1], out=out)
 
-    sel_e, out_e = ctx.alloc_selection(w.Lq), torch.zeros_like(q)
-    step(sel_e, out_e)
-    torch.cuda.synchronize()
-    state_e = ctx.state.clone()
-    sel_g, out_g = ctx.alloc_selection(w.Lq), torch.zeros_like(q)
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g):
-        step(sel_g, out_g)
-    for _ in range(3):
-        out_g.fill_(float("nan"))
+    def eager(q):
+        sel, out = ctx.alloc_selection(w.Lq), torch.zeros_like(q)
+        step(q, sel, out, ctx.alloc_selection(w.Lq))
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        return sel[0].clone(), sel[1].clone(), out.clone()
+
+    refs = [eager(q) for q in qs]
+    graphs = []
+    for _ in range(2):
+        qb = torch.zeros_like(qs[0])
+        sel_g, out_g, scr = ctx.alloc_selection(w.Lq), torch.zeros_like(qb), ctx.alloc_selection(w.Lq)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step(qb, sel_g, out_g, scr)
+        graphs.append((g, qb, sel_g, out_g))
+    # a call issued directly after captures that have not been replayed yet
+    e = eager(qs[1])
+    assert torch.equal(e[2].view(torch.int16), refs[1][2].view(torch.int16)) and torch.equal(e[1], refs[1][1])
+
+    def check(got_sel, got_out, ref):
+        assert torch.equal(got_sel[1], ref[1])
+        for h in range(w.H):
+            n = int(ref[1][h, 0])
+            assert torch.equal(got_sel[0][h, 0, :n], ref[0][h, 0, :n]), h
+        assert torch.equal(got_out.view(torch.int16), ref[2].view(torch.int16))
+
+    for gi, qi in [(1, 0), (0, 1), (0, 2), (1, 3), (1, 1), (0, 0), (1, 2)]:
+        g, qb, sel_g, out_g = graphs[gi]
+        qb.copy_(qs[qi])
+        out_g.copy_(qs[(qi + 1) % 4])        # the first selection of the graph scores this tensor
+        sel_g[1].fill_(-1)
         g.replay()
         torch.cuda.synchronize()
         assert ctx.device_status() == 0
-        assert torch.equal(sel_g[1], sel_e[1]) and torch.equal(sel_g[0], sel_e[0])
-        assert torch.equal(out_g.view(torch.int16), out_e.view(torch.int16))
-        assert torch.equal(ctx.state, state_e)
+        check(sel_g, out_g, refs[qi])
+        if gi == 0 and qi == 2:              # an eager step between replays
+            e = eager(qs[3])
+            check((e[0], e[1]), e[2], refs[3])
     assert ctx.n_tokens == n0 + w.chunk
+    ctx.destroy()
+
+
+@pytest.mark.gpu
+def test_grid_barrier_wait_that_runs_out_is_reported_and_leaves_the_context_usable(cuda_device):
+    """The one place where CTAs wait for each other is the grid barrier of the selection kernel.
+    Its wait is bounded: with the bound set to a few milliseconds and the barrier's arrive count
+    put where the last arrival can never be seen, the kernel must end by itself, report
+    HSA_ERR_DEVICE_TIMEOUT, leave every list of the call empty (a forward call on it is the linear
+    branch alone), and the next call must be clean."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["mid_d128"]
+    ctx = Hn.build_context(w, cuda_device)
+    Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w).to(cuda_device)
+    budgets = W.gen_budgets(w).to(cuda_device)
+    ref_idx, ref_cnt = ctx.select_blocks(q, budgets)
+    assert ctx.device_status() == 0 and int(ref_cnt.sum()) > 0
+    words = ctx.barrier_words()
+    assert words.tolist() == [0, 0]
+    ctx.set_wait_limit_ns(5_000_000)
+    words[0] = 0x40000000                      # no arrival will ever be the last one
+    idx, cnt = ctx.alloc_selection(w.Lq)
+    cnt.fill_(7)
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    ctx.select_blocks(q, budgets, sel=(idx, cnt))
+    t1.record()
+    torch.cuda.synchronize()
+    assert t0.elapsed_time(t1) < 1000.0        # milliseconds: the wait gave up at its bound
+    assert int(cnt.abs().sum()) == 0
+    out = ctx.forward(q, idx, cnt)
+    lin = ctx.forward(q, idx, cnt, flags=hsa.HSA_FWD_NO_SPARSE)
+    assert torch.equal(out, lin)
+    assert ctx.device_status() == hsa.HSA_ERR_DEVICE_TIMEOUT
+    assert ctx.barrier_words().tolist() == [0, 0] and ctx.device_status() == 0
+    idx2, cnt2 = ctx.select_blocks(q, budgets)
+    assert ctx.device_status() == 0
+    assert torch.equal(cnt2, ref_cnt) and torch.equal(idx2, ref_idx)
+    ctx.destroy()
 
 
 @pytest.mark.gpu
