@@ -82,6 +82,8 @@ WORKLOADS = {
     "mid_causal": Workload("mid_causal", H=2, d=128, Lq=300, chunk=300, n_chunks=5, topk=6,
                            seed=14, causal=True, q_inside=True),
     "mid_linformer": Workload("mid_linformer", H=3, d=128, Lq=300, chunk=328, n_chunks=4, topk=6, seed=16),
+    # the layer's own sizes with three history chunks: Linformer segments of one chunk each
+    "cfg2_linformer": Workload("cfg2_linformer", H=12, d=128, Lq=4680, chunk=4680, n_chunks=3, topk=64, seed=17),
     "mid_shuffle": Workload("mid_shuffle", H=2, d=128, Lq=260, chunk=260, n_chunks=9, topk=12,
                             seed=15, shuffle_pages=True),
 }

@@ -223,6 +223,70 @@ def test_full_size_sampled_parity(name, cuda_device):
     ctx.destroy()
 
 
+def test_full_size_per_tile_selection_sampled(cuda_device):
+    """cfg2 with one selection per 128-row query tile (37 groups x 12 heads, the granularity the
+    sparse branch is defined at): every list against the oracle, outputs on sampled rows."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["cfg2"]
+    gt = 128
+    ctx = Hn.build_context(w, cuda_device, max_topk=w.topk)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    budgets = W.gen_budgets(w)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    si, sc = ctx.select_blocks(qd, budgets.to(cuda_device), group_tokens=gt)
+    assert tuple(sc.shape) == (w.H, 37)
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, scores = O.select_blocks(qn, Kn, w.q_pos0, False, budgets.tolist(), gt)
+    Hn.check_selection(sel_gpu, sel_ref, scores)
+    assert len({tuple(x) for x in sel_gpu[0]}) > 1, "the groups of a head must not all pick the same blocks"
+    rows = W.sample_rows(w, n_random=256).numpy()
+    ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, False, sel_gpu, gt, rows=rows, linear_form="state")
+    out = Hn.f64(ctx.forward(qd, si, sc, group_tokens=gt))
+    o_sp = Hn.f64(ctx.forward(qd, si, sc, group_tokens=gt, flags=hsa.HSA_FWD_NO_LINEAR))
+    assert ctx.device_status() == 0
+    Hn.assert_close(o_sp[rows], ref["O_sp"][rows], "O_sp")
+    Hn.assert_close(out[rows], ref["out"][rows], "out")
+    assert np.isfinite(out).all()
+    ctx.destroy()
+
+
+def test_linformer_full_size_segments_sampled(cuda_device):
+    """The Linformer form at the layer's own sizes: rank 256, segments of one 4680-token chunk,
+    three segments, 12 heads; outputs on sampled rows (rows are independent)."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["cfg2_linformer"]
+    rank, seg = 256, w.chunk
+    ek, ev = W.gen_linformer_weights(w, rank, seg)
+    ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=w.Lq, max_topk=w.topk,
+                         lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=rank, lin_seg_tokens=seg,
+                         e_k=ek.to(cuda_device), e_v=ev.to(cuda_device), device=cuda_device)
+    for pool in (ctx.k_pool, ctx.v_pool, ctx.kc_pool, ctx.vc_pool):
+        pool.fill_(0xFF)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    budgets = W.gen_budgets(w)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    si, sc = ctx.select_blocks(qd, budgets.to(cuda_device))
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, scores = O.select_blocks(qn, Kn, w.N, False, budgets.tolist())
+    Hn.check_selection(sel_gpu, sel_ref, scores)
+    rows = W.sample_rows(w, n_random=256).numpy()
+    Kt, Vt = O.linformer_compress(Kn, Vn, Hn.f32(ek), Hn.f32(ev), seg)
+    assert Kt.shape[0] == w.n_chunks * rank
+    o_lin_ref = O.linformer_branch(qn[rows], Kt, Vt)
+    o_sp_ref = O.sparse_branch(qn, Kn, Vn, sel_gpu, w.N, False, rows=rows)[rows]
+    out = Hn.f64(ctx.forward(qd, si, sc))
+    o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
+    assert ctx.device_status() == 0
+    Hn.assert_close(o_lin[rows], o_lin_ref, "O_lin (Linformer)")
+    Hn.assert_close(out[rows], o_lin_ref + o_sp_ref, "out")
+    assert np.isfinite(out).all()
+    ctx.destroy()
+
+
 def test_safe_pass_when_later_blocks_dominate(cuda_device):
     """Scores of later blocks exceed the first block's row maximum by far more than the fixed
     exponent reference of the normal pass allows: the tile must be redone with a running maximum
@@ -272,10 +336,13 @@ def _sampled_forward_check(w, ctx, K, V, q, device, n_random=192):
     ref = O.hsa_forward(qn, K, V, K.shape[0], False, sel_gpu, rows=rows, linear_form="state")
     out = Hn.f64(ctx.forward(qd, si, sc))
     o_sp = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_LINEAR))
+    o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
     assert ctx.device_status() == 0
     Hn.assert_close(o_sp[rows], ref["O_sp"][rows], "O_sp")
+    # the linear branch on its own: inside `out` it is an order of magnitude below the sparse branch
+    Hn.assert_close(o_lin[rows], ref["O_lin"][rows], "O_lin")
     Hn.assert_close(out[rows], ref["out"][rows], "out")
-    assert np.isfinite(out).all()
+    assert np.isfinite(out).all() and np.isfinite(o_lin).all()
     return sel_gpu
 
 
@@ -309,11 +376,12 @@ def test_long_history_and_head_adaptive_budgets_sampled(name, cuda_device):
     ctx.destroy()
 
 
-def test_rollout_steps_sampled(cuda_device):
-    """cfg5 shape: append a chunk, select, forward, 80 times on one layer's context; the oracle
-    checks the steps at chunks 0, 1, 39 and 79 (its linear state is carried along in fp64)."""
+@pytest.mark.parametrize("layer", [0, 29])
+def test_rollout_steps_sampled(layer, cuda_device):
+    """cfg5 shape: append a chunk, select, forward, 80 times on one layer's context (the first and
+    the last layer of the stack); the oracle checks the steps at chunks 0, 1, 39 and 79 (its linear
+    state is carried along in fp64)."""
     w = W.WORKLOADS["cfg5"]
-    layer = 29
     ctx = Hn.build_context(w, cuda_device, max_topk=w.topk)
     Ks, Vs = [], []
     S = np.zeros((w.H, w.d, w.d))

@@ -476,3 +476,42 @@ def test_retrieved_pages_mask_the_selection():
     got2, _ = O.select_blocks_mixed(q, K, N, False, [-1, 99], inter_pages=2, intra_first_page=10,
                                     kv_pages=[0], kv_page_blocks=3)
     assert all(got2[h][0].tolist() == [0, 1, 10, 11] for h in range(2))   # block (2, 3) straddles the page end
+
+
+# ---------------------------------------------------------------- row subsets and the state form
+@pytest.mark.parametrize("causal,group_tokens", [(False, 0), (True, 0), (False, 128), (True, 128)])
+def test_row_subset_and_state_form_match_brute_force_on_those_rows(causal, group_tokens):
+    """The full-size GPU parity cases evaluate the oracle on a subset of query rows
+    (rows=...) and, for non-causal cases, with the linear branch in its state form.
+    Both must give, on the chosen rows, what the pure-Python brute force gives for them,
+    and exact zeros on every other row."""
+    H, d, Lq, N = 2, 8, 300, 330                    # 6 blocks (tail 10), 3 query groups of 128
+    q, K, V = rnd((Lq, H, d), 40), rnd((N, H, d), 41), rnd((N, H, d), 42)
+    q_pos0 = N - Lq if causal else N
+    sel, _ = O.select_blocks(q, K, q_pos0, causal, [2, 3], group_tokens)
+    rows = np.array([0, 1, 127, 128, 131, 255, 256, 299])
+    groups = O.group_bounds(Lq, group_tokens)
+    g_of = lambda i: next(g for g, (a, e) in enumerate(groups) if a <= i < e)
+    keysets = [[[j for b in sel[h][g_of(i)] for j in range(64 * int(b), min(N, 64 * int(b) + 64))]
+                if i in rows else [] for i in range(Lq)] for h in range(H)]
+    sp_ref = np.array(brute.attention_rows(q, K, V, N, H, d, Lq, q_pos0, causal, keysets))
+    lin_ref = np.array(brute.linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal))
+    other = np.setdiff1d(np.arange(Lq), rows)
+    lin_ref[other] = 0.0
+    sp = O.sparse_branch(q, K, V, sel, q_pos0, causal, group_tokens, rows=rows)
+    lp = O.linear_parallel(q, K, V, q_pos0, causal, rows=rows)
+    assert np.abs(sp - sp_ref).max() < 1e-12 and np.abs(sp[other]).max() == 0.0
+    assert np.abs(lp - lin_ref).max() < 1e-12 and np.abs(lp[other]).max() == 0.0
+    for form in ("parallel", "state"):
+        r = O.hsa_forward(q, K, V, q_pos0, causal, sel, group_tokens, rows=rows, linear_form=form)
+        assert np.abs(r["O_sp"] - sp_ref).max() < 1e-12
+        assert np.abs(r["O_lin"] - lin_ref).max() < 1e-11
+        assert np.abs(r["out"] - (sp_ref + lin_ref)).max() < 1e-11
+        assert np.abs(r["out"][other]).max() == 0.0
+        full = O.hsa_forward(q, K, V, q_pos0, causal, sel, group_tokens, linear_form=form)
+        assert np.abs(full["out"][rows] - r["out"][rows]).max() < 1e-11
+    # the same with gates: rows outside the subset stay exactly zero
+    g1, g2 = rnd((Lq, H), 43), rnd((Lq, H, d), 44)
+    r = O.hsa_forward(q, K, V, q_pos0, causal, sel, group_tokens, g1, g2, 1, rows=rows, linear_form="state")
+    sig = lambda x: 1.0 / (1.0 + np.exp(-x))
+    assert np.abs(r["out"] - (sig(g1)[:, :, None] * lin_ref + sig(g2) * sp_ref)).max() < 1e-11
