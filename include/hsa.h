@@ -289,8 +289,8 @@ int hsa_device_status(hsa_ctx* ctx, int32_t* status_out);
 int hsa_set_wait_limit_ns(hsa_ctx* ctx, uint64_t wait_ns);
 
 /* Byte offsets inside the workspace, for tests and monitoring: the int32 status word, and the
- * two uint32 words {arrive count, generation} of the selection kernel's grid barrier (both are
- * zero whenever no selection kernel is running). */
+ * two uint32 words {arrive count, generation} of the selection kernel's grid barrier (the count
+ * is zero whenever no selection kernel is running; the generation advances by two per launch). */
 int hsa_workspace_layout(hsa_ctx* ctx, size_t* off_status, size_t* off_barrier);
 
 /* Synchronises the device, reads and clears a counter: the number of (query tile, head) work

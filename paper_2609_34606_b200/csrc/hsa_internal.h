@@ -60,8 +60,8 @@ struct SelectArgs {
   int32_t* sel_cnt;
   int kcap;
   int32_t* status;
-  unsigned* barrier;  // grid barrier of the single-launch path: {arrive count, generation}, both zero
-                      // when no launch is in flight (null: three launches)
+  unsigned* barrier;  // grid barrier of the single-launch path: {arrive count, generation}, the count
+                      // zero when no launch is in flight (null: three launches)
   unsigned long long wait_ns;  // bound of a wait at that barrier
   // candidate geometry: pages before the first intra-chunk page are selected in runs of inter_pages pages against
   // budgets[], the pages from it on one by one against intra_budgets[] (null: all of them)

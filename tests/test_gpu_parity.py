@@ -743,7 +743,7 @@ def test_grid_barrier_wait_that_runs_out_is_reported_and_leaves_the_context_usab
     ref_idx, ref_cnt = ctx.select_blocks(q, budgets)
     assert ctx.device_status() == 0 and int(ref_cnt.sum()) > 0
     words = ctx.barrier_words()
-    assert words.tolist() == [0, 0]
+    assert int(words[0]) == 0                  # the arrive count is back at zero after every launch
     ctx.set_wait_limit_ns(5_000_000)
     words[0] = 0x40000000                      # no arrival will ever be the last one
     idx, cnt = ctx.alloc_selection(w.Lq)
