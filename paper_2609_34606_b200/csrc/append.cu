@@ -197,10 +197,25 @@ __global__ void state_reduce_kernel(AppendArgs a) {
     hl[2 * DD] = oh;
     hl[3 * DD] = __float2bfloat16_rn(s_old - __bfloat162float(oh));
   } else {
-    const size_t o = static_cast<size_t>(h) * D + (idx - DD);
+    const int k = idx - DD;
+    const size_t o = static_cast<size_t>(h) * D + k;
     const float z_old = a.z[o];
+    const float z_new = z_old + add;
     a.z_prev[o] = z_old;
-    a.z[o] = z_old + add;
+    a.z[o] = z_new;
+    if (D == 128) {
+      // operand images of z (current, previous): element (row n, dim k) of a K-major tile with the
+      // 128-byte swizzle sits at slab (k / 64), row n, 16-byte chunk ((k % 64) / 8) ^ (n % 8)
+      const int slab = k >> 6, kk = k & 63, c = kk >> 3;
+      const float zs[2] = {z_new, z_old};
+#pragma unroll
+      for (int w = 0; w < 2; ++w) {
+        uint8_t* img = a.zop + static_cast<size_t>(h * 2 + w) * kZopBytes + slab * (kZopBytes / 2) + (kk & 7) * 2;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(zs[w]);
+        *reinterpret_cast<__nv_bfloat16*>(img + 0 * 128 + ((c ^ 0) << 4)) = hi;
+        *reinterpret_cast<__nv_bfloat16*>(img + 1 * 128 + ((c ^ 1) << 4)) = __float2bfloat16_rn(zs[w] - __bfloat162float(hi));
+      }
+    }
   }
 }
 

@@ -36,7 +36,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   // state
-  size_t S, z, S_prev, z_prev, hilo, ksum, state_total;
+  size_t S, z, S_prev, z_prev, hilo, zop, ksum, state_total;
   // workspace
   size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ad_w, ad_idx, ad_gini, ad_wsum,
       part_o, part_l, part_ref, part_ticket, ws_total;
@@ -75,6 +75,7 @@ Layout make_layout(const hsa_config* c) {
   L.S_prev = o; o = align_up(o + H * D * D * 4, 1024);
   L.z_prev = o; o = align_up(o + H * D * 4, 1024);
   L.hilo = o;   o = align_up(o + H * 4 * D * D * 2, 1024);
+  L.zop = o;    o = align_up(o + H * 2 * kZopBytes, 1024);
   L.ksum = o;   o = align_up(o + H * P * D * 4, 1024);
   L.state_total = o;
   const size_t tiles = (static_cast<size_t>(c->max_q_tokens) + kTileM - 1) / kTileM;
@@ -322,6 +323,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   a.S_prev = reinterpret_cast<float*>(stt + ctx->lay.S_prev);
   a.z_prev = reinterpret_cast<float*>(stt + ctx->lay.z_prev);
   a.hilo = reinterpret_cast<__nv_bfloat16*>(stt + ctx->lay.hilo);
+  a.zop = stt + ctx->lay.zop;
   a.spart = reinterpret_cast<float*>(ws + ctx->lay.spart);
   int nsplit = ctx->nsm / a.H;
   if (nsplit < 1) nsplit = 1;
@@ -535,6 +537,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   p.n_blocks = static_cast<int>((ctx->n_tokens + kBlock - 1) / kBlock);
   p.use_prev = causal_lin ? 1 : 0;
   p.z = reinterpret_cast<const float*>(stt + (causal_lin ? ctx->lay.z_prev : ctx->lay.z));
+  p.zop = stt + ctx->lay.zop;
   p.g_lin = static_cast<const __nv_bfloat16*>(g_lin);
   p.g_sp = static_cast<const __nv_bfloat16*>(g_sp);
   p.g_ts = gate_tok_stride;

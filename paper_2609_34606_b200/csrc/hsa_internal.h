@@ -11,6 +11,10 @@ namespace hsa {
 constexpr int kBlock = HSA_PAGE_TOKENS;  // tokens per KV block = tokens per page
 constexpr int kTileM = 128;              // query rows per work item of the forward kernel
 constexpr int kStateSplitMax = 16;       // token-axis splits of the state update (per head)
+// z as a [16 x 128] bf16 K-major operand image (128-byte swizzle, two slabs of 64 dims): row 0 holds
+// the bf16 rounding of z, row 1 the bf16 rounding of the remainder, rows 2..15 are zero, so that
+// phi(Q) times it gives the denominator phi(q).z as the sum of two accumulator columns
+constexpr int kZopBytes = 4096;
 constexpr int kFwdSplitMax = 16;         // CTAs a long (query tile, head) of the forward kernel is split over
 
 __host__ __device__ inline int64_t min64(int64_t a, int64_t b) { return a < b ? a : b; }
@@ -36,6 +40,7 @@ struct AppendArgs {
   float* S_prev;    // state before this append
   float* z_prev;
   __nv_bfloat16* hilo;  // [H][2 cur/prev][2 hi/lo][D][D]
+  uint8_t* zop;         // [H][2 cur/prev][kZopBytes]: z as a tensor-core operand (head_dim 128)
   float* spart;         // [H][nsplit][D*D + D] scratch
   int nsplit;
   int lin_state;  // update the linear state?
@@ -97,6 +102,7 @@ struct FwdParams {
   const int32_t* page_table;
   int n_blocks;
   const float* z;       // [H][D] state the linear branch applies
+  const uint8_t* zop;   // [H][2 cur/prev][kZopBytes]: the same z as a tensor-core operand
   int state_row0_mul;   // row of the hi/lo state tensor map = ((h*2 + use_prev)*2 + hl)*D
   int use_prev;
   const __nv_bfloat16* g_lin;

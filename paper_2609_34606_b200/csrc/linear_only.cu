@@ -2,16 +2,21 @@
 //   out[i,h] = g_lin * phi(q_i)^T S[h] / (phi(q_i)^T z[h]),   phi(x) = elu(x) + 1
 // A lean kernel for the case with no sparse branch: the only traffic is Q in and out out, so it is
 // bound by HBM, not by the tensor cores.
-// One persistent CTA per SM walks over a contiguous run of (head, query tile) items; the roles form
-// a pipeline, so that the load of one tile, the phi(Q) arithmetic of the next, the MMAs of a third
-// and the write-out of a fourth overlap:
-//   warp 0      (one lane)  TMA loads of the [128 x 128] Q tiles into a three-stage ring
-//   warps 2-9   phi(Q) written in place (it is the K-major A operand) + the denominators phi(q).z
-//   warp 1      (one lane)  16 tcgen05 MMAs per tile against S_hi and S_lo (kept in shared memory;
-//               reloaded by the same lane when the run crosses into the next head) into one of two
-//               TMEM accumulators
-//   warps 10-17 accumulator -> normalised, gated bf16 rows staged in the tile's ring stage (phi(Q)
-//               is dead by then) -> TMA store -> the stage goes back to warp 0
+// One persistent CTA per SM owns a contiguous run of (head, query tile) items (three at the measured
+// size) and asks for the head's state and all of its Q tiles at once, before anything else is set
+// up, so that the DRAM latency is paid once.  Roles:
+//   warps 0-15  workers, thread = (row, quarter of the dims): phi(q) as packed bf16 into TMEM (the A
+//               operand: with A in TMEM the MMAs read only the state from shared memory, which
+//               leaves half of its bandwidth to the workers), and later the accumulator ->
+//               normalised, gated bf16 row staged where the Q tile was; the loop runs phi(tile i + 1)
+//               before the write-out of tile i, so that the tensor cores work on tile i meanwhile
+//   warp 16     (one lane) the TMA loads; per tile 32 tcgen05 MMAs phi(Q) S_hi + phi(Q) S_lo and 8 small
+//               ones phi(Q) [z_hi z_lo]: the denominator comes out of the tensor cores as two more
+//               accumulator columns
+//   warp 17     (one lane) TMA store of a finished tile; refills the tile's stage when the run is
+//               longer than the ring
+// (Q and the output go through shared memory by TMA: per-thread 16-byte global accesses at the
+// 3 KB row pitch of a [tokens][H][d] tensor were measured 70 % slower.)
 // Every wait is bounded; on expiry the CTA records a timeout and leaves.
 #include <cuda_bf16.h>
 
@@ -20,43 +25,36 @@
 
 namespace hsa {
 
-#ifdef HSA_TIMING
-__device__ long long g_lo_timing[256];
-#define LO_T(slot)                                                        \
-  do {                                                                    \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) {                     \
-      long long t_;                                                       \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));               \
-      g_lo_timing[(slot)] = t_;                                           \
-    }                                                                     \
-  } while (0)
-#else
-#define LO_T(slot) \
-  do {             \
-  } while (0)
-#endif
-
 namespace {
 
-constexpr int kLoStages = 3;                  // Q ring
-constexpr int kLoGroup = 256;                 // threads of the phi group and of the epilogue group
-constexpr int kLoThreads = 64 + 2 * kLoGroup;
-constexpr int kLoTile = 128 * 128 * 2;        // one [128 x 128] bf16 tile = two swizzled slabs
+constexpr int kLoStages = 3;                    // Q ring
+#ifndef HSA_LO_PARTS
+#define HSA_LO_PARTS 2
+#endif
+constexpr int kLoParts = HSA_LO_PARTS;           // bf16 parts of S fed to the tensor cores: hi + lo
+constexpr int kLoSlots = 2;                     // TMEM slots: accumulator + phi(Q) operand
+constexpr int kLoWorkers = 512;                 // warps 0..15
+constexpr int kLoThreads = kLoWorkers + 64;
+constexpr int kLoIssueWarp = kLoWorkers / 32, kLoStoreWarp = kLoIssueWarp + 1;
+constexpr int kLoTile = 128 * 128 * 2;          // one [128 x 128] bf16 tile = two swizzled slabs
 constexpr int kLoHalf = kLoTile / 2;
-constexpr int kLoStats = kLoStages * 2 * 128 * 4;  // partial denominators per stage
-constexpr int kLoSmem = (2 + kLoStages) * kLoTile + kLoStats + 256 + 1024;
-constexpr uint32_t kLoTmemCols = 256;         // two accumulators
+constexpr int kLoZop = kZopBytes;               // [16 x 128] bf16 K-major operand: row 0 = z_hi, row 1 = z_lo
+constexpr int kLoSmem = (2 + kLoStages) * kLoTile + kLoZop + 512 + 1024;
+constexpr uint32_t kLoTmemCols = 512;
+constexpr uint32_t kLoSlotCols = 256;           // per slot: 128 numerator columns, 16 for the denominator, 64 of phi(Q)
+constexpr uint32_t kLoColDen = 128, kLoColA = 160;
 
 struct LoBars {
   uint64_t q_full[kLoStages];     // Q tile landed
-  uint64_t q_empty[kLoStages];    // output tile stored: the stage may be refilled
-  uint64_t phi_ready[kLoStages];  // phi(Q) written
-  uint64_t mma_done[2];           // accumulator final
-  uint64_t acc_free[2];           // accumulator read back
-  uint64_t s_full;                // state tiles landed
+  uint64_t out_ready[kLoStages];  // output tile staged (one arrival per worker warp)
+  uint64_t phi_ready[kLoSlots];   // phi(Q) written (one arrival per worker warp)
+  uint64_t mma_done[kLoSlots];    // accumulator final, phi(Q) operand dead
+  uint64_t acc_free[kLoSlots];    // accumulator read back (one arrival per worker warp)
+  uint64_t s_full;                // state tiles and z operand landed
   uint32_t tmem_base;
   volatile int abort_flag;
 };
+static_assert(sizeof(LoBars) <= 512, "barrier block must fit its shared-memory slot");
 
 __device__ __forceinline__ bool lo_wait(uint64_t* bar, uint32_t parity, LoBars* bars, int32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -71,10 +69,21 @@ __device__ __forceinline__ bool lo_wait(uint64_t* bar, uint32_t parity, LoBars* 
 
 __device__ __forceinline__ float lo_phi(float x) {
   float e;  // elu(x) + 1 = max(x, 0) + exp(min(x, 0))
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(x, 0.f) * 1.4426950408889634f));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(x * 1.4426950408889634f, 0.f)));
   return fmaxf(x, 0.f) + e;
 }
 
+// plain (untiled) bulk copy global -> shared, completion on an mbarrier
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(reinterpret_cast<uint64_t>(gmem)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(taddr) : "memory");
+}
 }  // namespace
 
 __global__ void __launch_bounds__(kLoThreads, 1)
@@ -84,235 +93,245 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
   extern __shared__ uint8_t lo_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(lo_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  uint8_t* s_state = smem;                 // S_hi | S_lo, MN-major B operands
-  uint8_t* s_ring = smem + 2 * kLoTile;    // Q tile -> phi(Q) -> output tile, per stage
-  float* stats = reinterpret_cast<float*>(smem + (2 + kLoStages) * kLoTile);  // [stage][half][128]
-  LoBars* bars = reinterpret_cast<LoBars*>(smem + (2 + kLoStages) * kLoTile + kLoStats);
+  uint8_t* s_state = smem;                        // S_hi | S_lo, MN-major B operands
+  uint8_t* s_zop = smem + 2 * kLoTile;            // z operand
+  uint8_t* s_ring = smem + 2 * kLoTile + kLoZop;  // Q tile -> output tile, per stage
+  LoBars* bars = reinterpret_cast<LoBars*>(smem + (2 + kLoStages) * kLoTile + kLoZop);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp == 0) LO_T(0);
   const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
   // this CTA's run of items (item = head * n_tiles + tile)
   const int i_begin = static_cast<int>(static_cast<int64_t>(blockIdx.x) * n_items / gridDim.x);
   const int i_end = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * n_items / gridDim.x);
   const int my_items = i_end - i_begin;
 
-  if (threadIdx.x == 0) {
+  auto load_q = [&](int it) {
+    const int s = it % kLoStages;
+    const int item = i_begin + it, h = item / n_tiles, tile = item % n_tiles;
+    mbar_expect_tx(&bars->q_full[s], kLoTile);
+    for (int dh = 0; dh < 2; ++dh)
+      tma_load_3d(s_ring + s * kLoTile + dh * kLoHalf, &tm_q, &bars->q_full[s], dh * 64, h, tile * kTileM);
+  };
+  auto load_state = [&](int h) {
+    mbar_expect_tx(&bars->s_full, kLoParts * kLoTile + kLoZop);
+    for (int hl = 0; hl < kLoParts; ++hl) {
+      const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
+      for (int kb = 0; kb < 2; ++kb)
+        for (int dh = 0; dh < 2; ++dh)
+          tma_load_2d(s_state + hl * kLoTile + dh * kLoHalf + kb * (kBlock * 128), &tm_state, &bars->s_full, dh * 64,
+                      rbase + kb * 64);
+    }
+    bulk_load(s_zop, p.zop + static_cast<size_t>(h * 2 + p.use_prev) * kLoZop, kLoZop, &bars->s_full);
+  };
+
+  // the kernel behind this one may be scheduled as soon as this grid's CTAs have all started
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == kLoIssueWarp * 32) {
     for (int s = 0; s < kLoStages; ++s) {
       mbar_init(&bars->q_full[s], 1);
-      mbar_init(&bars->q_empty[s], 1);
-      mbar_init(&bars->phi_ready[s], kLoGroup);
+      mbar_init(&bars->out_ready[s], kLoWorkers / 32);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < kLoSlots; ++a) {
+      mbar_init(&bars->phi_ready[a], kLoWorkers / 32);
       mbar_init(&bars->mma_done[a], 1);
-      mbar_init(&bars->acc_free[a], kLoGroup);
+      mbar_init(&bars->acc_free[a], kLoWorkers / 32);
     }
     mbar_init(&bars->s_full, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
-    tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_state);
+    // launched as a programmatic dependent: nothing of the kernel before this one is read earlier
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // every load this CTA will need at first, at once: the DRAM latency is paid once
+    if (my_items > 0) {
+      load_q(0);
+      load_state(i_begin / n_tiles);
+      for (int it = 1; it < my_items && it < kLoStages; ++it) load_q(it);
+    }
     tma_prefetch_desc(&tm_out);
   }
-  if (warp == 1) {
+  if (warp == kLoStoreWarp) {
     tmem_alloc(&bars->tmem_base, kLoTmemCols);
     tmem_relinquish();
   }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  if (warp == 0) LO_T(1);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ Q producer (one lane)
-    if (elect_one_sync()) {
-      for (int it = 0; it < my_items; ++it) {
-        const int s = it % kLoStages;
-        if (it >= kLoStages && !lo_wait(&bars->q_empty[s], ((it / kLoStages) - 1) & 1, bars, p.status)) break;
-        const int item = i_begin + it, h = item / n_tiles, tile = item % n_tiles;
-        mbar_expect_tx(&bars->q_full[s], kLoTile);
-        for (int dh = 0; dh < 2; ++dh)
-          tma_load_3d(s_ring + s * kLoTile + dh * kLoHalf, &tm_q, &bars->q_full[s], dh * 64, h, tile * kTileM);
-      }
-    }
-  } else if (warp == 1) {
+  if (warp == kLoIssueWarp) {
     // ------------------------------------------------------------------ MMA issuer (one lane)
     if (elect_one_sync()) {
       constexpr uint32_t kHiSw = desc_hi_sw128(1024);
       constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
-      int cur_h = -1, s_loads = 0;
+      constexpr uint32_t idesc_z = idesc_bf16_f32(128, 16, 0, 0);
+      int cur_h = my_items > 0 ? i_begin / n_tiles : -1, s_loads = 0;
+      bool s_ok = false;
       for (int it = 0; it < my_items; ++it) {
-        const int s = it % kLoStages, a = it & 1;
+        const int a = it % kLoSlots;
         const int h = (i_begin + it) / n_tiles;
         if (h != cur_h) {
           // next head: its state replaces the old one once the MMAs that read the old one are done
-          if (it > 0 && !lo_wait(&bars->mma_done[(it - 1) & 1], ((it - 1) >> 1) & 1, bars, p.status)) break;
-          mbar_expect_tx(&bars->s_full, 2 * kLoTile);
-          for (int hl = 0; hl < 2; ++hl) {
-            const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
-            for (int kb = 0; kb < 2; ++kb)
-              for (int dh = 0; dh < 2; ++dh)
-                tma_load_2d(s_state + hl * kLoTile + dh * kLoHalf + kb * (kBlock * 128), &tm_state, &bars->s_full,
-                            dh * 64, rbase + kb * 64);
-          }
+          if (!lo_wait(&bars->mma_done[(it - 1) % kLoSlots], ((it - 1) / kLoSlots) & 1, bars, p.status)) break;
+          load_state(h);
+          cur_h = h;
+          s_ok = false;
+        }
+        if (!s_ok) {
           if (!lo_wait(&bars->s_full, s_loads & 1, bars, p.status)) break;
           ++s_loads;
-          cur_h = h;
+          s_ok = true;
         }
-        if (!lo_wait(&bars->phi_ready[s], (it / kLoStages) & 1, bars, p.status)) break;
-        if (it >= 2 && !lo_wait(&bars->acc_free[a], ((it >> 1) - 1) & 1, bars, p.status)) break;
+        if (!lo_wait(&bars->phi_ready[a], (it / kLoSlots) & 1, bars, p.status)) break;
+        if (it >= kLoSlots && !lo_wait(&bars->acc_free[a], ((it / kLoSlots) - 1) & 1, bars, p.status)) break;
         tc_fence_after();
-        const uint32_t a_lo = desc_lo_sw128(smem_u32(s_ring + s * kLoTile), 16);
-        for (int hl = 0; hl < 2; ++hl) {
+        const uint32_t acc = tmem + kLoSlotCols * a;
+        const uint32_t a_op = acc + kLoColA;  // phi(Q): 16 bf16 of K per 8 columns
+        for (int hl = 0; hl < kLoParts; ++hl) {
           const uint32_t b_lo = desc_lo_sw128(smem_u32(s_state + hl * kLoTile), kLoHalf);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = ((kk / 4) * kLoHalf + (kk % 4) * 32) >> 4;
-            tc_mma_ss_lo(tmem + 128 * a, a_lo + off, b_lo + kk * 128, kHiSw, idesc, (hl > 0 || kk > 0) ? 1u : 0u);
-          }
+          for (int kk = 0; kk < D / 16; ++kk)
+            tc_mma_ts_lo(acc, a_op + kk * 8, b_lo + kk * 128, kHiSw, idesc, (hl > 0 || kk > 0) ? 1u : 0u);
+        }
+        const uint32_t z_lo = desc_lo_sw128(smem_u32(s_zop), 16);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t zoff = ((kk / 4) * (kLoZop / 2) + (kk % 4) * 32) >> 4;
+          tc_mma_ts_lo(acc + kLoColDen, a_op + kk * 8, z_lo + zoff, kHiSw, idesc_z, kk > 0 ? 1u : 0u);
         }
         tc_commit(&bars->mma_done[a]);
-        LO_T(16 + it * 8 + 2);
       }
     }
-  } else if (warp < 2 + kLoGroup / 32) {
-    // ------------------------------------------------------------------ phi(Q) + denominators
-    const int t = threadIdx.x - 64;
-    const int r = t & 127, half = t >> 7;  // row of the tile, which 64 dims of it
-    const int cbase = half * 64;
-#pragma unroll 1
-    for (int it = 0; it < my_items; ++it) {
-      const int s = it % kLoStages;
-      const int h = (i_begin + it) / n_tiles;
-      if (!lo_wait(&bars->q_full[s], (it / kLoStages) & 1, bars, p.status)) break;
-      if (warp == 2) LO_T(16 + it * 8 + 0);
-      uint8_t* s_q = s_ring + s * kLoTile;
-      const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
-      // phi of this thread's half row, in place; the partial denominator uses the rounded values
-      // (two accumulators: the sum is not one long dependent chain)
-      float den0 = 0.f, den1 = 0.f;
-#pragma unroll
-      for (int c16 = 0; c16 < 8; ++c16) {
-        const float4 za = z4[c16 * 2], zb = z4[c16 * 2 + 1];
-        const float z[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
-        const int cc = cbase / 8 + c16;  // 16-byte chunk of the row
-        uint4* cell = reinterpret_cast<uint4*>(s_q + (cc >> 3) * kLoHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4));
-        const uint4 raw = *cell;
-        const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
-        uint32_t o[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float a0 = lo_phi(__uint_as_float(qw[i] << 16));
-          const float a1 = lo_phi(__uint_as_float(qw[i] & 0xffff0000u));
-          o[i] = pack_bf16(a0, a1);
-          den0 = fmaf(__uint_as_float(o[i] << 16), z[2 * i], den0);
-          den1 = fmaf(__uint_as_float(o[i] & 0xffff0000u), z[2 * i + 1], den1);
+  } else if (warp == kLoStoreWarp) {
+    // ------------------------------------------------------------------ stores + refills (one lane)
+    if (elect_one_sync()) {
+      for (int it = 0; it < my_items; ++it) {
+        const int s = it % kLoStages;
+        const int item = i_begin + it, h = item / n_tiles, tile = item % n_tiles;
+        if (!lo_wait(&bars->out_ready[s], (it / kLoStages) & 1, bars, p.status)) break;
+        uint8_t* s_q = s_ring + s * kLoTile;
+        for (int dh = 0; dh < 2; ++dh) tma_store_3d(&tm_out, s_q + dh * kLoHalf, dh * 64, h, tile * kTileM);
+        tma_store_commit();
+        if (it + kLoStages < my_items) {
+          tma_store_wait_read();  // the tile must stay put until it has been read
+          load_q(it + kLoStages);
         }
-        *cell = make_uint4(o[0], o[1], o[2], o[3]);
       }
-      stats[(s * 2 + half) * 128 + r] = den0 + den1;
-      fence_proxy_async_smem();  // generic-proxy writes above -> visible to the tensor cores
-      mbar_arrive(&bars->phi_ready[s]);  // (release: the epilogue group reads stats after the MMAs)
-      if (warp == 2) LO_T(16 + it * 8 + 1);
+      tma_store_wait_read();  // shared memory may go once the stores have read it
     }
   } else {
-    // ------------------------------------------------------------------ epilogue
-    const int e = threadIdx.x - 64 - kLoGroup;
-    const int quad = warp & 3;                         // TMEM lane quadrant of this warp
-    const int half = (warp - (2 + kLoGroup / 32)) >> 2;  // which 64 dims of the row
+    // ------------------------------------------------------------------ workers
+    // thread = (row, quarter of the dims): the same cells of the stage hold its Q and its output;
+    // the row is also its TMEM lane
+    const int quad = warp & 3, cq = warp >> 2;
     const int r = quad * 32 + lane;
-    const int cbase = half * 64;
     const uint32_t lane_off = static_cast<uint32_t>(quad * 32) << 16;
+    uint32_t cell[4];  // byte offsets of the thread's four 16-byte chunks inside a stage
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int cc = cq * 4 + i;
+      cell[i] = (cc >> 3) * kLoHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4);
+    }
     const bool sig = p.gate_act == 1;
+    const bool plain = p.g_lin == nullptr && p.lin_num == nullptr;  // no gate, no causal partials
     bool ok = true;
 #pragma unroll 1
-    for (int it = 0; it < my_items && ok; ++it) {
-      const int s = it % kLoStages, a = it & 1;
-      const int item = i_begin + it, h = item / n_tiles, tile = item % n_tiles;
-      const int row0 = tile * kTileM, row = row0 + r;
-      uint8_t* s_q = s_ring + s * kLoTile;
-      ok = lo_wait(&bars->mma_done[a], (it >> 1) & 1, bars, p.status);
-      if (!ok) break;
-      if (warp == 10) LO_T(16 + it * 8 + 3);
-      tc_fence_after();
-      float den = stats[(s * 2) * 128 + r] + stats[(s * 2 + 1) * 128 + r];
-      const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
-      const float* lnum = nullptr;
-      if (wr && p.lin_num != nullptr) {
-        lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D;
-        den += p.lin_den[static_cast<size_t>(row) * p.H + h];
-      }
-      const float inv_den = den > 0.f ? 1.f / den : 0.f;
-      const __nv_bfloat16* gl =
-          (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
-      const int g_ds = static_cast<int>(p.g_ds);
-#pragma unroll 1
-      for (int c0 = cbase; c0 < cbase + 64; c0 += 32) {
-        uint32_t acc[32];
-        tmem_ld32(tmem + lane_off + 128 * a + c0, acc);
-        tc_wait_ld();
-        if (c0 + 32 == cbase + 64) {  // last read of the accumulator: the MMAs of tile it + 2 may have it
-          tc_fence_before();
-          mbar_arrive(&bars->acc_free[a]);
+    for (int it = 0; it <= my_items && ok; ++it) {
+      if (it < my_items) {
+        // ---- phi of tile it into TMEM slot it % 2 (its last reader, the MMAs of tile it - 2, is done:
+        // the write-out of that tile, which waited for them, comes earlier in this loop)
+        const int s = it % kLoStages;
+        ok = lo_wait(&bars->q_full[s], (it / kLoStages) & 1, bars, p.status);
+        if (!ok) break;
+        const uint8_t* s_q = s_ring + s * kLoTile;
+        uint4 raw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) raw[i] = *reinterpret_cast<const uint4*>(s_q + cell[i]);
+        uint32_t o[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw[i]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            o[4 * i + e] = pack_bf16(lo_phi(__uint_as_float(qw[e] << 16)), lo_phi(__uint_as_float(qw[e] & 0xffff0000u)));
         }
+        // this thread's 32 values of phi(q) are 16 columns of its TMEM lane
+        tmem_st16(tmem + lane_off + kLoSlotCols * (it % kLoSlots) + kLoColA + cq * 16, o);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->phi_ready[it % kLoSlots]);
+      }
+      if (it >= 1) {
+        // ---- write-out of tile it - 1
+        const int jt = it - 1;
+        const int s = jt % kLoStages, a = jt % kLoSlots;
+        const int item = i_begin + jt, h = item / n_tiles, tile = item % n_tiles;
+        const int row = tile * kTileM + r;
+        uint8_t* s_q = s_ring + s * kLoTile;
+        ok = lo_wait(&bars->mma_done[a], (jt / kLoSlots) & 1, bars, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t acc = tmem + lane_off + kLoSlotCols * a;
+        uint32_t v[32], d0, d1;
+        tmem_ld32(acc + cq * 32, v);
+        tmem_ld2(acc + kLoColDen, d0, d1);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->acc_free[a]);
+        float den = __uint_as_float(d0) + __uint_as_float(d1);
+        const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
         uint32_t packed[16];
-        if (gl == nullptr && lnum == nullptr) {
+        if (plain) {
+          const float inv_den = den > 0.f ? 1.f / den : 0.f;
 #pragma unroll
           for (int i = 0; i < 32; i += 2)
-            packed[i >> 1] = pack_bf16(__uint_as_float(acc[i]) * inv_den, __uint_as_float(acc[i + 1]) * inv_den);
+            packed[i >> 1] = pack_bf16(__uint_as_float(v[i]) * inv_den, __uint_as_float(v[i + 1]) * inv_den);
         } else {
+          const float* lnum = nullptr;
+          if (wr && p.lin_num != nullptr) {
+            lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D + cq * 32;
+            den += p.lin_den[static_cast<size_t>(row) * p.H + h];
+          }
+          const float inv_den = den > 0.f ? 1.f / den : 0.f;
+          const __nv_bfloat16* gl =
+              (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
+          const int g_ds = static_cast<int>(p.g_ds);
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
             float w0 = inv_den, w1 = inv_den, l0 = 0.f, l1 = 0.f;
             if (gl) {
-              const float g0 = __bfloat162float(gl[(c0 + i) * g_ds]), g1 = __bfloat162float(gl[(c0 + i + 1) * g_ds]);
+              const float g0 = __bfloat162float(gl[(cq * 32 + i) * g_ds]), g1 = __bfloat162float(gl[(cq * 32 + i + 1) * g_ds]);
               w0 *= sig ? __fdividef(1.f, 1.f + __expf(-g0)) : g0;
               w1 *= sig ? __fdividef(1.f, 1.f + __expf(-g1)) : g1;
             }
             if (lnum) {
-              l0 = lnum[c0 + i];
-              l1 = lnum[c0 + i + 1];
+              l0 = lnum[i];
+              l1 = lnum[i + 1];
             }
-            packed[i >> 1] = pack_bf16(w0 * (__uint_as_float(acc[i]) + l0), w1 * (__uint_as_float(acc[i + 1]) + l1));
+            packed[i >> 1] = pack_bf16(w0 * (__uint_as_float(v[i]) + l0), w1 * (__uint_as_float(v[i + 1]) + l1));
           }
         }
-        // the phi(Q) tile is dead: the output row goes where it was, in the swizzled layout the
-        // output tensor map expects
+        // the Q tile is dead (each thread has read its own cells): the output row goes where it was,
+        // in the swizzled layout the output tensor map expects
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int cc = (c0 >> 3) + q4;
-          *reinterpret_cast<uint4*>(s_q + (cc >> 3) * kLoHalf + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) =
-              make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
-        }
-      }
-      if (warp == 10) LO_T(16 + it * 8 + 4);
-      fence_proxy_async_smem();
-      asm volatile("bar.sync 1, %0;" ::"n"(kLoGroup) : "memory");
-      if (e == 0) {
-        for (int dh = 0; dh < 2; ++dh) tma_store_3d(&tm_out, s_q + dh * kLoHalf, dh * 64, h, row0);
-        tma_store_commit();
-        tma_store_wait_read();  // the tile must stay put until it has been read
-        mbar_arrive(&bars->q_empty[s]);
-        LO_T(16 + it * 8 + 5);
+        for (int i = 0; i < 4; ++i)
+          *reinterpret_cast<uint4*>(s_q + cell[i]) =
+              make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->out_ready[s]);
       }
     }
-    if (e == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    if (warp == 10) LO_T(2);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kLoStoreWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kLoTmemCols);
   }
 }
-
-#ifdef HSA_TIMING
-extern "C" int hsa_debug_read_lo_timing(long long* host_out, int n) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_lo_timing, sizeof(long long) * n));
-}
-#endif
 
 cudaError_t linear_only_init() {
   return cudaFuncSetAttribute(hsa_linear_only_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLoSmem);
@@ -323,8 +342,17 @@ cudaError_t launch_linear_only(const FwdParams& p, int nsm, const CUtensorMap& t
   const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
   const int n_items = n_tiles * p.H;
   const int grid = n_items < nsm ? n_items : nsm;  // one persistent CTA per SM
-  hsa_linear_only_kernel<<<grid, kLoThreads, kLoSmem, st>>>(p, n_items, tm_q, tm_state, tm_out);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kLoThreads);
+  cfg.dynamicSmemBytes = kLoSmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, hsa_linear_only_kernel, p, n_items, tm_q, tm_state, tm_out);
 }
 
 }  // namespace hsa

@@ -758,7 +758,8 @@ def test_grid_barrier_wait_that_runs_out_is_reported_and_leaves_the_context_usab
     assert int(cnt.abs().sum()) == 0
     out = ctx.forward(q, idx, cnt)
     lin = ctx.forward(q, idx, cnt, flags=hsa.HSA_FWD_NO_SPARSE)
-    assert torch.equal(out, lin)
+    # (two different kernels: the same values up to the last bf16 bit)
+    assert float((out.float() - lin.float()).abs().max()) <= 1e-3 and float(lin.float().abs().max()) > 1e-2
     assert ctx.device_status() == hsa.HSA_ERR_DEVICE_TIMEOUT
     assert ctx.barrier_words().tolist() == [0, 0] and ctx.device_status() == 0
     idx2, cnt2 = ctx.select_blocks(q, budgets)
