@@ -33,34 +33,57 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_34606_b200 import workloads as W  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one hsa_forward_kernel<128, false> launch on cfg2, from
-# the ncu capture summarised in profiles/hsa_forward_kernel_cfg2.md (40.43 MB + 0.77 MB)
-NCU_TRAFFIC_BYTES = {"cfg2": 41.20e6}
+
+
+def ncu_traffic(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one forward-kernel launch on `workload`, as
+    recorded from the last ncu capture (a small tracked JSON beside the ncu summaries), or None."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        rec = json.load(open(path)).get("hsa_forward_kernel", {}).get(workload)
+        return None if rec is None else float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"])
+    except (OSError, ValueError, KeyError):
+        return None
+
+
 METRIC = "hsa_effective_tflops"
 UNIT = "TFLOP/s"
 RING = 4  # distinct (q, k, v, out) input sets rotated between steps (> L2 in total)
 
 
 # ----------------------------------------------------------------------------- work model
-def step_flops(w: W.Workload, sel_tokens_per_head) -> dict:
-    """Algorithmic FLOPs of one step (masked / unselected keys count as zero work)."""
+def step_flops(w: W.Workload, sel_row_tokens, lin: str = "state", lin_rank: int = 0) -> dict:
+    """Algorithmic FLOPs of one step (masked / unselected keys count as zero work).
+    sel_row_tokens = sum over heads and query groups of (rows of the group) x (valid tokens of its
+    selected blocks); with one selection per head that is Lq x the selected tokens of the head."""
     Lq, d, H = w.Lq, w.d, w.H
-    sparse = 4.0 * Lq * d * float(sum(sel_tokens_per_head))          # QK^T + PV
-    lin_apply = 2.0 * Lq * d * (d + 1) * H                            # phi(Q) S and phi(Q) z
-    state = 2.0 * w.chunk * d * (d + 1) * H                           # S += phi(K)^T V, z
+    sparse = 4.0 * d * float(sel_row_tokens)                          # QK^T + PV
     select = 2.0 * Lq * H * d + 2.0 * w.n_blocks * H * d
+    if lin == "linformer":
+        # compressed rows of all complete segments, softmax attention over them; the append projects
+        # one segment: K~ = E_K^T K, V~ = E_V^T V
+        lin_apply = 4.0 * Lq * (w.n_chunks * lin_rank) * d * H
+        state = 2.0 * 2.0 * lin_rank * w.chunk * d * H
+    else:
+        lin_apply = 2.0 * Lq * d * (d + 1) * H                        # phi(Q) S and phi(Q) z
+        state = 2.0 * w.chunk * d * (d + 1) * H                       # S += phi(K)^T V, z
     return {"forward": sparse + lin_apply, "append": state, "select": select,
-            "total": sparse + lin_apply + state + select}
+            "total": sparse + lin_apply + state + select, "sparse": sparse, "linear": lin_apply}
 
 
-def step_bytes(w: W.Workload, sel_tokens_per_head) -> dict:
-    """Algorithmic HBM bytes per call."""
+def step_bytes(w: W.Workload, sel_tokens) -> dict:
+    """Algorithmic HBM bytes per call (sel_tokens: valid tokens of the distinct selected blocks)."""
     Lq, d, H = w.Lq, w.d, w.H
     qo = Lq * H * d * 2
-    fwd = 2 * qo + sum(sel_tokens_per_head) * d * 4 + H * d * d * 4
+    fwd = 2 * qo + sel_tokens * d * 4 + H * d * d * 4
     app = 4 * w.chunk * H * d * 2 + H * d * d * 4 * 2
     sel = qo + w.n_blocks * H * d * 4
     return {"forward": float(fwd), "append": float(app), "select": float(sel)}
+
+
+def workload_desc(w: W.Workload) -> str:
+    return (f"{w.name}: H={w.H} d={w.d} chunk={w.Lq} history={w.N} tokens ({w.n_blocks} blocks of 64) " +
+            (f"top-{w.topk} blocks/head" if not w.budget_set else f"budgets per head from {list(w.budget_set)} (-1 = all)"))
 
 
 def load_peaks() -> dict:
@@ -138,9 +161,15 @@ def bench_ours(args, rank: int, world: int):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = W.WORKLOADS[args.workload]
+    gt = args.group_tokens
+    lin_kw = {}
+    if args.lin == "linformer":
+        ek, ev = W.gen_linformer_weights(w, args.lin_rank, w.chunk)
+        lin_kw = dict(lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=args.lin_rank, lin_seg_tokens=w.chunk,
+                      e_k=ek.to(dev), e_v=ev.to(dev))
     ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk),
                          max_topk=w.n_blocks if w.budget_set else max(w.topk, 1),
-                         page_order=W.gen_page_order(w, w.n_blocks), device=dev)
+                         page_order=W.gen_page_order(w, w.n_blocks), device=dev, **lin_kw)
     for c in range(w.n_chunks - 1):
         k, v = W.gen_kv_chunk(w, c, layer=rank)
         ctx.append_kv(k.to(dev), v.to(dev))
@@ -162,7 +191,7 @@ def bench_ours(args, rank: int, world: int):
         host.append(hs + [torch.empty_like(q).pin_memory()])
         devs.append([t.to(dev) for t in (q, k, v)] + [torch.empty(q.shape, dtype=torch.bfloat16, device=dev)])
     budgets = W.gen_budgets(w).to(dev)
-    sel = ctx.alloc_selection(w.Lq)
+    sel = ctx.alloc_selection(w.Lq, gt)
 
     def step(i, ev=None, from_host=False, with_forward=True):
         q, k, v, out = devs[i % RING]
@@ -180,11 +209,11 @@ def bench_ours(args, rank: int, world: int):
         ctx.append_kv(k, v)
         if ev:
             ev[1].record()
-        ctx.select_blocks(q, budgets, sel=sel)
+        ctx.select_blocks(q, budgets, group_tokens=gt, sel=sel)
         if ev:
             ev[2].record()
         if with_forward:
-            ctx.forward(q, sel[0], sel[1], out=out)
+            ctx.forward(q, sel[0], sel[1], group_tokens=gt, out=out)
         if ev:
             ev[3].record()
         if from_host:
@@ -201,9 +230,19 @@ def bench_ours(args, rank: int, world: int):
         step(i)
     torch.cuda.synchronize()
     assert ctx.device_status() == 0, "device-side error during warm-up"
-    cnt = sel[1].cpu().flatten().tolist()
+    cnt = sel[1].cpu()
     idx = sel[0].cpu()
-    sel_tokens = [sum(min(64, w.N - 64 * int(b)) for b in idx[h, 0, :cnt[h]].tolist()) for h in range(w.H)]
+    n_groups = cnt.shape[1]
+    rows_of = lambda g: (min(w.Lq, (g + 1) * gt) - g * gt) if gt else w.Lq
+    blk_tokens = lambda b: min(64, w.N - 64 * int(b))
+    sel_row_tokens, distinct = 0, 0
+    for h in range(w.H):
+        seen = set()
+        for g in range(n_groups):
+            blocks = idx[h, g, :int(cnt[h, g])].tolist()
+            sel_row_tokens += rows_of(g) * sum(blk_tokens(b) for b in blocks)
+            seen.update(blocks)
+        distinct += sum(blk_tokens(b) for b in seen)
 
     K = args.steps
     # eager pass with events between the calls: per-stage times (launch gaps included)
@@ -244,9 +283,11 @@ def bench_ours(args, rank: int, world: int):
         ctx.rewind(n_before)
         ctx.append_kv(devs[i % RING][1], devs[i % RING][2])
     NK = 5 * RING  # calls per graph
-    fwd = lambda flags: (lambda i: ctx.forward(devs[i % RING][0], sel[0], sel[1], out=devs[i % RING][3], flags=flags))
+    fwd = lambda flags: (lambda i: ctx.forward(devs[i % RING][0], sel[0], sel[1], group_tokens=gt,
+                                               out=devs[i % RING][3], flags=flags))
     kern = {"append": time_graph(capture(only_append, NK), NK),
-            "select": time_graph(capture(lambda i: ctx.select_blocks(devs[i % RING][0], budgets, sel=sel), NK), NK),
+            "select": time_graph(capture(lambda i: ctx.select_blocks(devs[i % RING][0], budgets, group_tokens=gt,
+                                                                     sel=sel), NK), NK),
             "forward": time_graph(capture(fwd(0), NK), NK),
             "linear_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_SPARSE), NK), NK),
             "sparse_only": time_graph(capture(fwd(hsa.HSA_FWD_NO_LINEAR), NK), NK)}
@@ -281,7 +322,33 @@ def bench_ours(args, rank: int, world: int):
     ms_total = e0.elapsed_time(e1)
     status = ctx.device_status()
 
-    # clocks: extend with an identical, untimed loop if the timed region was too short to sample
+    # the last replayed step against the same step issued call by call: selection and output bit for bit
+    last = (K - 1) % RING if (args.launch == "graph" and K % GS) or args.launch != "graph" else (GS - 1) % RING
+    sel_replayed = (sel[0].clone(), sel[1].clone())
+    out_replayed = devs[last][3].clone()
+    step(last)
+    torch.cuda.synchronize()
+    cnt_e = sel[1].cpu()
+    same = torch.equal(sel[1], sel_replayed[1]) and torch.equal(devs[last][3].view(torch.int16), out_replayed.view(torch.int16))
+    same = same and all(torch.equal(sel[0][h, g, :int(cnt_e[h, g])], sel_replayed[0][h, g, :int(cnt_e[h, g])])
+                        for h in range(w.H) for g in range(cnt_e.shape[1]))
+    if not same or ctx.device_status() != 0:
+        raise SystemExit("bench: the last replayed step differs from the same step issued call by call")
+
+    # spread of the step time: each replay of the 8-step graph timed on its own (>= 20 repeats)
+    reps = []
+    if args.launch == "graph":
+        evs_r = [torch.cuda.Event(enable_timing=True) for _ in range(25)]
+        torch.cuda.synchronize()
+        for i in range(24):
+            evs_r[i].record()
+            g_many.replay()
+        evs_r[24].record()
+        torch.cuda.synchronize()
+        reps = sorted(evs_r[i].elapsed_time(evs_r[i + 1]) / GS for i in range(24))
+
+    # clocks: sampled during the timed region; if that was too short for three samples, over an
+    # identical loop run right after it (said so in the record)
     probe = None
     if sampler is not None:
         time.sleep(0.15)
@@ -353,9 +420,12 @@ def bench_ours(args, rank: int, world: int):
         sampler.stop()
 
     from paper_2609_34606_b200 import sharding
-    ms_step, ms_e2e = sharding.max_over_ranks([ms_total / K, ms_e2e], device=dev)  # slowest rank
-    fl = step_flops(w, sel_tokens)
-    by = step_bytes(w, sel_tokens)
+    fl = step_flops(w, sel_row_tokens, args.lin, args.lin_rank)
+    # whole job: the FLOPs of all ranks over the slowest rank's time
+    agg_flops, sec_step = sharding.aggregate_throughput(fl["total"], ms_total / K * 1e-3, device=dev)
+    agg_e2e, sec_e2e = sharding.aggregate_throughput(fl["total"], ms_e2e * 1e-3, device=dev)
+    ms_step, ms_e2e = sec_step * 1e3, sec_e2e * 1e3
+    by = step_bytes(w, distinct)
     peaks = load_peaks()
     if rank == 0:
         if probe is not None:
@@ -364,11 +434,13 @@ def bench_ours(args, rank: int, world: int):
         tf = lambda f, ms: f / (ms * 1e-3) / 1e12
         fwd_tf = tf(fl["forward"], kern["forward"])
         line = {
-            "metric": METRIC, "value": world * tf(fl["total"], ms_step), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": agg_flops / 1e12, "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{w.name}: H={w.H} d={w.d} chunk={w.Lq} history={w.N} tokens "
-                                   f"({w.n_blocks} blocks of 64) top-{w.topk} blocks/head",
+            "config": {"workload": workload_desc(w),
+                       "selection": "one per head for the whole chunk" if not gt else f"one per {gt}-row query tile",
+                       "linear_branch": ("running state (S, z)" if args.lin == "state" else
+                                         f"Linformer form, rank {args.lin_rank}, segments of {w.chunk} tokens"),
                        "step": f"restore the {w.n_chunks - 1}-chunk running state (S, z) + hsa_append_kv + "
                                "hsa_select_blocks + hsa_forward",
                        "launch": (f"CUDA graphs: the timed loop replays a graph of {2 * RING} consecutive steps "
@@ -378,6 +450,9 @@ def bench_ours(args, rank: int, world: int):
                              f"({RING * 4 * w.Lq * w.H * w.d * 2 / 1e6:.0f} MB > 126 MB L2)",
                        "replicas": world},
             "ms_per_chunk": ms_step,
+            "ms_per_step_repeats": ({"n": len(reps), "min": reps[0], "median": reps[len(reps) // 2], "max": reps[-1]}
+                                    if reps else None),
+            "replay_check": "last replayed step == the same step issued call by call (selection and output bits)",
             "eager_ms_per_step": ms_eager,
             "eager_stage_ms": {"append": stage[0], "select": stage[1], "forward": stage[2]},
             "kernel_ms": {k2: kern[k2] for k2 in ("append", "select", "forward")},
@@ -386,13 +461,13 @@ def bench_ours(args, rank: int, world: int):
             "forward_modes_ms": {"linear_only": ms_lin_only, "sparse_only": ms_sp_only,
                                  "linear_only_gbs": (2 * w.Lq * w.H * w.d * 2 + w.H * w.d * w.d * 4) / ms_lin_only / 1e6},
             "clocks": clocks,
-            "e2e": {"value": world * tf(fl["total"], ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+            "e2e": {"value": agg_e2e / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": 3 * w.Lq * w.H * w.d * 2, "d2h_bytes_per_step": w.Lq * w.H * w.d * 2},
             "gpu_launches": 4 * K,  # append_fused, state_reduce, select_fused, hsa_forward per step
             "device_status": status,
             "roofline": {"kernel": "hsa_forward_kernel<128, false>", "bound": "tensor", "achieved": fwd_tf,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tf / peaks["bf16_tflops"],
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": by["forward"],
+                         "traffic": ncu_traffic(w.name), "algorithmic_bytes": by["forward"],
                          "peak_source": peaks["source"] + " (burst)",
                          "frac_of_sustained": fwd_tf / peaks["bf16_tflops_sustained"],
                          "timing": "average duration of the call replayed from CUDA graphs, CUDA events",
@@ -473,7 +548,7 @@ def bench_rollout(args, rank: int, world: int):
     sampler.stop()
     status = max(c.device_status() for c in ctxs)
     # work model: 64 full blocks per head from the first chunk on (a chunk alone is 73 blocks)
-    fl = step_flops(w, [w.topk * 64] * w.H)
+    fl = step_flops(w, w.Lq * w.topk * 64 * w.H)
     steps = w.n_chunks * layers
     best = min(runs, key=lambda r: r["ms_total"])
     ms_step = best["ms_total"] / steps
@@ -497,14 +572,26 @@ def bench_rollout(args, rank: int, world: int):
 
 # ----------------------------------------------------------------------------- oracle (CPU)
 def oracle_step(w: W.Workload, data, rows):
-    """One bounded oracle step: block selection over the full history, then both branches and the
-    merge on `rows` query rows (state form of the linear branch).  Returns seconds."""
+    """One bounded oracle step, stage by stage: block selection over the full history, the sparse
+    branch on `rows` query rows, the linear branch (state from scratch, applied to the chunk), the
+    merge.  Returns (seconds in all, selection, seconds per stage)."""
     from oracle import hsa_oracle as O
     q, K, V = data
-    t0 = time.perf_counter()
+    t = [time.perf_counter()]
     sel, _ = O.select_blocks(q, K, w.q_pos0, w.causal, W.gen_budgets(w).tolist())
-    O.hsa_forward(q, K, V, w.q_pos0, w.causal, sel, rows=rows, linear_form="state")
-    return time.perf_counter() - t0, sel
+    t.append(time.perf_counter())
+    o_sp = O.sparse_branch(q, K, V, sel, w.q_pos0, w.causal, rows=rows)
+    t.append(time.perf_counter())
+    if w.causal:
+        o_lin = O.linear_parallel(q, K, V, w.q_pos0, True, rows)
+    else:
+        S, z = O.linear_state(K, V)
+        o_lin = O.linear_from_state(q, S, z)
+    t.append(time.perf_counter())
+    O.merge(o_lin, o_sp)
+    t.append(time.perf_counter())
+    stages = dict(zip(("select", "sparse", "linear", "merge"), (b - a for a, b in zip(t, t[1:]))))
+    return t[-1] - t[0], sel, stages
 
 
 def oracle_data(w: W.Workload):
@@ -514,8 +601,8 @@ def oracle_data(w: W.Workload):
 
 
 def oracle_value(w: W.Workload, sel, rows, seconds: float) -> float:
-    sel_tokens = [sum(min(64, w.N - 64 * int(b)) for b in sel[h][0]) for h in range(w.H)]
-    fl = step_flops(w, sel_tokens)
+    sel_tokens = sum(min(64, w.N - 64 * int(b)) for h in range(w.H) for b in sel[h][0])
+    fl = step_flops(w, w.Lq * sel_tokens)
     frac = len(rows) / w.Lq
     flops = fl["forward"] * frac + fl["select"] + fl["append"] * w.n_chunks  # state built from scratch
     return flops / seconds / 1e12
@@ -525,13 +612,16 @@ def cpu_baseline(w: W.Workload, rows: int = 256) -> dict:
     import numpy as np
     data = oracle_data(w)
     r = np.sort(W.random_rows(w, rows).numpy())
-    secs = []
+    secs, stage_sum = [], {}
     while sum(secs) < 10.0 and len(secs) < 8:      # about 10 s of CPU work in all
-        sec, sel = oracle_step(w, data, r)
+        sec, sel, stages = oracle_step(w, data, r)
         secs.append(sec)
+        for k2, v2 in stages.items():
+            stage_sum[k2] = stage_sum.get(k2, 0.0) + v2
     sec = sum(secs) / len(secs)
     return {"value": oracle_value(w, sel, r, sec), "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
             "kind": "oracle", "seconds": sec, "repeats": len(secs),
+            "stage_seconds": {k2: v2 / len(secs) for k2, v2 in stage_sum.items()},
             "sample": f"block selection over the full {w.N}-token history + linear state from scratch + both "
                       f"branches and merge on {len(r)} seeded query rows of {w.Lq}; algorithmic FLOPs of that "
                       "sample / wall time"}
@@ -550,7 +640,7 @@ def bench_reference(args, rank: int, world: int):
         oracle_step(w, data, r)
     secs = []
     for _ in range(K):
-        s, sel = oracle_step(w, data, r)
+        s, sel, _ = oracle_step(w, data, r)
         secs.append(s)
     sec = sum(secs) / len(secs)
     val = oracle_value(w, sel, r, sec)
@@ -561,8 +651,7 @@ def bench_reference(args, rank: int, world: int):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{w.name}: H={w.H} d={w.d} chunk={w.Lq} history={w.N} tokens "
-                               f"({w.n_blocks} blocks of 64) top-{w.topk} blocks/head", "sample": sample},
+        "config": {"workload": workload_desc(w)},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}), flush=True)
@@ -571,7 +660,9 @@ def bench_reference(args, rank: int, world: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=6000,
+                    help="timed steps (the default makes the timed region about a second long, so that the "
+                         "clock samples belong to it)")
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
@@ -579,20 +670,63 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="rollout workloads: number of layers (0 = the workload's)")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="how the timed steps are issued: replayed CUDA graphs (default) or call by call")
+    ap.add_argument("--group-tokens", type=int, default=0,
+                    help="0: one selection per head for the whole chunk; 128: one per 128-row query tile")
+    ap.add_argument("--lin", default="state", choices=["state", "linformer"],
+                    help="linear branch: the running-state form (measured configuration) or the Linformer form")
+    ap.add_argument("--lin-rank", type=int, default=256, help="Linformer projection rank")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", action="store_true",
                     help="profiling run: set-up, warm-up and the K timed steps only (no clock probe loop, "
                          "no end-to-end loop, no CPU baseline), for use under ncu")
+    ap.add_argument("--rank-check", action="store_true",
+                    help="start the ranks, let them meet over gloo and report the aggregation of stand-in "
+                         "numbers, then exit before any GPU is touched (checks the launcher on a CPU box)")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be >= 1")
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl == "ours":
+        # started by hand with --gpus N: start the N ranks ourselves (one process per GPU)
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.impl == "ours" and world != args.gpus:
+        sys.exit(f"bench: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if args.rank_check:
+        rank_check(rank, world)
+    elif args.impl == "reference":
         bench_reference(args, rank, world)
     elif W.WORKLOADS[args.workload].layers > 1:
         if rank == 0:
             bench_rollout(args, rank, world)
     else:
         bench_ours(args, rank, world)
+
+
+def rank_check(rank: int, world: int) -> None:
+    """The multi-rank bookkeeping of bench_ours without a GPU: rendezvous, barrier, whole-job
+    throughput of stand-in numbers (rank r: 1 unit of work in 1 + r seconds)."""
+    import torch.distributed as dist
+    from paper_2609_34606_b200 import sharding
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    thr, slowest = sharding.aggregate_throughput(1.0, 1.0 + rank)
+    if rank == 0:
+        print(json.dumps({"rank_check": True, "n_gpus": world, "local_rank": int(os.environ.get("LOCAL_RANK", "0")),
+                          "value": thr, "slowest_s": slowest}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n: int, argv, env=None) -> int:
+    """Runs this script as n ranks under torch.distributed.run on this node (rendezvous on 127.0.0.1);
+    returns the launcher's exit code."""
+    port = 29500 + os.getpid() % 2000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd, env=env)
 
 
 if __name__ == "__main__":

@@ -49,3 +49,22 @@ def test_two_ranks_gloo():
     assert l0 == list(range(15)) and l1 == list(range(15, 30))
     assert slow0 == slow1 == 2.0 and thr0 == thr1 == 30.0 / 2.0
     assert mx0 == mx1 == [2.0, 10.0]
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself; with --rank-check they meet over
+    gloo, aggregate stand-in numbers (2 units of work over the slower rank's 2 s) and stop before any
+    GPU is touched.  A rank count that contradicts the launcher's is refused."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--rank-check"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["value"] == 1.0 and lines[0]["slowest_s"] == 2.0
+    bad = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4", "--rank-check"],
+                         capture_output=True, text=True, env=dict(env, WORLD_SIZE="2", RANK="0"), timeout=120)
+    assert bad.returncode != 0 and "--gpus 4" in bad.stderr
