@@ -237,21 +237,6 @@ __global__ void state_reduce_kernel(AppendArgs a) {
 // and finally the CTA writes its partial S and z for the fixed-order reduction of stage C.
 // Every wait is bounded; on expiry the CTA records a timeout and leaves.
 // ---------------------------------------------------------------------------------------
-#ifdef HSA_TIMING
-__device__ long long g_af_timing[1024];
-#define AF_T(slot)                                                                   \
-  do {                                                                               \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (slot) < 1024) { \
-      long long t_;                                                                  \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                          \
-      g_af_timing[(slot)] = t_;                                                      \
-    }                                                                                \
-  } while (0)
-#else
-#define AF_T(slot) \
-  do {             \
-  } while (0)
-#endif
 
 namespace {
 
@@ -328,7 +313,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
 
   const int h = blockIdx.y, split = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp == 0) AF_T(0);
   const int64_t b_first = a.n0 / kBlock, b_last = (a.n0 + a.n_new - 1) / kBlock;
   const int64_t bs = b_first + static_cast<int64_t>(split) * blocks_per_cta;
   const int64_t be = min64(b_last + 1, bs + blocks_per_cta);
@@ -375,7 +359,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  if (warp == 0) AF_T(1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (one lane)
@@ -385,7 +368,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
         const int s = bi % kAfDepth;
         ok = af_wait(&bars->full[s], (bi / kAfDepth) & 1, bars, a.status);
         if (!ok) break;
-        AF_T(16 + bi * 8 + 0);
         const int64_t b = bs + bi;
         if (b * kBlock >= a.n0) {  // the block holds nothing older: whole tiles go to its page
           uint8_t* st = ring + s * kAfStage;
@@ -396,18 +378,14 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
           tma_store_2d(&tm_vpool, st + kAfTile + kAfTile / 2, 64, prow);
         }
         tma_store_commit();
-        AF_T(16 + bi * 8 + 1);
         if (bi >= 1 && bi - 1 + kAfDepth < nblk) {
           // refill the stage of block bi - 1: its stores have read it, the tensor cores are done
           asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-          AF_T(16 + bi * 8 + 2);
           ok = af_wait(&bars->consumed[(bi - 1) % kAfDepth], ((bi - 1) / kAfDepth) & 1, bars, a.status);
-          AF_T(16 + bi * 8 + 3);
           if (ok) issue_loads(bi - 1 + kAfDepth);
         }
       }
       asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // every page write has landed
-      AF_T(2);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (one lane)
@@ -419,7 +397,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
       for (int bi = 0; bi < nblk; ++bi) {
         const int s = bi % kAfDepth, hb = bi & 1;
         if (!af_wait(&bars->phi_ready[hb], (bi >> 1) & 1, bars, a.status)) break;
-        AF_T(256 + bi * 4 + 0);
         tc_fence_after();
         uint8_t* st = ring + s * kAfStage;
         const uint32_t a_k = desc_lo_sw128(smem_u32(st), kAfTile / 2);
@@ -443,7 +420,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
           tc_mma_ss_lo(tmem + kAfColKs + hb * 16, a_k + kk * 128, b_ones, hi, idesc_1, kk > 0 ? 1u : 0u);
         tc_commit(&bars->consumed[s]);
         tc_commit(&bars->mma_done[hb]);
-        AF_T(256 + bi * 4 + 1);
       }
     }
   } else if (warp >= 2 + kAfWorkers / 32) {
@@ -485,7 +461,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
       const int64_t b = bs + bi;
       ok = af_wait(&bars->full[s], (bi / kAfDepth) & 1, bars, a.status);
       if (!ok) break;
-      if (warp == 2) AF_T(512 + bi * 4 + 0);
       const uint8_t* st_k = ring + s * kAfStage;
       uint4 kreg[4];
 #pragma unroll
@@ -509,7 +484,6 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
         ok = af_wait(&bars->mma_done[hb], ((bi >> 1) - 1) & 1, bars, a.status);
         if (!ok) break;
       }
-      if (warp == 2) AF_T(512 + bi * 4 + 1);
       uint8_t* st_hi = hilo + hb * kAfHilo;
       uint8_t* st_lo = st_hi + kAfTile;
       // rows outside the chunk (only in its first and last block) add nothing to the state
@@ -537,13 +511,11 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
       }
       fence_proxy_async_smem();  // generic-proxy writes above -> visible to the tensor cores
       mbar_arrive(&bars->phi_ready[hb]);
-      if (warp == 2) AF_T(512 + bi * 4 + 2);
     }
     // the partial state, once every MMA is done: the last two blocks' barriers, in block order (a
     // group has not watched the other group's barrier, so it must not skip a phase of it)
     for (int bj = max(0, nblk - 2); bj < nblk && ok; ++bj)
       ok = af_wait(&bars->mma_done[bj & 1], (bj >> 1) & 1, bars, a.status);
-    if (warp == 2) AF_T(3);
     tc_fence_after();
     float* out = a.spart + (static_cast<size_t>(h) * a.nsplit + split) * (D * D + D);
     const int row = quad * 32 + lane;
@@ -582,21 +554,13 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
       out[D * D + row] = __uint_as_float(v[0]);
     }
   }
-  if (warp == 2) AF_T(4);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, kAfTmemCols);
   }
-  if (warp == 0) AF_T(5);
 }
-
-#ifdef HSA_TIMING
-extern "C" int hsa_debug_read_af_timing(long long* host_out, int n) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_af_timing, sizeof(long long) * n));
-}
-#endif
 
 cudaError_t append_init() {
   return cudaFuncSetAttribute(append_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);

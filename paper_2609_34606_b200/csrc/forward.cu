@@ -34,13 +34,8 @@ namespace hsa {
 
 namespace {
 
-#ifndef HSA_GROUPS
-#define HSA_GROUPS 2
-#endif
-#ifndef HSA_SMREGS
-#define HSA_SMREGS 224
-#endif
-constexpr int kGroups = HSA_GROUPS;  // softmax groups; group g takes the KV steps j = g (mod kGroups)
+constexpr int kGroups = 2;     // softmax groups; group g takes the KV steps j = g (mod kGroups)
+constexpr int kSoftmaxRegs = 224;  // registers per softmax thread after the hand-over (56 for the others)
 constexpr int kThreads = 128 + 128 * kGroups;
 constexpr int kStages = 3;   // K ring and V ring depth
 constexpr int kSBufs = 3;    // score buffers in TMEM
@@ -82,34 +77,7 @@ struct Bars {
 };
 static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory slot");
 
-#ifndef HSA_INTERLEAVE
-#define HSA_INTERLEAVE 8
-#endif
-#ifndef HSA_L2AHEAD
-#define HSA_L2AHEAD 1
-#endif
-#ifndef HSA_PDL
-#define HSA_PDL 1
-#endif
-#ifndef HSA_CONTINUOUS
-#define HSA_CONTINUOUS 8
-#endif
-#ifdef HSA_TIMING
-#ifndef HSA_T_BX
-#define HSA_T_BX 0
-#define HSA_T_BY 0
-#endif
-__device__ long long g_hsa_timing[4096];
-#define HSA_T(slot)                                                      \
-  do {                                                                   \
-    if (blockIdx.x == HSA_T_BX && blockIdx.y == HSA_T_BY && lane == 0 && (slot) < 4096) \
-      g_hsa_timing[(slot)] = clock64();                                  \
-  } while (0)
-#else
-#define HSA_T(slot) \
-  do {              \
-  } while (0)
-#endif
+constexpr int kExpLag = 8;  // columns between scale-and-shift, exponential and row sum in the softmax pipeline
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
@@ -198,7 +166,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   float* stats = reinterpret_cast<float*>(smem + L::kStats);  // [group][row][l, den, -, -]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp == 4) HSA_T(3000);
   // barriers, TMEM allocation and the CTA-wide barrier that publishes them
   auto setup = [&]() {
     if (threadIdx.x == 0) {
@@ -218,9 +185,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   // read before the wait; the plain kernel does its set-up first, under that kernel's tail (a split
   // CTA may still leave without any set-up, so it sets up after it has seen its list).
   if (!SPLIT) setup();
-#if HSA_PDL
   asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
   const int tile = blockIdx.x, h = blockIdx.y;
   const int row0 = tile * kTileM;
   const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
@@ -250,7 +215,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (SPLIT) setup();
   const uint32_t tmem = bars->tmem_base;
-  if (warp == 4) HSA_T(3001);
 
   // attempt 0: fast pass (fixed exponent reference); attempt 1 only if a step overflowed: safe
   // pass.  Both role branches run the same attempt loop and meet at the same CTA-wide barriers.
@@ -272,9 +236,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < 4) {
     // Register budget: the CTA is allocated 168 x 384 registers.  The 128 threads here give back
-    // 168 - 56 each (14336), exactly what the 256 softmax threads take to reach 224 (HSA_SMREGS);
+    // 168 - 56 each (14336), exactly what the 256 softmax threads take to reach 224 (kSoftmaxRegs);
     // a split that asks for more than is given back would block at setmaxnreg.inc for ever.
-    static_assert(128 * (168 - 56) >= 256 * (HSA_SMREGS - 168), "setmaxnreg.inc would never be satisfied");
+    static_assert(128 * (168 - 56) >= 256 * (kSoftmaxRegs - 168), "setmaxnreg.inc would never be satisfied");
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
 #pragma unroll 1
     for (int attempt = 0; attempt < 2; ++attempt) {
@@ -354,7 +318,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
         }
       }
-    } else if (HSA_L2AHEAD && warp == 2 && attempt == 0) {
+    } else if (warp == 2 && attempt == 0) {
       // ================================================================= L2 look-ahead
       // The tiles of a (head, group) walk through the same list at about the same time.  Each of
       // them asks a slice of the list (entries tile-in-group, + tiles-per-group, ...) into L2 when
@@ -377,7 +341,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t q_lo = desc_lo_sw128(smem_u32(smem + L::kQ), 16);
         bool ok = wait_bar(&bars->q_full, 0, bars, p.status);
         tc_fence_after();
-        HSA_T(3011);
         auto issue_qk = [&](int j) -> bool {
           const int s = j % kStages;
           if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
@@ -408,14 +371,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
           const int b = j % kSBufs;
-          HSA_T(2048 + j * 8 + 0);
           ok = wait_bar(&bars->p_full[b], (j / kSBufs) & 1, bars, p.status);
           if (!ok) break;
-          HSA_T(2048 + j * 8 + 1);
           ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
           if (!ok) break;
           tc_fence_after();
-          HSA_T(2048 + j * 8 + 2);
           constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
           const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
           const uint32_t o_acc = tmem + kColO;
@@ -431,11 +391,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           tc_commit(&bars->v_empty[s]);
           tc_commit(&bars->pv_done);
-          HSA_T(2048 + j * 8 + 3);
           // the scores of step j+3 overwrite the P just consumed: issued after the P V above,
           // the tensor pipe runs them in order
           if (j + kSBufs < nsteps) ok = issue_qk(j + kSBufs);
-          HSA_T(2048 + j * 8 + 4);
         }
         if (ok) tc_commit(&bars->o_done);
         if (ok && p.do_linear) {
@@ -462,11 +420,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       safe = true;
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(HSA_SMREGS));
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
 #pragma unroll 1
     for (int attempt = 0; attempt < 2; ++attempt) {
       // ================================================================= softmax groups + epilogue
-      const int grp = (warp - 4) >> 2;  // group g takes the steps j = g (mod 3)
+      const int grp = (warp - 4) >> 2;  // group g takes the steps j = g (mod 2)
       const int quad = warp & 3;        // TMEM lane quadrant this warp may access
       const int r = quad * 32 + lane;   // row inside the tile
       const int row = row0 + r;         // query index inside the chunk
@@ -498,7 +456,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
         // and kept in registers until the epilogue
         ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
-        if (quad == 0) HSA_T(3012 + grp);
         const uint8_t* qrow = smem + L::kQ + r * 128;
         const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
 #pragma unroll
@@ -521,7 +478,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         den_part += den_part2;
       }
 
-      if (quad == 0) HSA_T(3014 + grp);
       // block ids of the next step are fetched one step ahead, off the critical path
       int nb0 = 0, nb1 = 0;
       if (first < nsteps) {
@@ -537,11 +493,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         const int b = j % kSBufs;
         const uint32_t s_tmem = tmem + lane_off + kColS + 128 * b;
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 0);
         ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], (j / kSBufs) & 1, bars, p.status));
         if (!ok) break;
         tc_fence_after();
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 1);
         uint32_t cbuf[2][32];  // two 32-column chunks of the score row in flight
         // the first chunk is requested at once: its latency runs under the bookkeeping below
         // (the steps that look for the row maximum first issue their own loads)
@@ -623,25 +577,22 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             t_ref = (m_used == -INFINITY) ? 0.f : m_used * sl2;
           }
         } else if (j < kGroups) {
-          // first step of groups 1 and 2 in the fast pass: take the reference group 0 fixed
+          // first step of group 1 in the fast pass: take the reference group 0 fixed
           ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready, 0, bars, p.status));
           if (!ok) break;
           t_ref = bars->mref[r];
         }
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 2);
         // exponentials in four chunks of 32 columns: the load of the next chunk and the store of
         // the previous P chunk run under the arithmetic of the current one
         const float nt = -t_ref;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial row sums
         if (!early_ld) tmem_ld32(s_tmem, cbuf[0]);
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 3);
-#if HSA_CONTINUOUS
         if (nchunks == 4 && !need_mask) {
           // full, unmasked step (the usual case): ONE software pipeline over the 128 columns --
           // scale-and-shift of column i, exponential of column i - LAG, row sum and bf16 pack of
           // column i - 2 LAG -- that does not drain at the chunk boundaries; the TMEM load of the next
           // chunk is issued when the pipeline enters a chunk, the P store when it leaves one
-          constexpr int LAG = HSA_CONTINUOUS;
+          constexpr int LAG = kExpLag;
           float y[128];
           uint32_t pk[2][16];
 #pragma unroll
@@ -662,7 +613,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
           }
         } else
-#endif
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           if (c < nchunks) {
@@ -681,7 +631,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             // two exponentials (the SFU takes one warp instruction per 8 cycles)
             float y[32];
             uint32_t pk[16];
-            constexpr int LAG = HSA_INTERLEAVE;
+            constexpr int LAG = kExpLag;
             constexpr int LAG2 = LAG;
 #pragma unroll
             for (int i = 0; i < 32 + LAG + LAG2; ++i) {
@@ -694,7 +644,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               }
             }
             tmem_st16(s_tmem + 16 * c, pk);
-            if (quad == 0) HSA_T(3100 + grp * 256 + (j / kGroups) * 8 + c);
           }
         }
         {
@@ -703,11 +652,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           // a weight far above the fixed reference: finite here, but the tile is redone safely
           if (!safe && !(lstep <= kRedoSum)) bars->redo = 1;
         }
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 4);
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(&bars->p_full[b]);
-        if (quad == 0) HSA_T(grp * 1024 + (j / kGroups) * 8 + 5);
       }
 
       // ---------------------------------------------------------------- epilogue
@@ -716,7 +663,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
         tc_fence_after();
       }
-      if (quad == 0) HSA_T(3002 + grp);
       if (ok && p.do_linear && epi) {
         if constexpr (D == 128) {
           tmem_st32(tmem + lane_off + kColPhi + grp * 32, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
@@ -730,7 +676,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // publish this group's partial row sum and denominator, then read the other group's
       stats[(grp * 128 + r) * 4 + 0] = l;
       stats[(grp * 128 + r) * 4 + 1] = den_part;
-      if (quad == 0) HSA_T(3004 + grp);
       named_bar_sync(1, 128 * kGroups);
       float lsum = 0.f, den = 0.f;
 #pragma unroll
@@ -803,7 +748,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
         tc_fence_after();
       }
-      if (quad == 0) HSA_T(3006 + grp);
       // The output tile is staged in the Q tile's shared memory.  A tile with no step and no linear
       // branch has not looked at Q at all: its TMA load may still be in flight and must land first.
       if (ok && epi && nsteps == 0 && !p.do_linear)
@@ -859,7 +803,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           uint32_t oa[16], ln[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) oa[i] = ln[i] = 0u;
-          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 0);
           if (SPLIT && nsplit > 1) {
             // merged accumulator: sum over the parts of factor * partial, from the dumps
             float acc[16];
@@ -886,7 +829,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
           tc_wait_ld();
-          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 1);
           uint32_t packed[8];
           {
           // gate weights and causal partials are fetched under ONE branch each per trip (a branch
@@ -943,7 +885,6 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             packed[i >> 1] = pack_bf16(res[0], res[1]);
           }
           }
-          if (quad == 0) HSA_T(3040 + grp * 16 + ((c0 - cbase) / 16) * 3 + 2);
           // stage the row into the Q tile's shared memory (dead by now; each thread touches only
           // its own row) in the 128-byte-swizzled layout the output tensor map expects
           {
@@ -967,24 +908,17 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tma_store_wait_read();  // the tile must stay in shared memory until it has been read
         }
       }
-      if (quad == 0) HSA_T(3008 + grp);
       if (!end_of_attempt()) break;
       safe = true;
     }
   }
 
-  if (warp == 4) HSA_T(3010);
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
 }
 
-#ifdef HSA_TIMING
-extern "C" int hsa_debug_read_timing(long long* host_out, int n) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_hsa_timing, sizeof(long long) * n));
-}
-#endif
 
 cudaError_t forward_init() {
   cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128, false>,
@@ -1016,7 +950,7 @@ cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q, c
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = HSA_PDL ? 1 : 0;
+  cfg.numAttrs = 1;
   if (D == 128) {
     if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, true>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
     return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, false>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
