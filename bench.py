@@ -169,7 +169,7 @@ def bench_ours(args, rank: int, world: int):
                       e_k=ek.to(dev), e_v=ev.to(dev))
     ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk),
                          max_topk=w.n_blocks if w.budget_set else max(w.topk, 1),
-                         page_order=W.gen_page_order(w, w.n_blocks), device=dev, **lin_kw)
+                         page_order=W.gen_page_order(w, w.n_blocks), device=dev, split_blocks=args.split_blocks, **lin_kw)
     for c in range(w.n_chunks - 1):
         k, v = W.gen_kv_chunk(w, c, layer=rank)
         ctx.append_kv(k.to(dev), v.to(dev))
@@ -660,8 +660,8 @@ def bench_reference(args, rank: int, world: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=6000,
-                    help="timed steps (the default makes the timed region about a second long, so that the "
+    ap.add_argument("--steps", type=int, default=3000,
+                    help="timed steps (the default makes the timed region about half a second long, so that the "
                          "clock samples belong to it)")
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -675,6 +675,8 @@ def main():
     ap.add_argument("--lin", default="state", choices=["state", "linformer"],
                     help="linear branch: the running-state form (measured configuration) or the Linformer form")
     ap.add_argument("--lin-rank", type=int, default=256, help="Linformer projection rank")
+    ap.add_argument("--split-blocks", type=int, default=0,
+                    help="blocks per part when a long list is split over several CTAs (0 = the library's default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", action="store_true",
                     help="profiling run: set-up, warm-up and the K timed steps only (no clock probe loop, "

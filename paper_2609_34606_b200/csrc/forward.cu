@@ -186,7 +186,55 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   // CTA may still leave without any set-up, so it sets up after it has seen its list).
   if (!SPLIT) setup();
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int tile = blockIdx.x, h = blockIdx.y;
+  int tile = blockIdx.x, h = blockIdx.y, part = blockIdx.z;
+  // Parts of a list of `st` two-page steps.  balance > 0: the steps one SM would run if the whole
+  // launch were spread evenly; a list is cut into the fewest parts none of which is longer than that
+  // (no part shorter than 16 steps).  balance == 0: parts of split_blocks blocks.
+  auto parts_of = [&](int st, int balance) -> int {
+    const int want = balance > 0 ? min((st + balance - 1) / balance, max(1, st / 16))
+                                 : (st + p.split_blocks / 2 - 1) / (p.split_blocks / 2);
+    int ns = min(p.max_splits, max(1, want));
+    const int per = (st + ns - 1) / ns;
+    if (per > 0) ns = (st + per - 1) / per;  // no empty part
+    return ns;
+  };
+  int balance = 0;
+  if (SPLIT && p.remap) {
+    // Longest lists first.  With one list per head every (tile, part) of a head costs the same, so the
+    // heads are ranked by the steps one part of theirs takes and the grid walks through them in that
+    // order (part-major inside a head: CTAs that run side by side gather the same pages); the heavy
+    // parts start in the first wave and the short lists fill the tail.  Every warp works the mapping
+    // out for itself from the H list lengths (a few dozen shuffles), so nothing has to be shared.
+    const int n_tiles = p.n_tiles;
+    int my_cnt = (lane < p.H && p.do_sparse) ? p.sel_cnt[lane] : 0;
+    my_cnt = max(0, min(my_cnt, min(p.kcap, p.n_blocks)));
+    const int st = (my_cnt + 1) / 2;
+    int total = st;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    balance = max(1, static_cast<int>((static_cast<int64_t>(total) * n_tiles + p.nsm - 1) / p.nsm));
+    const int ns = parts_of(st, balance);
+    const int per = (st + ns - 1) / ns;
+    const int n_items = lane < p.H ? ns * n_tiles : 0;
+    int rank = 0;
+    for (int i = 0; i < p.H; ++i) {
+      const int other = __shfl_sync(0xffffffffu, per, i);
+      rank += (other > per || (other == per && i < lane)) ? 1 : 0;
+    }
+    int start = 0;
+    for (int i = 0; i < p.H; ++i) {
+      const int r_i = __shfl_sync(0xffffffffu, rank, i), n_i = __shfl_sync(0xffffffffu, n_items, i);
+      if (r_i < rank) start += n_i;
+    }
+    const int lin = static_cast<int>(blockIdx.x);  // (one-dimensional grid of nsm + H * n_tiles CTAs: the
+                                                   // balance rule never makes more parts than that)
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < p.H && lin >= start && lin < start + n_items);
+    if (hit == 0u) return;  // beyond the last real work item
+    h = __ffs(hit) - 1;
+    const int local = lin - __shfl_sync(0xffffffffu, start, h);
+    part = local / n_tiles;
+    tile = local % n_tiles;
+  }
   const int row0 = tile * kTileM;
   const int g = p.group_tokens > 0 ? row0 / p.group_tokens : 0;
   const int32_t* sel = p.sel_idx + (static_cast<size_t>(h) * p.n_groups + g) * p.kcap;
@@ -195,13 +243,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   // A long list is split over the CTAs (tile, head, 0 .. nsplit - 1): each takes a run of whole
   // two-page steps; CTAs beyond nsplit leave before they set anything up.
   int nsplit = 1;
-  const int part = blockIdx.z;
-  if (SPLIT && gridDim.z > 1) {
+  if (SPLIT && p.max_splits > 1) {
     const int steps_total = (cnt + 1) / 2;
-    const int split_steps = p.split_blocks / 2;
-    nsplit = min(static_cast<int>(gridDim.z), max(1, (steps_total + split_steps - 1) / split_steps));
+    nsplit = parts_of(steps_total, balance);
     const int steps_per = (steps_total + nsplit - 1) / nsplit;
-    if (steps_per > 0) nsplit = (steps_total + steps_per - 1) / steps_per;  // no empty part
     if (part >= nsplit) return;
     if (nsplit > 1) {
       const int b_lo = 2 * part * steps_per;
@@ -210,7 +255,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       cnt = b_hi - b_lo;
     }
   }
-  const int slot = (tile * p.H + h) * static_cast<int>(gridDim.z) + part;  // this CTA's partial-result slot
+  const int slot = (tile * p.H + h) * p.max_splits + part;  // this CTA's partial-result slot
   const int nsteps = (cnt + 1) / 2;
 
   if (SPLIT) setup();
@@ -324,7 +369,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // them asks a slice of the list (entries tile-in-group, + tiles-per-group, ...) into L2 when
       // it starts, so that between them the whole list is on its way long before the rings reach it.
       if (!SPLIT && p.k_pool != nullptr && elect_one_sync()) {  // (split tiles: measured slower with it)
-        const int n_tiles = static_cast<int>(gridDim.x);
+        const int n_tiles = p.n_tiles;
         const int tpg = p.group_tokens > 0 ? max(1, p.group_tokens / kTileM) : n_tiles;  // tiles per group
         for (int e = kStages * 2 + tile % tpg; e < cnt; e += tpg) {
           const int blk = sel[e];
@@ -935,12 +980,18 @@ cudaError_t forward_init() {
   return e;
 }
 
-cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+cudaError_t launch_forward(const FwdParams& p_in, int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                            const CUtensorMap& tm_v, const CUtensorMap& tm_state, const CUtensorMap& tm_out,
                            cudaStream_t st) {
-  const int n_tiles = (p.n_q + kTileM - 1) / kTileM;
-  dim3 grid(n_tiles, p.H, p.max_splits > 1 ? p.max_splits : 1);
+  const int n_tiles = (p_in.n_q + kTileM - 1) / kTileM;
+  FwdParams p = p_in;
+  p.n_tiles = n_tiles;
   const bool split = p.max_splits > 1;
+  // One list per head and few heads: the split kernel ranks the heads itself and walks a
+  // one-dimensional grid longest lists first; its balance rule makes at most nsm + H * n_tiles parts.
+  p.remap = split && p.n_groups == 1 && p.H <= 32;
+  dim3 grid(n_tiles, p.H, split ? p.max_splits : 1);
+  if (p.remap) grid = dim3(p.nsm + p.H * n_tiles);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(kThreads);

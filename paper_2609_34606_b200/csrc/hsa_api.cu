@@ -553,6 +553,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   p.do_sparse = do_sparse;
   p.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   p.max_splits = 1;
+  p.nsm = ctx->nsm;
   p.k_pool = static_cast<const uint8_t*>(ctx->buf.k_pool);
   p.v_pool = static_cast<const uint8_t*>(ctx->buf.v_pool);
   if (do_sparse && ctx->lay.fwd_splits > 1) {

@@ -121,6 +121,8 @@ struct FwdParams {
   // (grid z = max_splits); each dumps its unnormalised O, row sums and exponent references, the last
   // one to take a ticket merges them and writes the output
   int max_splits, split_blocks;
+  int n_tiles, remap;    // set by the launcher: query tiles; 1 = one-dimensional grid, longest lists first
+  int nsm;               // SMs of the device (the split rule balances the launch over them)
   float* part_o;         // [tiles][H][max_splits][128][D]
   float* part_l;         // [tiles][H][max_splits][128]
   float* part_ref;       // [tiles][H][max_splits][128]
