@@ -9,6 +9,7 @@
 #include <cmath>
 #include <mutex>
 
+#include "grid_sync.cuh"
 #include "hsa_internal.h"
 
 namespace hsa {
@@ -526,52 +527,12 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
 // The three stages in ONE cooperative launch (all CTAs co-resident): query tile sums, grid
 // barrier, scores, grid barrier, top-k.  Saves two launches and their drain / ramp-up.
 //
-// The grid barrier lives entirely on the device: two words in the workspace, an arrive count and
-// a generation.  A CTA reads the generation, arrives, and waits for the generation to change; the
-// last CTA to arrive puts the count back to zero and advances the generation.  Nothing depends on
-// host-side bookkeeping, so a launch captured in a CUDA graph behaves the same on every replay,
-// in any order with other launches.  The wait is bounded (wait_ns): on expiry the CTA records a
-// timeout in the status word and the kernel ends with every list of the call counted as empty.
-// The host clears the two words when it reads that status (hsa_device_status).
+// The grid barrier (device_barrier: two words in the workspace, an arrive count and a generation)
+// lives entirely on the device, so a launch captured in a CUDA graph behaves the same on every
+// replay, in any order with other launches.  Its wait is bounded (wait_ns): on expiry the CTA
+// records a timeout in the status word and the kernel ends with every list of the call counted
+// as empty.  The host clears the two words when it reads that status (hsa_device_status).
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ bool grid_barrier(unsigned* bar, int32_t* status, unsigned long long wait_ns) {
-  __shared__ int bar_ok;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int ok = 1;
-    unsigned gen;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(bar + 1) : "memory");
-    __threadfence();
-    const unsigned arrived = atomicAdd(bar, 1u);
-    if (arrived == gridDim.x - 1) {
-      bar[0] = 0u;  // ordered before the new generation by the release below
-      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(bar + 1), "r"(gen + 1u) : "memory");
-    } else {
-      unsigned long long t0 = 0;
-      for (unsigned i = 0;; ++i) {
-        unsigned v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar + 1) : "memory");
-        if (v != gen) break;
-        if ((i & 63u) == 63u) {
-          unsigned long long now;
-          asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-          if (t0 == 0) t0 = now;
-          // another CTA gave up already, or this one has waited long enough
-          if (*reinterpret_cast<volatile int32_t*>(status) == kDevTimeout || now - t0 > wait_ns) {
-            atomicCAS(status, 0, kDevTimeout);
-            ok = 0;
-            break;
-          }
-        }
-      }
-    }
-    __threadfence();
-    bar_ok = ok;
-  }
-  __syncthreads();
-  return bar_ok != 0;
-}
-
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   extern __shared__ uint32_t fused_keys[];
@@ -593,7 +554,7 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
     qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
   }
-  if (!grid_barrier(a.barrier, a.status, a.wait_ns)) {
+  if (!device_barrier(a.barrier, gridDim.x, a.status, a.wait_ns)) {
     give_up();
     return;
   }
@@ -614,7 +575,7 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
       __syncthreads();
     }
   }
-  if (!grid_barrier(a.barrier, a.status, a.wait_ns)) {
+  if (!device_barrier(a.barrier, gridDim.x, a.status, a.wait_ns)) {
     give_up();
     return;
   }
