@@ -146,13 +146,42 @@ __device__ __forceinline__ int cand_visible(const CandGeom& g, int64_t p_last) {
 // ---------------------------------------------------------------------------------------
 constexpr int kScoreBlocksPerCta = 32;
 
-// rebuild = false: qs[0, D) still holds the mean query of this (group, head) from the item before
+// The key sums one item needs, per lane: candidates chunk * 32 + i * 8 + warp, dims lane * PER .. + PER - 1
+// of at most two pages each.  They depend on nothing the kernel computes, so the fused kernel asks
+// for those of its first item before the first grid barrier and lets their latency run under it.
+template <int D, bool MIXED>
+struct ScoreOperands {
+  static constexpr int PER = D / 32, NB = kScoreBlocksPerCta / 8, NP = MIXED ? 2 : 1;
+  float kv[NB][NP][PER];
+};
+template <int D, bool MIXED>
+__device__ __forceinline__ void scores_load(const SelectArgs& a, int chunk, int h, ScoreOperands<D, MIXED>& op) {
+  using O = ScoreOperands<D, MIXED>;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const CandGeom cg = cand_geom<MIXED>(a);
+#pragma unroll
+  for (int i = 0; i < O::NB; ++i) {
+    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+    const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
+    const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
+#pragma unroll
+    for (int pg = 0; pg < O::NP; ++pg)
+#pragma unroll
+      for (int e = 0; e < O::PER; ++e)
+        op.kv[i][pg][e] =
+            pg < np ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp + pg) * D + lane * O::PER + e] : 0.f;
+  }
+}
+
+// rebuild = false: qs[0, D) still holds the mean query of this (group, head) from the item before;
+// loaded = true: `op` already holds this item's key sums
 template <int D, bool MIXED>
 __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs,
-                                            bool rebuild = true) {
+                                            ScoreOperands<D, MIXED>& op, bool rebuild = true, bool loaded = false) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
+  if (!loaded) scores_load<D, MIXED>(a, chunk, h, op);  // in flight while the mean query is rebuilt
   if (rebuild) {
     // 256 / D threads per column, each summing an interleaved subset of the tile partials with
     // up to 20 loads in flight (one round trip for a chunk of up to 40 tiles at head_dim 128); the subsets are then added in a fixed order
@@ -185,18 +214,7 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
   const CandGeom cg = cand_geom<MIXED>(a);
   constexpr int NB = kScoreBlocksPerCta / 8;  // candidates per warp
   constexpr int NP = MIXED ? 2 : 1;           // pages per candidate at most
-  float kv[NB][NP][PER];
-#pragma unroll
-  for (int i = 0; i < NB; ++i) {
-    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
-    const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
-    const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
-#pragma unroll
-    for (int pg = 0; pg < NP; ++pg)
-#pragma unroll
-      for (int e = 0; e < PER; ++e)
-        kv[i][pg][e] = pg < np ? a.ksum[(static_cast<size_t>(h) * a.max_pages + fp + pg) * D + lane * PER + e] : 0.f;
-  }
+  auto& kv = op.kv;
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
     const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
@@ -338,7 +356,8 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   __shared__ double qs[D + 256];  // mean query, then the per-way partial sums
-  scores_item<D, MIXED>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs);
+  ScoreOperands<D, MIXED> op;
+  scores_item<D, MIXED>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs, op);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -550,6 +569,14 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
     for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x)
       if (threadIdx.x == 0) a.sel_cnt[it] = 0;  // it = h * n_groups + g
   };
+  // one selection per head: a CTA takes a run of consecutive (head, chunk) score items; the key sums
+  // of the first one are requested now, ahead of the query sums and the first barrier
+  const int n_items = n_chunks * a.H;
+  const int per = (n_items + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  const int it0 = static_cast<int>(blockIdx.x) * per, it1 = min(n_items, it0 + per);
+  ScoreOperands<D, MIXED> op;
+  const bool ahead = a.n_groups == 1 && it0 < it1;
+  if (ahead) scores_load<D, MIXED>(a, it0 % n_chunks, it0 / n_chunks, op);
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
     qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
@@ -562,15 +589,11 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
     for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x)
       scores_item_groups<D, MIXED>(a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
   } else {
-    // a CTA takes a run of consecutive (head, chunk) items: the mean query of a head is rebuilt
-    // from the tile partials only when the run enters the head
-    const int n_items = n_chunks * a.H;
-    const int per = (n_items + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
-    const int it0 = static_cast<int>(blockIdx.x) * per, it1 = min(n_items, it0 + per);
+    // the mean query of a head is rebuilt from the tile partials only when the run enters the head
     int h_cur = -1;
     for (int it = it0; it < it1; ++it) {
       const int h = it / n_chunks;
-      scores_item<D, MIXED>(a, it % n_chunks, 0, h, reinterpret_cast<double*>(scratch), h != h_cur);
+      scores_item<D, MIXED>(a, it % n_chunks, 0, h, reinterpret_cast<double*>(scratch), op, h != h_cur, it == it0);
       h_cur = h;
       __syncthreads();
     }
