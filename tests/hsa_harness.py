@@ -8,7 +8,7 @@ import torch
 from oracle import hsa_oracle as O
 from paper_2609_34606_b200 import workloads as W
 
-# spec tolerances for bf16 inputs with fp32 accumulation
+# tolerances of the benchmark spec for bf16 inputs with fp32 accumulation
 MAX_ABS = 2e-2
 MEAN_ABS = 2e-3
 REL_FRO = 1e-2      # additional relative check (outputs are small for N(0,1) inputs)
