@@ -63,6 +63,11 @@ typedef enum {
 #define HSA_CFG_CAUSAL 1u
 /* hsa_config.flags: reserve workspace for hsa_select_blocks_adaptive (needs max_pages <= 8192) */
 #define HSA_CFG_ADAPTIVE 2u
+/* hsa_config.flags: run the selection kernel in its grid-barrier form (one cooperative launch whose
+ * CTAs meet at two device-wide barriers in global memory) instead of the default form, in which the
+ * CTAs of a head form a thread-block cluster and meet at hardware cluster barriers.  The library
+ * falls back to the grid-barrier form by itself where clusters of 8 CTAs cannot be launched. */
+#define HSA_CFG_GRID_BARRIER_SELECT 4u
 
 /* hsa_forward flags: the paper's "linear only" / "sparse only" ablation modes (Table 4) */
 #define HSA_FWD_NO_LINEAR 1u

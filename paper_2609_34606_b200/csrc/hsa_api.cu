@@ -419,6 +419,7 @@ int hsa_select_blocks_ex(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_s
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   a.barrier = reinterpret_cast<unsigned*>(ws + ctx->lay.status + 8);
   a.wait_ns = ctx->wait_ns;
+  a.use_clusters = (ctx->cfg.flags & HSA_CFG_GRID_BARRIER_SELECT) ? 0 : 1;
   if (opts) {
     a.inter_pages = opts->inter_block_pages;
     a.intra_first_page1 = opts->intra_first_page >= 0 ? static_cast<int64_t>(opts->intra_first_page) + 1 : 0;

@@ -68,6 +68,7 @@ struct SelectArgs {
   unsigned* barrier;  // grid barrier of the single-launch path: {arrive count, generation}, the count
                       // zero when no launch is in flight (null: three launches)
   unsigned long long wait_ns;  // bound of a wait at that barrier
+  int use_clusters;            // 1: one thread-block cluster per head (hardware cluster barriers) where the device allows
   // candidate geometry: pages before the first intra-chunk page are selected in runs of inter_pages pages against
   // budgets[], the pages from it on one by one against intra_budgets[] (null: all of them)
   int inter_pages;           // 0 or 1: every page on its own

@@ -1,9 +1,10 @@
 // hsa_select_blocks kernels: mean query per group, pooled block scores
 //   s[h,g,b] = mean_q(g) . (Ksum[h,b] / cnt_b) * scale
 // and an exact per-(head, group) top-k by radix select, all on the device:
-// query partial sums -> scores (many CTAs) -> top-k (one CTA per head and group).
-// The three stages run as one cooperative launch with two grid barriers where the device
-// supports it, else as three launches.
+// query partial sums -> scores (many CTAs) -> top-k (one block of 256 threads per head and group).
+// The stages run in one of three forms (see launch_select): a kernel for the query sums followed
+// by one thread-block cluster per head, one cooperative launch with two grid barriers, or three
+// launches.
 #include <cuda_bf16.h>
 
 #include <cmath>
@@ -14,14 +15,25 @@
 
 namespace hsa {
 
+// The stages below are written for a block of 256 threads.  That block is either a whole CTA (tid =
+// threadIdx.x, barrier 0) or one of several sub-blocks of a larger CTA, each with its own named
+// barrier (the cluster form of the fused kernel runs three of them per CTA).
+struct Blk {
+  int tid;  // 0..255 inside the block
+  int bar;  // named barrier of the block
+};
+__device__ __forceinline__ void blk_sync(const Blk& blk) {
+  asm volatile("bar.sync %0, 256;" ::"r"(blk.bar) : "memory");
+}
+
 // ---------------------------------------------------------------------------------------
 // Stage 1: column sums of q over one 128-token tile and one head -> qpart[tile][h][D].
 // ---------------------------------------------------------------------------------------
 template <int D>
-__device__ __forceinline__ void qsum_item(const SelectArgs& a, int tile, int h, float (*red)[D]) {
+__device__ __forceinline__ void qsum_item(const Blk& blk, const SelectArgs& a, int tile, int h, float (*red)[D]) {
   constexpr int CH = D / 8;
   constexpr int RP = 256 / CH;
-  const int c8 = threadIdx.x % CH, rg = threadIdx.x / CH;
+  const int c8 = blk.tid % CH, rg = blk.tid / CH;
   const int t_hi = min(a.n_q, tile * kTileM + kTileM);
   float acc[8];
 #pragma unroll
@@ -49,19 +61,23 @@ __device__ __forceinline__ void qsum_item(const SelectArgs& a, int tile, int h, 
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) red[rg][c8 * 8 + i] = acc[i];
-  __syncthreads();
-  if (threadIdx.x < D) {
+  blk_sync(blk);
+  if (blk.tid < D) {
     float s = 0.f;
 #pragma unroll
-    for (int r = 0; r < RP; ++r) s += red[r][threadIdx.x];
-    a.qpart[(static_cast<size_t>(tile) * a.H + h) * D + threadIdx.x] = s;
+    for (int r = 0; r < RP; ++r) s += red[r][blk.tid];
+    a.qpart[(static_cast<size_t>(tile) * a.H + h) * D + blk.tid] = s;
   }
 }
 
 template <int D>
 __global__ void __launch_bounds__(256) qsum_partial_kernel(SelectArgs a) {
   __shared__ float red[256 / (D / 8)][D];
-  qsum_item<D>(a, blockIdx.x, blockIdx.y, red);
+  // (no-ops unless launched with programmatic stream serialization: wait for the kernel before this
+  // one, let the kernel behind this one be scheduled early -- it waits for this grid's end itself)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  qsum_item<D>(Blk{static_cast<int>(threadIdx.x), 0}, a, blockIdx.x, blockIdx.y, red);
 }
 
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -69,18 +85,18 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // ascending with the float order
 }
 
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
-  // 256 threads; returns the exclusive prefix of v over threadIdx.x and the block total
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__device__ __forceinline__ int block_exclusive_scan(const Blk& blk, int v, int* warp_sums, int* total) {
+  // 256 threads; returns the exclusive prefix of v over blk.tid and the block total
+  const int lane = blk.tid & 31, warp = blk.tid >> 5;
   int incl = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const int n = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += n;
   }
-  __syncthreads();
+  blk_sync(blk);
   if (lane == 31) warp_sums[warp] = incl;
-  __syncthreads();
+  blk_sync(blk);
   int base = 0, tot = 0;
 #pragma unroll
   for (int w = 0; w < 8; ++w) {
@@ -155,9 +171,9 @@ struct ScoreOperands {
   float kv[NB][NP][PER];
 };
 template <int D, bool MIXED>
-__device__ __forceinline__ void scores_load(const SelectArgs& a, int chunk, int h, ScoreOperands<D, MIXED>& op) {
+__device__ __forceinline__ void scores_load(const Blk& blk, const SelectArgs& a, int chunk, int h, ScoreOperands<D, MIXED>& op) {
   using O = ScoreOperands<D, MIXED>;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = blk.tid & 31, warp = blk.tid >> 5;
   const CandGeom cg = cand_geom<MIXED>(a);
 #pragma unroll
   for (int i = 0; i < O::NB; ++i) {
@@ -176,18 +192,18 @@ __device__ __forceinline__ void scores_load(const SelectArgs& a, int chunk, int 
 // rebuild = false: qs[0, D) still holds the mean query of this (group, head) from the item before;
 // loaded = true: `op` already holds this item's key sums
 template <int D, bool MIXED>
-__device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int g, int h, double* qs,
+__device__ __forceinline__ void scores_item(const Blk& blk, const SelectArgs& a, int chunk, int g, int h, double* qs,
                                             ScoreOperands<D, MIXED>& op, bool rebuild = true, bool loaded = false) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = blk.tid & 31, warp = blk.tid >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
-  if (!loaded) scores_load<D, MIXED>(a, chunk, h, op);  // in flight while the mean query is rebuilt
+  if (!loaded) scores_load<D, MIXED>(blk, a, chunk, h, op);  // in flight while the mean query is rebuilt
   if (rebuild) {
     // 256 / D threads per column, each summing an interleaved subset of the tile partials with
     // up to 20 loads in flight (one round trip for a chunk of up to 40 tiles at head_dim 128); the subsets are then added in a fixed order
     constexpr int WAYS = 256 / D;
     constexpr int kInFlight = 20;
-    const int col = threadIdx.x % D, way = threadIdx.x / D;
+    const int col = blk.tid % D, way = blk.tid / D;
     const int tile_lo = q_lo / kTileM, tile_hi = (q_hi + kTileM - 1) / kTileM;
     double s = 0.0;
     for (int t0 = tile_lo + way; t0 < tile_hi; t0 += kInFlight * WAYS) {
@@ -200,15 +216,15 @@ __device__ __forceinline__ void scores_item(const SelectArgs& a, int chunk, int 
     }
     double* part = qs + D;  // [WAYS][D]
     part[way * D + col] = s;
-    __syncthreads();
-    if (threadIdx.x < D) {
+    blk_sync(blk);
+    if (blk.tid < D) {
       double t = 0.0;
 #pragma unroll
-      for (int w = 0; w < WAYS; ++w) t += part[w * D + threadIdx.x];
-      qs[threadIdx.x] = t / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
+      for (int w = 0; w < WAYS; ++w) t += part[w * D + blk.tid];
+      qs[blk.tid] = t / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
     }
   }
-  __syncthreads();
+  blk_sync(blk);
   constexpr int PER = D / 32;
   uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
   const CandGeom cg = cand_geom<MIXED>(a);
@@ -263,9 +279,9 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
 }
 
 template <int D, bool MIXED>
-__device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chunk, int h, double* qs) {
+__device__ __forceinline__ void scores_item_groups(const Blk& blk, const SelectArgs& a, int chunk, int h, double* qs) {
   constexpr int GB = kGroupBatch, PITCH = D + 4, KS = D / 4;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = blk.tid & 31, warp = blk.tid >> 5;
   const int gtok = a.group_tokens;  // > 0 here, a multiple of the tile height
   const CandGeom cg = cand_geom<MIXED>(a);
   const int c0 = chunk * kScoreBlocksPerCta + 8 * (warp & 3);  // this warp's eight candidates
@@ -317,7 +333,7 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
       float part[NV];  // independent loads first, then the adds
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
-        const int idx = threadIdx.x + 256 * v;
+        const int idx = blk.tid + 256 * v;
         const int g = g0 + idx / D, col = idx % D;
         const int t = g * tiles_per_group + tt;
         part[v] = (g < a.n_groups && t * kTileM < a.n_q) ? __ldcg(&a.qpart[(static_cast<size_t>(t) * a.H + h) * D + col]) : 0.f;
@@ -327,12 +343,12 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
     }
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
-      const int idx = threadIdx.x + 256 * v;
+      const int idx = blk.tid + 256 * v;
       const int gi = idx / D, g = g0 + gi;
       const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
       qs[gi * PITCH + idx % D] = g < a.n_groups ? sum[v] * (static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo)) : 0.0;
     }
-    __syncthreads();
+    blk_sync(blk);
     const int row0 = 8 * (warp >> 2);  // this warp's eight rows of the batch
     if (g0 + row0 < a.n_groups && c0 < cg.nc) {  // warp-uniform
       // A fragment: element (m = lane / 4, k = lane % 4) of every k-step
@@ -349,15 +365,17 @@ __device__ __forceinline__ void scores_item_groups(const SelectArgs& a, int chun
         if (c + 1 < cg.nc) keys[c + 1] = masked[1] ? 0u : order_key(static_cast<float>(d1 * inv_cnt[1]));
       }
     }
-    __syncthreads();
+    blk_sync(blk);
   }
 }
 
 template <int D, bool MIXED>
 __global__ void __launch_bounds__(256) block_scores_kernel(SelectArgs a) {
   __shared__ double qs[D + 256];  // mean query, then the per-way partial sums
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // (see qsum_partial_kernel)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   ScoreOperands<D, MIXED> op;
-  scores_item<D, MIXED>(a, blockIdx.x, blockIdx.y, blockIdx.z, qs, op);
+  scores_item<D, MIXED>(Blk{static_cast<int>(threadIdx.x), 0}, a, blockIdx.x, blockIdx.y, blockIdx.z, qs, op);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -377,7 +395,7 @@ struct TopkShared {
 // index order as the pages of candidates c0 + i; returns the number of pages emitted (whether or
 // not they fitted below kcap).  All 256 threads call it; keys live in shared memory.
 template <bool MIXED>
-__device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budget, const CandGeom& cg, int c0,
+__device__ __forceinline__ int topk_range(const Blk& blk, const uint32_t* keys, int n, int budget, const CandGeom& cg, int c0,
                                           int32_t* out, int out_pos0, int kcap, TopkShared* sh, bool masked) {
   int* hist = sh->hist;
   int* warp_sums = sh->warp_sums;
@@ -385,9 +403,9 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
   int n_eff = n;
   if (MIXED && masked) {
     int my0 = 0, tot0 = 0;
-    for (int b = threadIdx.x; b < n; b += 256) my0 += (keys[b] == 0u);
-    block_exclusive_scan(my0, warp_sums, &tot0);
-    __syncthreads();
+    for (int b = blk.tid; b < n; b += 256) my0 += (keys[b] == 0u);
+    block_exclusive_scan(blk, my0, warp_sums, &tot0);
+    blk_sync(blk);
     n_eff = n - tot0;
   }
   if (budget < 0 || budget > n_eff) budget = n_eff;
@@ -399,24 +417,24 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
     int krem = budget;
     for (int pass = 3; pass >= 0; --pass) {
       const int shift = pass * 8;
-      hist[threadIdx.x] = 0;
-      __syncthreads();
-      for (int b = threadIdx.x; b < n; b += 256) {
+      hist[blk.tid] = 0;
+      blk_sync(blk);
+      for (int b = blk.tid; b < n; b += 256) {
         const uint32_t k = keys[b];
         if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
       }
-      __syncthreads();
+      blk_sync(blk);
       // thread t owns bin 255 - t: an inclusive prefix over t is the count of keys in bins >= own
-      const int bin = 255 - static_cast<int>(threadIdx.x);
+      const int bin = 255 - static_cast<int>(blk.tid);
       const int mine = hist[bin];
       int tot;
-      const int above = block_exclusive_scan(mine, warp_sums, &tot);  // keys in strictly higher bins
+      const int above = block_exclusive_scan(blk, mine, warp_sums, &tot);  // keys in strictly higher bins
       if (above < krem && above + mine >= krem) {                     // exactly one thread
         sh->prefix = prefix | (static_cast<uint32_t>(bin) << shift);
         sh->krem = krem - above;  // still to take among keys matching the longer prefix
         sh->exact = (above + mine == krem);
       }
-      __syncthreads();
+      blk_sync(blk);
       prefix = sh->prefix;
       krem = sh->krem;
       mask |= 255u << shift;
@@ -430,7 +448,7 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
 
   // index-ordered compaction: thread t owns the contiguous range [t*per, t*per+per)
   const int per = (n + 255) / 256;
-  const int lo = min(n, static_cast<int>(threadIdx.x) * per), hi = min(n, lo + per);
+  const int lo = min(n, static_cast<int>(blk.tid) * per), hi = min(n, lo + per);
   const bool use_mask = per <= 32;  // the thread's range fits a 32-bit mask: ONE walk over the keys
   int ties_before = 0, dummy;
   uint32_t gt = 0, eq = 0;  // candidates above the threshold / equal to it, as bits of the range
@@ -447,11 +465,11 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
           eq |= bit;
       }
     }
-    if (!take_all && budget > 0) ties_before = block_exclusive_scan(__popc(eq), warp_sums, &dummy);
+    if (!take_all && budget > 0) ties_before = block_exclusive_scan(blk, __popc(eq), warp_sums, &dummy);
   } else if (!take_all && budget > 0) {
     int my_ties = 0;
     for (int b = lo; b < hi; ++b) my_ties += (keys[b] == thr);
-    ties_before = block_exclusive_scan(my_ties, warp_sums, &dummy);
+    ties_before = block_exclusive_scan(blk, my_ties, warp_sums, &dummy);
   }
   auto chosen = [&](int b, int& t) -> bool {
     if (take_all) return !(MIXED && masked) || keys[b] != 0u;
@@ -484,7 +502,7 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
       if (chosen(b, t)) my_pages += cand_pages<MIXED>(cg, c0 + b);
   }
   int total = 0;
-  int pos = out_pos0 + block_exclusive_scan(my_pages, warp_sums, &total);
+  int pos = out_pos0 + block_exclusive_scan(blk, my_pages, warp_sums, &total);
   auto emit = [&](int b) {
     const int fp = cand_first_page<MIXED>(cg, c0 + b);
     const int np = cand_pages<MIXED>(cg, c0 + b);
@@ -502,12 +520,12 @@ __device__ __forceinline__ int topk_range(const uint32_t* keys, int n, int budge
     for (int b = lo; b < hi; ++b)
       if (chosen(b, t)) emit(b);
   }
-  __syncthreads();  // hist / warp_sums are reused by the next call
+  blk_sync(blk);  // hist / warp_sums are reused by the next call
   return total;
 }
 
 template <bool MIXED>
-__device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
+__device__ __forceinline__ void topk_item(const Blk& blk, const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
   const CandGeom cg = cand_geom<MIXED>(a);
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_hi = min(a.n_q, g * gtok + gtok);
@@ -516,20 +534,20 @@ __device__ __forceinline__ void topk_item(const SelectArgs& a, int g, int h, uin
   // last query position
   const int ncand = a.causal ? cand_visible<MIXED>(cg, p_last) : cg.nc;
   const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
-  for (int b = threadIdx.x; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
-  if (threadIdx.x == 0) {
+  for (int b = blk.tid; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
+  if (blk.tid == 0) {
     sh->prefix = 0;
     sh->krem = 0;
   }
-  __syncthreads();
+  blk_sync(blk);
   int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
   // inter-chunk candidates against the head's budget, then intra-chunk ones against theirs
   const int n_inter = min(ncand, cg.ni);
-  int total = topk_range<MIXED>(keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh, a.kv_pages != nullptr);
+  int total = topk_range<MIXED>(blk, keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh, a.kv_pages != nullptr);
   if (MIXED && ncand > n_inter)
-    total += topk_range<MIXED>(keys + n_inter, ncand - n_inter, a.intra_budgets ? a.intra_budgets[h] : -1, cg, cg.ni, out,
+    total += topk_range<MIXED>(blk, keys + n_inter, ncand - n_inter, a.intra_budgets ? a.intra_budgets[h] : -1, cg, cg.ni, out,
                         total, a.kcap, sh, false);
-  if (threadIdx.x == 0) {
+  if (blk.tid == 0) {
     a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
     if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
   }
@@ -539,7 +557,9 @@ template <bool MIXED>
 __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   extern __shared__ uint32_t topk_keys[];
   __shared__ TopkShared sh;
-  topk_item<MIXED>(a, blockIdx.x, blockIdx.y, topk_keys, &sh);
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // (see qsum_partial_kernel)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  topk_item<MIXED>(Blk{static_cast<int>(threadIdx.x), 0}, a, blockIdx.x, blockIdx.y, topk_keys, &sh);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -560,6 +580,7 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   constexpr int kScratch = kGroupBytes > 256 / (D / 8) * D * 4 ? kGroupBytes : 256 / (D / 8) * D * 4;
   __shared__ __align__(16) unsigned char scratch[kScratch];
   __shared__ TopkShared sh;
+  const Blk blk{static_cast<int>(threadIdx.x), 0};
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
@@ -576,9 +597,9 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   const int it0 = static_cast<int>(blockIdx.x) * per, it1 = min(n_items, it0 + per);
   ScoreOperands<D, MIXED> op;
   const bool ahead = a.n_groups == 1 && it0 < it1;
-  if (ahead) scores_load<D, MIXED>(a, it0 % n_chunks, it0 / n_chunks, op);
+  if (ahead) scores_load<D, MIXED>(blk, a, it0 % n_chunks, it0 / n_chunks, op);
   for (int it = blockIdx.x; it < n_tiles * a.H; it += gridDim.x) {
-    qsum_item<D>(a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
+    qsum_item<D>(blk, a, it % n_tiles, it / n_tiles, reinterpret_cast<float(*)[D]>(scratch));
     __syncthreads();
   }
   if (!device_barrier(a.barrier, gridDim.x, a.status, a.wait_ns)) {
@@ -587,13 +608,13 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   }
   if (a.n_groups > 1) {
     for (int it = blockIdx.x; it < n_chunks * a.H; it += gridDim.x)
-      scores_item_groups<D, MIXED>(a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
+      scores_item_groups<D, MIXED>(blk, a, it % n_chunks, it / n_chunks, reinterpret_cast<double*>(scratch));
   } else {
     // the mean query of a head is rebuilt from the tile partials only when the run enters the head
     int h_cur = -1;
     for (int it = it0; it < it1; ++it) {
       const int h = it / n_chunks;
-      scores_item<D, MIXED>(a, it % n_chunks, 0, h, reinterpret_cast<double*>(scratch), op, h != h_cur, it == it0);
+      scores_item<D, MIXED>(blk, a, it % n_chunks, 0, h, reinterpret_cast<double*>(scratch), op, h != h_cur, it == it0);
       h_cur = h;
       __syncthreads();
     }
@@ -607,8 +628,82 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   // may take their places and do its set-up meanwhile.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
-    topk_item<MIXED>(a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
+    topk_item<MIXED>(blk, a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
     __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// The same three stages with the CTAs of a head forming a thread-block cluster: everything a head
+// needs -- its query tile sums, its scores, its lists -- is produced inside its cluster, so the two
+// synchronisation points are hardware cluster barriers (release / acquire at cluster scope) instead
+// of grid-wide barriers in global memory, and the launch needs no co-residency of the whole grid.
+// grid = H clusters of CS CTAs; a CTA holds kSubBlocks blocks of 256 threads, each of which takes
+// work items of its own (slot = cluster rank * kSubBlocks + sub-block), so that the 37 query tiles
+// of a head are read in one round trip.
+// ---------------------------------------------------------------------------------------
+constexpr int kSubBlocks = 3;
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <int D>
+struct ClusterSmem {
+  static constexpr int kGroupBytes = kGroupBatch * (D + 4) * 8;
+  static constexpr int kScratch = kGroupBytes > 256 / (D / 8) * D * 4 ? kGroupBytes : 256 / (D / 8) * D * 4;
+  static constexpr int kFixed = (kSubBlocks * kScratch + kSubBlocks * static_cast<int>(sizeof(TopkShared)) + 15) / 16 * 16;
+};
+
+template <int D, bool MIXED>
+__global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(SelectArgs a, int cluster_ctas, int topk_subs, int with_qsum) {
+  // dynamic shared memory: per sub-block scratch (tile-sum partials / mean query / a batch of mean
+  // queries) | per sub-block top-k bookkeeping | [topk_subs][blocks] keys
+  extern __shared__ __align__(16) unsigned char cl_smem[];
+  constexpr int kScratch = ClusterSmem<D>::kScratch;
+  const int sub = static_cast<int>(threadIdx.x) / 256;
+  const Blk blk{static_cast<int>(threadIdx.x) % 256, 1 + sub};
+  unsigned char* scratch = cl_smem + sub * kScratch;
+  TopkShared* sh_all = reinterpret_cast<TopkShared*>(cl_smem + kSubBlocks * kScratch);
+  uint32_t* cl_keys = reinterpret_cast<uint32_t*>(cl_smem + ClusterSmem<D>::kFixed);
+  const int h = static_cast<int>(blockIdx.x) / cluster_ctas;
+  const int slot = (static_cast<int>(blockIdx.x) % cluster_ctas) * kSubBlocks + sub;
+  const int n_slots = cluster_ctas * kSubBlocks;
+  // launched as a programmatic dependent: the kernel before this one is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
+  // the key sums of this block's first score item are requested ahead of the query sums
+  ScoreOperands<D, MIXED> op;
+  const bool ahead = a.n_groups == 1 && slot < n_chunks;
+  if (ahead) scores_load<D, MIXED>(blk, a, slot, h, op);
+  if (with_qsum) {
+    for (int tile = slot; tile < n_tiles; tile += n_slots) {
+      qsum_item<D>(blk, a, tile, h, reinterpret_cast<float(*)[D]>(scratch));
+      blk_sync(blk);
+    }
+    cluster_sync_all();  // the head's tile sums are complete and visible to its cluster
+  }
+  if (a.n_groups > 1) {
+    for (int chunk = slot; chunk < n_chunks; chunk += n_slots)
+      scores_item_groups<D, MIXED>(blk, a, chunk, h, reinterpret_cast<double*>(scratch));
+  } else {
+    for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
+      scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot);
+      blk_sync(blk);
+    }
+  }
+  cluster_sync_all();  // ... and so are its score keys
+  // the kernel behind this one may take the places of the CTAs that leave now
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (sub < topk_subs) {
+    const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
+    uint32_t* keys = cl_keys + static_cast<size_t>(sub) * static_cast<size_t>(nblk > 0 ? nblk : 1);
+    const int slot3 = (static_cast<int>(blockIdx.x) % cluster_ctas) * topk_subs + sub;
+    for (int g = slot3; g < a.n_groups; g += cluster_ctas * topk_subs) {
+      topk_item<MIXED>(blk, a, g, h, keys, sh_all + sub);
+      blk_sync(blk);
+    }
   }
 }
 
@@ -750,7 +845,7 @@ __global__ void __launch_bounds__(256) adaptive_pick_kernel(SelectArgs a, Adapti
   int my_sel = 0;
   for (int b = lo; b < hi; ++b) my_sel += flags[b];
   int total = 0;
-  int pos = block_exclusive_scan(my_sel, warp_sums, &total);
+  int pos = block_exclusive_scan(Blk{static_cast<int>(threadIdx.x), 0}, my_sel, warp_sums, &total);
   int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
   for (int b = lo; b < hi; ++b) {
     if (flags[b]) {
@@ -824,21 +919,115 @@ cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+namespace {
+// Cluster size (8 CTAs, the portable maximum) if the cluster form can be launched on this device for
+// the given instance and shared-memory size, else 0.
+int cluster_size_for(const void* fn, size_t smem, int threads) {
+  const int cs = 8;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(cs);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) == cudaSuccess && n >= 1) return cs;
+  cudaGetLastError();
+  return 0;
+}
+
+// One launch as a programmatic dependent of the kernel before it on the stream.
+cudaError_t launch_pdl(const void* fn, dim3 grid, dim3 block, size_t smem, void** params, cudaStream_t st,
+                       int cluster = 0, bool cooperative = false) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[3];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n++].val.programmaticStreamSerializationAllowed = 1;
+  if (cluster > 0) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[n].val.clusterDim.y = 1;
+    attr[n++].val.clusterDim.z = 1;
+  }
+  if (cooperative) {
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n++].val.cooperative = 1;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelExC(&cfg, fn, params);
+}
+}  // namespace
+
+// Three forms, all programmatic dependents of the kernel before them:
+//   cluster form        query tile sums as a kernel of their own (they read the whole chunk and want
+//                       every SM), then one cluster of 8 CTAs per head for scores and lists, with one
+//                       hardware cluster barrier between them -- the default while a head has at most
+//                       kClusterMaxChunks score items (short and medium histories)
+//   grid-barrier form   one cooperative launch over all SMs with two device barriers -- long histories
+//                       (the score stage then wants every SM too), and on request
+//   three launches      for devices without cooperative launch and for callers without a barrier word
+constexpr int kClusterMaxChunks = 2 * 8 * kSubBlocks;
+
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   int nsm = 0;
   const bool mixed = a.inter_pages > 1 || a.intra_first_page1 > 0 || a.kv_pages != nullptr;
+  const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;
+  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+  SelectArgs aa = a;
+  void* p_args[1] = {&aa};
+  const void* f_qsum = a.D == 128 ? reinterpret_cast<const void*>(qsum_partial_kernel<128>)
+                                  : reinterpret_cast<const void*>(qsum_partial_kernel<64>);
+  // candidates per head (coarse candidates make fewer; an upper bound is enough to choose the form)
+  const int64_t n_chunks_max = (nblk_all + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
+  if (a.use_clusters && n_chunks_max <= kClusterMaxChunks) {
+    const size_t key_bytes = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
+    const int topk_subs = kSubBlocks;
+    const size_t fixed = a.D == 128 ? ClusterSmem<128>::kFixed : ClusterSmem<64>::kFixed;
+    const size_t smem = fixed + key_bytes * topk_subs;
+    const void* fn = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(select_cluster_kernel<128, true>)
+                                         : reinterpret_cast<const void*>(select_cluster_kernel<128, false>))
+                                : (mixed ? reinterpret_cast<const void*>(select_cluster_kernel<64, true>)
+                                         : reinterpret_cast<const void*>(select_cluster_kernel<64, false>));
+    // the cluster size is looked up once per instance, for the largest shared-memory size the form
+    // is used with (a cluster that fits with that fits with less)
+    constexpr size_t kMaxSmem = 96 * 1024;
+    static int cached_cs[2][2] = {{-1, -1}, {-1, -1}};  // [D == 128][mixed]
+    int& cs = cached_cs[a.D == 128][mixed];
+    bool ok = smem <= kMaxSmem;
+    if (ok && cs < 0) {
+      ok = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxSmem)) == cudaSuccess;
+      cs = ok ? cluster_size_for(fn, kMaxSmem, 256 * kSubBlocks) : 0;
+    }
+    if (ok && cs > 0) {
+      cudaError_t e1 = launch_pdl(f_qsum, dim3(n_tiles, a.H), dim3(256), 0, p_args, st);
+      if (e1 != cudaSuccess) return e1;
+      int cs_arg = cs, subs_arg = topk_subs, qsum_arg = 0;
+      void* params[4] = {&aa, &cs_arg, &subs_arg, &qsum_arg};
+      return launch_pdl(fn, dim3(static_cast<unsigned>(cs * a.H)), dim3(256 * kSubBlocks), smem, params, st, cs);
+    }
+    cudaGetLastError();  // no cluster of that shape on this device: the forms below
+  }
   if (a.barrier && coop_info(&nsm)) {
     // one cooperative launch for all three stages
-    const int64_t nblk_all = (a.n_tokens + kBlock - 1) / kBlock;
     const size_t smem_keys = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
-    SelectArgs aa = a;
     const void* fn = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(select_fused_kernel<128, true>)
                                          : reinterpret_cast<const void*>(select_fused_kernel<128, false>))
                                 : (mixed ? reinterpret_cast<const void*>(select_fused_kernel<64, true>)
                                          : reinterpret_cast<const void*>(select_fused_kernel<64, false>));
     if (smem_keys > 24 * 1024)
       cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_keys));
-    // 256 threads, 48..57 registers and under 12 KB of shared memory per CTA plus the keys:
+    // 256 threads, at most 80 registers and under 12 KB of shared memory per CTA plus the keys:
     // three CTAs per SM are co-resident while the keys stay below 48 KB
     int per_sm = 3;
     if (smem_keys > 48 * 1024) {
@@ -846,61 +1035,25 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
       if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, 256, smem_keys) != cudaSuccess || occ < 1) occ = 1;
       per_sm = occ < 3 ? occ : 3;
     }
-    const unsigned grid = static_cast<unsigned>(nsm * per_sm);
-    void* params[1] = {&aa};
-    // cooperative (all CTAs co-resident: they meet at two grid barriers) and a programmatic
-    // dependent of the kernel before it (its launch overlaps that kernel's tail)
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = smem_keys;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    return cudaLaunchKernelExC(&cfg, fn, params);
+    // cooperative: all CTAs co-resident, they meet at two grid barriers
+    return launch_pdl(fn, dim3(static_cast<unsigned>(nsm * per_sm)), dim3(256), smem_keys, p_args, st, 0, true);
   }
-  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
-  dim3 g1(n_tiles, a.H);
-  if (a.D == 128)
-    qsum_partial_kernel<128><<<g1, 256, 0, st>>>(a);
-  else
-    qsum_partial_kernel<64><<<g1, 256, 0, st>>>(a);
-  cudaError_t e = cudaGetLastError();
+  // three launches, each a programmatic dependent of the one before
+  cudaError_t e = launch_pdl(f_qsum, dim3(n_tiles, a.H), dim3(256), 0, p_args, st);
   if (e != cudaSuccess) return e;
-  const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-  if (nblk > 0) {
-    dim3 g2(static_cast<unsigned>((nblk + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta), a.n_groups, a.H);
-    if (a.D == 128) {
-      if (mixed)
-        block_scores_kernel<128, true><<<g2, 256, 0, st>>>(a);
-      else
-        block_scores_kernel<128, false><<<g2, 256, 0, st>>>(a);
-    } else {
-      if (mixed)
-        block_scores_kernel<64, true><<<g2, 256, 0, st>>>(a);
-      else
-        block_scores_kernel<64, false><<<g2, 256, 0, st>>>(a);
-    }
-    e = cudaGetLastError();
+  if (nblk_all > 0) {
+    dim3 g2(static_cast<unsigned>(n_chunks_max), a.n_groups, a.H);
+    const void* f2 = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(block_scores_kernel<128, true>)
+                                         : reinterpret_cast<const void*>(block_scores_kernel<128, false>))
+                                : (mixed ? reinterpret_cast<const void*>(block_scores_kernel<64, true>)
+                                         : reinterpret_cast<const void*>(block_scores_kernel<64, false>));
+    e = launch_pdl(f2, g2, dim3(256), 0, p_args, st);
     if (e != cudaSuccess) return e;
   }
-  const size_t smem = static_cast<size_t>(nblk > 0 ? nblk : 1) * sizeof(uint32_t);
-  dim3 g3(a.n_groups, a.H);
-  if (mixed) {
-    if (smem > 40 * 1024)
-      cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    topk_kernel<true><<<g3, 256, smem, st>>>(a);
-  } else {
-    if (smem > 40 * 1024)
-      cudaFuncSetAttribute(topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    topk_kernel<false><<<g3, 256, smem, st>>>(a);
-  }
-  return cudaGetLastError();
+  const size_t smem = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
+  const void* f3 = mixed ? reinterpret_cast<const void*>(topk_kernel<true>) : reinterpret_cast<const void*>(topk_kernel<false>);
+  if (smem > 40 * 1024) cudaFuncSetAttribute(f3, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  return launch_pdl(f3, dim3(a.n_groups, a.H), dim3(256), smem, p_args, st);
 }
 
 }  // namespace hsa

@@ -31,6 +31,7 @@ HSA_ERR_DEVICE_BOUNDS = -6
 HSA_LIN_NONE, HSA_LIN_STATE, HSA_LIN_LINFORMER = 0, 1, 2
 HSA_CFG_CAUSAL = 1
 HSA_CFG_ADAPTIVE = 2
+HSA_CFG_GRID_BARRIER_SELECT = 4
 HSA_FWD_NO_LINEAR, HSA_FWD_NO_SPARSE = 1, 2
 PAGE_TOKENS = 64
 TILE_M = 128
@@ -319,12 +320,14 @@ class HSAContext:
                  lin_mode: int = HSA_LIN_STATE, gate_act: int = 0, softmax_scale: float = 0.0,
                  causal: bool = False, page_order: Optional[torch.Tensor] = None,
                  device: str | torch.device = "cuda:0", adaptive: bool = False, lin_rank: int = 0, lin_seg_tokens: int = 0,
-                 e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None, split_blocks: int = 0):
+                 e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None, split_blocks: int = 0,
+                 grid_barrier_select: bool = False):
         self.device = torch.device(device)
         self.H, self.d = H, d
         self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
         self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
-                              softmax_scale, (HSA_CFG_CAUSAL if causal else 0) | (HSA_CFG_ADAPTIVE if adaptive else 0),
+                              softmax_scale, (HSA_CFG_CAUSAL if causal else 0) | (HSA_CFG_ADAPTIVE if adaptive else 0) |
+                              (HSA_CFG_GRID_BARRIER_SELECT if grid_barrier_select else 0),
                               lin_rank, lin_seg_tokens, split_blocks)
         self.sizes = hsa_query_sizes(self.cfg)
         with torch.cuda.device(self.device):

@@ -24,14 +24,15 @@ def f32(t: torch.Tensor) -> np.ndarray:
 
 
 def build_context(w: W.Workload, device, max_topk=None, causal=None, extra_pages=0, lin_mode=1,
-                  gate_act=0, split_blocks=0):
+                  gate_act=0, split_blocks=0, grid_barrier_select=False):
     from paper_2609_34606_b200 import hsa
     max_pages = w.n_blocks + extra_pages
     order = W.gen_page_order(w, max_pages)
     ctx = hsa.HSAContext(w.H, w.d, max_pages=max_pages, max_q_tokens=max(w.Lq, w.chunk),
                          max_topk=max_topk or max(w.n_blocks, 1), lin_mode=lin_mode,
                          gate_act=gate_act, causal=w.causal if causal is None else causal,
-                         page_order=order, device=device, split_blocks=split_blocks)
+                         page_order=order, device=device, split_blocks=split_blocks,
+                         grid_barrier_select=grid_barrier_select)
     # poison the pools (0xFFFF is a bf16 NaN): anything read but never written shows up
     ctx.k_pool.fill_(0xFF)
     ctx.v_pool.fill_(0xFF)

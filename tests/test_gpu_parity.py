@@ -658,8 +658,8 @@ def test_long_lists_split_over_ctas_and_merged(name, causal, cuda_device):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("name", ["mid_d128", "mid_mix"])
-def test_steps_replayed_from_cuda_graphs_are_bit_identical(name, cuda_device):
+@pytest.mark.parametrize("name,grid_form", [("mid_d128", False), ("mid_mix", False), ("mid_d128", True), ("mid_mix", True)])
+def test_steps_replayed_from_cuda_graphs_are_bit_identical(name, grid_form, cuda_device):
     """append + select + forward captured in CUDA graphs (the cooperative launch and the
     programmatic-dependent launches are ordinary graph nodes) give exactly what the same calls give
     issued one by one -- with a different query chunk in the captured buffer at every replay (so a
@@ -667,7 +667,7 @@ def test_steps_replayed_from_cuda_graphs_are_bit_identical(name, cuda_device):
     replay's sums), two graphs captured one after the other and replayed out of capture order, two
     selection calls per graph, and eager calls in between."""
     w = W.WORKLOADS[name]
-    ctx = Hn.build_context(w, cuda_device, max_topk=max(w.n_blocks, 1))
+    ctx = Hn.build_context(w, cuda_device, max_topk=max(w.n_blocks, 1), grid_barrier_select=grid_form)
     Hn.append_history(ctx, w, cuda_device, n_chunks=w.n_chunks - 1)
     k, v = (t.to(cuda_device) for t in W.gen_kv_chunk(w, w.n_chunks - 1))
     qs = [W.gen_query(w, step=i).to(cuda_device) for i in range(4)]
@@ -729,14 +729,15 @@ def test_steps_replayed_from_cuda_graphs_are_bit_identical(name, cuda_device):
 
 @pytest.mark.gpu
 def test_grid_barrier_wait_that_runs_out_is_reported_and_leaves_the_context_usable(cuda_device):
-    """The one place where CTAs wait for each other is the grid barrier of the selection kernel.
-    Its wait is bounded: with the bound set to a few milliseconds and the barrier's arrive count
+    """The one place where CTAs wait for each other in global memory is the grid barrier of the
+    selection kernel's grid-barrier form (the default form synchronises the CTAs of a head through
+    hardware cluster barriers).  Its wait is bounded: with the bound set to a few milliseconds and the barrier's arrive count
     put where the last arrival can never be seen, the kernel must end by itself, report
     HSA_ERR_DEVICE_TIMEOUT, leave every list of the call empty (a forward call on it is the linear
     branch alone), and the next call must be clean."""
     from paper_2609_34606_b200 import hsa
     w = W.WORKLOADS["mid_d128"]
-    ctx = Hn.build_context(w, cuda_device)
+    ctx = Hn.build_context(w, cuda_device, grid_barrier_select=True)
     Hn.append_history(ctx, w, cuda_device)
     q = W.gen_query(w).to(cuda_device)
     budgets = W.gen_budgets(w).to(cuda_device)
@@ -766,6 +767,39 @@ def test_grid_barrier_wait_that_runs_out_is_reported_and_leaves_the_context_usab
     assert ctx.device_status() == 0
     assert torch.equal(cnt2, ref_cnt) and torch.equal(idx2, ref_idx)
     ctx.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,group_tokens,causal", [("mid_d128", 0, False), ("mid_d128", 128, False), ("mid_mix", 0, False),
+                                                      ("mid_causal", 128, True), ("mid_d64", 0, False), ("cfg2", 0, False),
+                                                      ("cfg2", 128, False)])
+def test_cluster_and_grid_barrier_forms_of_the_selection_agree(name, group_tokens, causal, cuda_device):
+    """The selection kernel has two forms (one thread-block cluster per head with hardware cluster
+    barriers; one cooperative launch with two grid barriers).  Both run the same stages on the same
+    data in the same order, so their lists must be identical bit for bit -- plain, per query tile,
+    and with the two sparse granularities."""
+    w = W.WORKLOADS[name]
+    res = []
+    for grid_form in (False, True):
+        ctx = Hn.build_context(w, cuda_device, causal=causal, grid_barrier_select=grid_form,
+                               max_topk=w.topk if name == "cfg2" else None)
+        Hn.append_history(ctx, w, cuda_device, n_chunks=min(w.n_chunks, 4) if name == "cfg2" else None)
+        q = W.gen_query(w).to(cuda_device)
+        budgets = W.gen_budgets(w).to(cuda_device)
+        q_pos0 = ctx.n_tokens - (w.Lq if causal else 0)
+        a = ctx.select_blocks(q, budgets, q_pos0=q_pos0, causal=causal, group_tokens=group_tokens)
+        p0 = max(0, ctx.n_tokens - w.chunk) // 64
+        b = ctx.select_blocks_ex(q, budgets, inter_block_pages=2, intra_first_page=p0, q_pos0=q_pos0, causal=causal,
+                                 group_tokens=group_tokens) if name != "cfg2" else a
+        assert ctx.device_status() == 0
+        res.append((Hn.selection_lists(*a), Hn.selection_lists(*b)))
+        ctx.destroy()
+    for x, y in zip(res[0], res[1]):
+        for h in range(w.H):
+            assert len(x[h]) == len(y[h])
+            for g in range(len(x[h])):
+                assert x[h][g].tolist() == y[h][g].tolist(), (h, g)
+    assert sum(len(l) for hl in res[0][0] for l in hl) > 0
 
 
 @pytest.mark.gpu
