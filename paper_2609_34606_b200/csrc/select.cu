@@ -634,13 +634,14 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------
-// The same three stages with the CTAs of a head forming a thread-block cluster: everything a head
-// needs -- its query tile sums, its scores, its lists -- is produced inside its cluster, so the two
-// synchronisation points are hardware cluster barriers (release / acquire at cluster scope) instead
-// of grid-wide barriers in global memory, and the launch needs no co-residency of the whole grid.
+// The score and list stages with the CTAs of a head forming a thread-block cluster: everything a
+// head's lists need -- its scores -- is produced inside its cluster, so the synchronisation point
+// between the two stages is a hardware cluster barrier (release / acquire at cluster scope) instead
+// of a grid-wide barrier in global memory, and the launch needs no co-residency of the whole grid.
+// The query tile sums come from qsum_partial_kernel, launched in front of this kernel (they read the
+// whole chunk and want every SM; this kernel waits for them as a programmatic dependent).
 // grid = H clusters of CS CTAs; a CTA holds kSubBlocks blocks of 256 threads, each of which takes
-// work items of its own (slot = cluster rank * kSubBlocks + sub-block), so that the 37 query tiles
-// of a head are read in one round trip.
+// work items of its own (slot = cluster rank * kSubBlocks + sub-block).
 // ---------------------------------------------------------------------------------------
 constexpr int kSubBlocks = 3;
 
@@ -656,7 +657,7 @@ struct ClusterSmem {
 };
 
 template <int D, bool MIXED>
-__global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(SelectArgs a, int cluster_ctas, int topk_subs, int with_qsum) {
+__global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(SelectArgs a, int cluster_ctas, int topk_subs) {
   // dynamic shared memory: per sub-block scratch (tile-sum partials / mean query / a batch of mean
   // queries) | per sub-block top-k bookkeeping | [topk_subs][blocks] keys
   extern __shared__ __align__(16) unsigned char cl_smem[];
@@ -671,19 +672,11 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   const int n_slots = cluster_ctas * kSubBlocks;
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
-  // the key sums of this block's first score item are requested ahead of the query sums
+  // the key sums of this block's first score item are requested first
   ScoreOperands<D, MIXED> op;
   const bool ahead = a.n_groups == 1 && slot < n_chunks;
   if (ahead) scores_load<D, MIXED>(blk, a, slot, h, op);
-  if (with_qsum) {
-    for (int tile = slot; tile < n_tiles; tile += n_slots) {
-      qsum_item<D>(blk, a, tile, h, reinterpret_cast<float(*)[D]>(scratch));
-      blk_sync(blk);
-    }
-    cluster_sync_all();  // the head's tile sums are complete and visible to its cluster
-  }
   if (a.n_groups > 1) {
     for (int chunk = slot; chunk < n_chunks; chunk += n_slots)
       scores_item_groups<D, MIXED>(blk, a, chunk, h, reinterpret_cast<double*>(scratch));
@@ -693,7 +686,7 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
       blk_sync(blk);
     }
   }
-  cluster_sync_all();  // ... and so are its score keys
+  cluster_sync_all();  // the score keys of the head are complete and visible to its cluster
   // the kernel behind this one may take the places of the CTAs that leave now
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (sub < topk_subs) {
@@ -1012,8 +1005,8 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
     if (ok && cs > 0) {
       cudaError_t e1 = launch_pdl(f_qsum, dim3(n_tiles, a.H), dim3(256), 0, p_args, st);
       if (e1 != cudaSuccess) return e1;
-      int cs_arg = cs, subs_arg = topk_subs, qsum_arg = 0;
-      void* params[4] = {&aa, &cs_arg, &subs_arg, &qsum_arg};
+      int cs_arg = cs, subs_arg = topk_subs;
+      void* params[3] = {&aa, &cs_arg, &subs_arg};
       return launch_pdl(fn, dim3(static_cast<unsigned>(cs * a.H)), dim3(256 * kSubBlocks), smem, params, st, cs);
     }
     cudaGetLastError();  // no cluster of that shape on this device: the forms below
