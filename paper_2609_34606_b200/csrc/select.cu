@@ -651,15 +651,14 @@ __device__ __forceinline__ void cluster_sync_all() {
 
 template <int D>
 struct ClusterSmem {
-  static constexpr int kGroupBytes = kGroupBatch * (D + 4) * 8;
-  static constexpr int kScratch = kGroupBytes > 256 / (D / 8) * D * 4 ? kGroupBytes : 256 / (D / 8) * D * 4;
-  static constexpr int kFixed = (kSubBlocks * kScratch + kSubBlocks * static_cast<int>(sizeof(TopkShared)) + 15) / 16 * 16;
+  static constexpr int kScratch = (D + 256) * 8;  // mean query + its per-way partial sums, fp64
+  static constexpr int kFixed = (kSubBlocks * kScratch + static_cast<int>(sizeof(TopkShared)) + 15) / 16 * 16;
 };
 
 template <int D, bool MIXED>
-__global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(SelectArgs a, int cluster_ctas, int topk_subs) {
-  // dynamic shared memory: per sub-block scratch (tile-sum partials / mean query / a batch of mean
-  // queries) | per sub-block top-k bookkeeping | [topk_subs][blocks] keys
+__global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(SelectArgs a, int cluster_ctas) {
+  // dynamic shared memory: per sub-block scratch (mean query and its partial sums) | top-k
+  // bookkeeping | the head's keys
   extern __shared__ __align__(16) unsigned char cl_smem[];
   constexpr int kScratch = ClusterSmem<D>::kScratch;
   const int sub = static_cast<int>(threadIdx.x) / 256;
@@ -673,31 +672,18 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
+  // (one list per head: the launcher sends per-tile selections to the grid-barrier form)
   // the key sums of this block's first score item are requested first
   ScoreOperands<D, MIXED> op;
-  const bool ahead = a.n_groups == 1 && slot < n_chunks;
-  if (ahead) scores_load<D, MIXED>(blk, a, slot, h, op);
-  if (a.n_groups > 1) {
-    for (int chunk = slot; chunk < n_chunks; chunk += n_slots)
-      scores_item_groups<D, MIXED>(blk, a, chunk, h, reinterpret_cast<double*>(scratch));
-  } else {
-    for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
-      scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot);
-      blk_sync(blk);
-    }
+  if (slot < n_chunks) scores_load<D, MIXED>(blk, a, slot, h, op);
+  for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
+    scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot);
+    blk_sync(blk);
   }
   cluster_sync_all();  // the score keys of the head are complete and visible to its cluster
   // the kernel behind this one may take the places of the CTAs that leave now
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (sub < topk_subs) {
-    const int64_t nblk = (a.n_tokens + kBlock - 1) / kBlock;
-    uint32_t* keys = cl_keys + static_cast<size_t>(sub) * static_cast<size_t>(nblk > 0 ? nblk : 1);
-    const int slot3 = (static_cast<int>(blockIdx.x) % cluster_ctas) * topk_subs + sub;
-    for (int g = slot3; g < a.n_groups; g += cluster_ctas * topk_subs) {
-      topk_item<MIXED>(blk, a, g, h, keys, sh_all + sub);
-      blk_sync(blk);
-    }
-  }
+  if (slot == 0) topk_item<MIXED>(blk, a, 0, h, cl_keys, sh_all);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -965,10 +951,11 @@ cudaError_t launch_pdl(const void* fn, dim3 grid, dim3 block, size_t smem, void*
 // Three forms, all programmatic dependents of the kernel before them:
 //   cluster form        query tile sums as a kernel of their own (they read the whole chunk and want
 //                       every SM), then one cluster of 8 CTAs per head for scores and lists, with one
-//                       hardware cluster barrier between them -- the default while a head has at most
-//                       kClusterMaxChunks score items (short and medium histories)
+//                       hardware cluster barrier between them -- the default for one list per head while
+//                       a head has at most kClusterMaxChunks score items (short and medium histories)
 //   grid-barrier form   one cooperative launch over all SMs with two device barriers -- long histories
-//                       (the score stage then wants every SM too), and on request
+//                       (the score stage then wants every SM too), one list per query tile (37 x H
+//                       lists want more than 24 blocks of threads per head), and on request
 //   three launches      for devices without cooperative launch and for callers without a barrier word
 constexpr int kClusterMaxChunks = 2 * 8 * kSubBlocks;
 
@@ -983,11 +970,10 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
                                   : reinterpret_cast<const void*>(qsum_partial_kernel<64>);
   // candidates per head (coarse candidates make fewer; an upper bound is enough to choose the form)
   const int64_t n_chunks_max = (nblk_all + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
-  if (a.use_clusters && n_chunks_max <= kClusterMaxChunks) {
+  if (a.use_clusters && a.n_groups == 1 && n_chunks_max <= kClusterMaxChunks) {
     const size_t key_bytes = static_cast<size_t>(nblk_all > 0 ? nblk_all : 1) * sizeof(uint32_t);
-    const int topk_subs = kSubBlocks;
     const size_t fixed = a.D == 128 ? ClusterSmem<128>::kFixed : ClusterSmem<64>::kFixed;
-    const size_t smem = fixed + key_bytes * topk_subs;
+    const size_t smem = fixed + key_bytes;
     const void* fn = a.D == 128 ? (mixed ? reinterpret_cast<const void*>(select_cluster_kernel<128, true>)
                                          : reinterpret_cast<const void*>(select_cluster_kernel<128, false>))
                                 : (mixed ? reinterpret_cast<const void*>(select_cluster_kernel<64, true>)
@@ -1005,8 +991,8 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
     if (ok && cs > 0) {
       cudaError_t e1 = launch_pdl(f_qsum, dim3(n_tiles, a.H), dim3(256), 0, p_args, st);
       if (e1 != cudaSuccess) return e1;
-      int cs_arg = cs, subs_arg = topk_subs;
-      void* params[3] = {&aa, &cs_arg, &subs_arg};
+      int cs_arg = cs;
+      void* params[2] = {&aa, &cs_arg};
       return launch_pdl(fn, dim3(static_cast<unsigned>(cs * a.H)), dim3(256 * kSubBlocks), smem, params, st, cs);
     }
     cudaGetLastError();  // no cluster of that shape on this device: the forms below
