@@ -3,7 +3,8 @@
 
 A "step" is one pass of the whole hot path for one query chunk of the
 1.3B-class video-DiT layer workload (H=12, d=128, chunk 4680 tokens, history
-10 chunks = 46,800 tokens, top-64 blocks per head): restore the 9-chunk state,
+10 chunks = 46,800 tokens, top-64 blocks per head): undo the previous step's append
+(hsa_rewind to the 9-chunk history, host bookkeeping only), then
 hsa_append_kv (chunk 10) -> hsa_select_blocks -> hsa_forward.  By default the
 step is captured once per input set in a CUDA graph and the timed loop replays
 the graphs (`--launch eager` issues the same calls one by one instead).
@@ -174,14 +175,9 @@ def bench_ours(args, rank: int, world: int):
         k, v = W.gen_kv_chunk(w, c, layer=rank)
         ctx.append_kv(k.to(dev), v.to(dev))
     n_before = ctx.n_tokens
-    # what a step changes and the next step must find as it was: the running state S, z (and the
-    # key sum of a partly filled last block, if the history does not end on a block boundary)
-    # (S and z sit next to each other at the start of the state buffer: one copy restores both)
-    assert ctx.S.data_ptr() == ctx.state.data_ptr() and ctx.z.data_ptr() > ctx.S.data_ptr()
-    sz_bytes = ctx.z.data_ptr() - ctx.state.data_ptr() + ctx.z.numel() * 4
-    sz_snap = ctx.state[:sz_bytes].clone()
-    tail_blk = n_before // 64 if n_before % 64 else None
-    ksum_snap = ctx.ksum[:, tail_blk].clone() if tail_blk is not None else None
+    # A step appends chunk n_chunks to the (n_chunks - 1)-chunk history; the next step first undoes that
+    # append (hsa_rewind to the length before it: host bookkeeping only -- the state before the append
+    # is still in the library's other state slot) and appends its own chunk.
     # host (pinned) and device copies of RING distinct input sets
     host, devs = [], []
     for r in range(RING):
@@ -200,9 +196,6 @@ def bench_ours(args, rank: int, world: int):
             q.copy_(hq, non_blocking=True)
             k.copy_(hk, non_blocking=True)
             v.copy_(hv, non_blocking=True)
-        ctx.state[:sz_bytes].copy_(sz_snap)
-        if tail_blk is not None:
-            ctx.ksum[:, tail_blk].copy_(ksum_snap)
         ctx.rewind(n_before)
         if ev:
             ev[0].record()
@@ -441,7 +434,7 @@ def bench_ours(args, rank: int, world: int):
                        "selection": "one per head for the whole chunk" if not gt else f"one per {gt}-row query tile",
                        "linear_branch": ("running state (S, z)" if args.lin == "state" else
                                          f"Linformer form, rank {args.lin_rank}, segments of {w.chunk} tokens"),
-                       "step": f"restore the {w.n_chunks - 1}-chunk running state (S, z) + hsa_append_kv + "
+                       "step": f"undo the previous step's append (back to the {w.n_chunks - 1}-chunk history) + hsa_append_kv + "
                                "hsa_select_blocks + hsa_forward",
                        "launch": (f"CUDA graphs: the timed loop replays a graph of {2 * RING} consecutive steps "
                                   "(single-step graphs for the remainder)"

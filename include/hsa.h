@@ -272,14 +272,19 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
 /* Host-tracked length of the history. */
 int hsa_get_info(hsa_ctx* ctx, int64_t* n_tokens, int32_t* n_blocks);
 
-/* Sets the history length back to n_tokens (<= current).  The pool keeps its pages, but the
- * key sums of the new tail block and the linear state are NOT recomputed: the caller must
- * restore the state buffer to the contents it had at that length (used by benchmarks that
- * replay the same append). */
+/* Sets the history length back to n_tokens (<= current).
+ * Undoing exactly the most recent hsa_append_kv (n_tokens = the length before it, no other rewind in
+ * between) needs nothing else: the linear state lives in two slots that take turns, so the state
+ * before that append is still there, and the key sum its first block had before the append is kept
+ * and reused by the next append from that length.  The same chunk, or another one, can then be
+ * appended again (benchmarks replay a step this way; a caller can drop a speculative chunk).
+ * Any other rewind keeps the pool's pages but recomputes nothing: the caller must put the state
+ * buffer (hsa_state_layout) back to the contents it had at that length. */
 int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens);
 
 /* Byte offsets inside the state buffer, for tests and snapshots:
- * S fp32 [H][d][d], z fp32 [H][d], key sums fp32 [H][max_pages][d]. */
+ * S fp32 [H][d][d], z fp32 [H][d] (of the slot that holds the current state: the offsets change with
+ * every hsa_append_kv and with an undoing hsa_rewind), key sums fp32 [H][max_pages][d]. */
 int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksum);
 
 /* Synchronises the device, reads and clears the status word: HSA_OK or a DEVICE_* code.

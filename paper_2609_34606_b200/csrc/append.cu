@@ -65,7 +65,12 @@ __global__ void __launch_bounds__(256) append_pool_ksum_kernel(AppendArgs a) {
 #pragma unroll
     for (int r = 0; r < RP; ++r) s += red[r][threadIdx.x];
     float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + threadIdx.x;
-    const float old = (t_lo > b * kBlock) ? *dst : 0.f;  // block already partly filled
+    float old = 0.f;
+    if (t_lo > b * kBlock) {  // block already partly filled: its sum before this append
+      float* saved = a.ksum_saved + static_cast<size_t>(h) * D + threadIdx.x;
+      old = a.tail_from_saved ? *saved : *dst;
+      if (!a.tail_from_saved) *saved = old;
+    }
     *dst = old + s;
   }
 }
@@ -163,8 +168,8 @@ __global__ void __launch_bounds__(256) state_partial_kernel(AppendArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Stage C: S_prev <- S, S <- S + sum of partials (fixed order), and the bf16 hi/lo split of
-// both (the forward kernel feeds hi and lo to the tensor cores as two bf16 operands).
+// Stage C: S[dst] <- S[src] + sum of partials (fixed order), with its bf16 hi/lo split (the forward
+// kernels feed hi and lo to the tensor cores as two bf16 operands), the same for z and its operand image.
 // ---------------------------------------------------------------------------------------
 __global__ void state_reduce_kernel(AppendArgs a) {
   const int D = a.D;
@@ -183,38 +188,28 @@ __global__ void state_reduce_kernel(AppendArgs a) {
   float add = 0.f;
 #pragma unroll
   for (int i = 0; i < kStateSplitMax; ++i) add += v[i];
+  const int dst = a.src_slot ^ 1;
   if (idx < DD) {
     const size_t o = static_cast<size_t>(h) * DD + idx;
-    const float s_old = a.S[o];
-    const float s_new = s_old + add;
-    a.S_prev[o] = s_old;
-    a.S[o] = s_new;
-    __nv_bfloat16* hl = a.hilo + static_cast<size_t>(h) * 4 * DD + idx;
+    const float s_new = a.S[a.src_slot][o] + add;
+    a.S[dst][o] = s_new;
+    __nv_bfloat16* hl = a.hilo + (static_cast<size_t>(h) * 2 + dst) * 2 * DD + idx;
     const __nv_bfloat16 nh = __float2bfloat16_rn(s_new);
-    const __nv_bfloat16 oh = __float2bfloat16_rn(s_old);
-    hl[0 * DD] = nh;
-    hl[1 * DD] = __float2bfloat16_rn(s_new - __bfloat162float(nh));
-    hl[2 * DD] = oh;
-    hl[3 * DD] = __float2bfloat16_rn(s_old - __bfloat162float(oh));
+    hl[0] = nh;
+    hl[DD] = __float2bfloat16_rn(s_new - __bfloat162float(nh));
   } else {
     const int k = idx - DD;
     const size_t o = static_cast<size_t>(h) * D + k;
-    const float z_old = a.z[o];
-    const float z_new = z_old + add;
-    a.z_prev[o] = z_old;
-    a.z[o] = z_new;
+    const float z_new = a.z[a.src_slot][o] + add;
+    a.z[dst][o] = z_new;
     if (D == 128) {
-      // operand images of z (current, previous): element (row n, dim k) of a K-major tile with the
-      // 128-byte swizzle sits at slab (k / 64), row n, 16-byte chunk ((k % 64) / 8) ^ (n % 8)
+      // operand image of z: element (row n, dim k) of a K-major tile with the 128-byte swizzle sits
+      // at slab (k / 64), row n, 16-byte chunk ((k % 64) / 8) ^ (n % 8)
       const int slab = k >> 6, kk = k & 63, c = kk >> 3;
-      const float zs[2] = {z_new, z_old};
-#pragma unroll
-      for (int w = 0; w < 2; ++w) {
-        uint8_t* img = a.zop + static_cast<size_t>(h * 2 + w) * kZopBytes + slab * (kZopBytes / 2) + (kk & 7) * 2;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(zs[w]);
-        *reinterpret_cast<__nv_bfloat16*>(img + 0 * 128 + ((c ^ 0) << 4)) = hi;
-        *reinterpret_cast<__nv_bfloat16*>(img + 1 * 128 + ((c ^ 1) << 4)) = __float2bfloat16_rn(zs[w] - __bfloat162float(hi));
-      }
+      uint8_t* img = a.zop + static_cast<size_t>(h * 2 + dst) * kZopBytes + slab * (kZopBytes / 2) + (kk & 7) * 2;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(z_new);
+      *reinterpret_cast<__nv_bfloat16*>(img + 0 * 128 + ((c ^ 0) << 4)) = hi;
+      *reinterpret_cast<__nv_bfloat16*>(img + 1 * 128 + ((c ^ 1) << 4)) = __float2bfloat16_rn(z_new - __bfloat162float(hi));
     }
   }
 }
@@ -436,7 +431,12 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
       if (lane == 0) mbar_arrive(&bars->ks_read[bj & 1]);
       const int64_t b = bs + bj;
       float* dst = a.ksum + (static_cast<size_t>(h) * a.max_pages + b) * D + quad * 32 + lane;
-      const float old = (a.n0 > b * kBlock) ? *dst : 0.f;  // block partly filled before
+      float old = 0.f;
+      if (a.n0 > b * kBlock) {  // block partly filled before: its sum before this append
+        float* saved = a.ksum_saved + static_cast<size_t>(h) * D + quad * 32 + lane;
+        old = a.tail_from_saved ? *saved : *dst;
+        if (!a.tail_from_saved) *saved = old;
+      }
       *dst = old + __uint_as_float(v[0]);
     }
   } else {

@@ -342,7 +342,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t ph = (j / kStages) & 1;
             ok = wait_bar(&bars->v_empty[s], ph ^ 1, bars, p.status);
             if (!ok) break;
-            const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
+            const int rbase = ((h * 2 + p.state_slot) * 2 + hl) * D;
             mbar_expect_tx(&bars->v_full[s], D * D * 2);
             for (int kb = 0; kb < DH; ++kb)
               for (int dh = 0; dh < DH; ++dh)

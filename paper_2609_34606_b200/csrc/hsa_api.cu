@@ -36,7 +36,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   // state
-  size_t S, z, S_prev, z_prev, hilo, zop, ksum, state_total;
+  size_t S, z, slot_S, slot_z, hilo, zop, ksum_saved, ksum, state_total;  // S, z: slot 0; slot_*: bytes per slot
   // workspace
   size_t status, page_table, qpart, keys, spart, lin_num, lin_den, ctable, csel, ccnt, olin, ad_w, ad_idx, ad_gini, ad_wsum,
       part_o, part_l, part_ref, part_ticket, ws_total;
@@ -70,12 +70,13 @@ Layout make_layout(const hsa_config* c) {
   Layout L{};
   const size_t H = c->num_heads, D = c->head_dim, P = c->max_pages;
   size_t o = 0;
-  L.S = o;      o = align_up(o + H * D * D * 4, 1024);
-  L.z = o;      o = align_up(o + H * D * 4, 1024);
-  L.S_prev = o; o = align_up(o + H * D * D * 4, 1024);
-  L.z_prev = o; o = align_up(o + H * D * 4, 1024);
+  L.slot_S = align_up(H * D * D * 4, 1024);
+  L.slot_z = align_up(H * D * 4, 1024);
+  L.S = o;      o += 2 * L.slot_S;
+  L.z = o;      o += 2 * L.slot_z;
   L.hilo = o;   o = align_up(o + H * 4 * D * D * 2, 1024);
   L.zop = o;    o = align_up(o + H * 2 * kZopBytes, 1024);
+  L.ksum_saved = o; o = align_up(o + H * D * 4, 1024);
   L.ksum = o;   o = align_up(o + H * P * D * 4, 1024);
   L.state_total = o;
   const size_t tiles = (static_cast<size_t>(c->max_q_tokens) + kTileM - 1) / kTileM;
@@ -132,6 +133,8 @@ struct hsa_ctx {
   float scale;
   int64_t n_tokens;
   int32_t last_append;  // tokens of the most recent append (0 after a rewind)
+  int cur_slot;         // state slot that holds the running state of the current history
+  int64_t tail_saved_for;  // history length whose tail-block key sum sits in the saved-tail buffer (-1: none)
   int nsm;
   CUtensorMap tm_k, tm_v, tm_state, tm_kc, tm_vc, tm_olin;
   int32_t n_segs;  // Linformer: complete segments compressed so far
@@ -233,6 +236,8 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
   ctx->last_append = 0;
   ctx->last_cuda_error = 0;
   ctx->n_segs = 0;
+  ctx->cur_slot = 0;
+  ctx->tail_saved_for = -1;
   ctx->wait_ns = 2000000000ull;
   ctx->page_table_host = pt;
   ctx->resident.assign(static_cast<size_t>(cfg->max_pages), 1);
@@ -318,10 +323,13 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   a.k_pool = static_cast<__nv_bfloat16*>(ctx->buf.k_pool);
   a.v_pool = static_cast<__nv_bfloat16*>(ctx->buf.v_pool);
   a.ksum = reinterpret_cast<float*>(stt + ctx->lay.ksum);
-  a.S = reinterpret_cast<float*>(stt + ctx->lay.S);
-  a.z = reinterpret_cast<float*>(stt + ctx->lay.z);
-  a.S_prev = reinterpret_cast<float*>(stt + ctx->lay.S_prev);
-  a.z_prev = reinterpret_cast<float*>(stt + ctx->lay.z_prev);
+  for (int sl = 0; sl < 2; ++sl) {
+    a.S[sl] = reinterpret_cast<float*>(stt + ctx->lay.S + sl * ctx->lay.slot_S);
+    a.z[sl] = reinterpret_cast<float*>(stt + ctx->lay.z + sl * ctx->lay.slot_z);
+  }
+  a.src_slot = ctx->cur_slot;
+  a.ksum_saved = reinterpret_cast<float*>(stt + ctx->lay.ksum_saved);
+  a.tail_from_saved = (ctx->n_tokens % kBlock) != 0 && ctx->tail_saved_for == ctx->n_tokens;
   a.hilo = reinterpret_cast<__nv_bfloat16*>(stt + ctx->lay.hilo);
   a.zop = stt + ctx->lay.zop;
   a.spart = reinterpret_cast<float*>(ws + ctx->lay.spart);
@@ -368,6 +376,8 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     ctx->n_segs += 1;
   }
   for (int64_t b = ctx->n_tokens / kBlock; b <= (n1 - 1) / kBlock; ++b) ctx->resident[static_cast<size_t>(b)] = 1;
+  if (ctx->n_tokens % kBlock) ctx->tail_saved_for = ctx->n_tokens;
+  if (a.lin_state) ctx->cur_slot ^= 1;  // the append wrote the other slot
   ctx->n_tokens = n1;
   ctx->last_append = n_tokens;
   return HSA_OK;
@@ -536,8 +546,8 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   p.n_groups = q_group_tokens > 0 ? (n_q + q_group_tokens - 1) / q_group_tokens : 1;
   p.page_table = reinterpret_cast<const int32_t*>(ws + ctx->lay.page_table);
   p.n_blocks = static_cast<int>((ctx->n_tokens + kBlock - 1) / kBlock);
-  p.use_prev = causal_lin ? 1 : 0;
-  p.z = reinterpret_cast<const float*>(stt + (causal_lin ? ctx->lay.z_prev : ctx->lay.z));
+  p.state_slot = ctx->cur_slot ^ (causal_lin ? 1 : 0);  // causal: the state before the chunk's own append
+  p.z = reinterpret_cast<const float*>(stt + ctx->lay.z + p.state_slot * ctx->lay.slot_z);
   p.zop = stt + ctx->lay.zop;
   p.g_lin = static_cast<const __nv_bfloat16*>(g_lin);
   p.g_sp = static_cast<const __nv_bfloat16*>(g_sp);
@@ -731,6 +741,12 @@ int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens) {
     if (n_tokens % ctx->cfg.lin_seg_tokens) return HSA_ERR_UNSUPPORTED;
     ctx->n_segs = static_cast<int32_t>(n_tokens / ctx->cfg.lin_seg_tokens);
   }
+  // Undoing exactly the last append: the state before it is still in the other slot, and the key
+  // sum its first block had before it is in the saved-tail buffer (the next append from this length
+  // takes it from there), so nothing has to be restored.
+  const bool undo = ctx->last_append > 0 && n_tokens == ctx->n_tokens - ctx->last_append;
+  if (undo && ctx->cfg.lin_mode == HSA_LIN_STATE) ctx->cur_slot ^= 1;
+  if (n_tokens < ctx->tail_saved_for) ctx->tail_saved_for = -1;
   ctx->n_tokens = n_tokens;
   ctx->last_append = 0;
   return HSA_OK;
@@ -738,8 +754,8 @@ int hsa_rewind(hsa_ctx* ctx, int64_t n_tokens) {
 
 int hsa_state_layout(hsa_ctx* ctx, size_t* off_S, size_t* off_z, size_t* off_ksum) {
   if (!ctx) return HSA_ERR_INVALID_ARG;
-  if (off_S) *off_S = ctx->lay.S;
-  if (off_z) *off_z = ctx->lay.z;
+  if (off_S) *off_S = ctx->lay.S + ctx->cur_slot * ctx->lay.slot_S;
+  if (off_z) *off_z = ctx->lay.z + ctx->cur_slot * ctx->lay.slot_z;
   if (off_ksum) *off_ksum = ctx->lay.ksum;
   return HSA_OK;
 }

@@ -35,12 +35,18 @@ struct AppendArgs {
   __nv_bfloat16* k_pool;
   __nv_bfloat16* v_pool;
   float* ksum;      // [H][max_pages][D]
-  float* S;         // [H][D][D]
-  float* z;         // [H][D]
-  float* S_prev;    // state before this append
-  float* z_prev;
-  __nv_bfloat16* hilo;  // [H][2 cur/prev][2 hi/lo][D][D]
-  uint8_t* zop;         // [H][2 cur/prev][kZopBytes]: z as a tensor-core operand (head_dim 128)
+  // The running state lives in two slots that take turns: an append reads slot src_slot and writes
+  // slot src_slot ^ 1, which becomes the current one; the other keeps the state before the append
+  // (what a causal forward over the appended chunk applies, and what undoing the append returns to).
+  float* S[2];          // [H][D][D] per slot
+  float* z[2];          // [H][D] per slot
+  int src_slot;
+  __nv_bfloat16* hilo;  // [H][2 slots][2 hi/lo][D][D]: bf16 hi + lo of S, what the forward kernels read
+  uint8_t* zop;         // [H][2 slots][kZopBytes]: z as a tensor-core operand (head_dim 128)
+  // key sum the (partly filled) first block of this append had before it: saved here when the append
+  // reads it from ksum, read from here instead when the append repeats one that was undone
+  float* ksum_saved;    // [H][D]
+  int tail_from_saved;
   float* spart;         // [H][nsplit][D*D + D] scratch
   int nsplit;
   int lin_state;  // update the linear state?
@@ -103,9 +109,8 @@ struct FwdParams {
   const int32_t* page_table;
   int n_blocks;
   const float* z;       // [H][D] state the linear branch applies
-  const uint8_t* zop;   // [H][2 cur/prev][kZopBytes]: the same z as a tensor-core operand
-  int state_row0_mul;   // row of the hi/lo state tensor map = ((h*2 + use_prev)*2 + hl)*D
-  int use_prev;
+  const uint8_t* zop;   // [H][2 slots][kZopBytes]: the same z as a tensor-core operand
+  int state_slot;       // slot the linear branch applies; row of the hi/lo tensor map = ((h*2 + slot)*2 + hl)*D
   const __nv_bfloat16* g_lin;
   const __nv_bfloat16* g_sp;
   int64_t g_ts, g_hs, g_ds;

@@ -115,13 +115,13 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
   auto load_state = [&](int h) {
     mbar_expect_tx(&bars->s_full, kLoParts * kLoTile + kLoZop);
     for (int hl = 0; hl < kLoParts; ++hl) {
-      const int rbase = ((h * 2 + p.use_prev) * 2 + hl) * D;
+      const int rbase = ((h * 2 + p.state_slot) * 2 + hl) * D;
       for (int kb = 0; kb < 2; ++kb)
         for (int dh = 0; dh < 2; ++dh)
           tma_load_2d(s_state + hl * kLoTile + dh * kLoHalf + kb * (kBlock * 128), &tm_state, &bars->s_full, dh * 64,
                       rbase + kb * 64);
     }
-    bulk_load(s_zop, p.zop + static_cast<size_t>(h * 2 + p.use_prev) * kLoZop, kLoZop, &bars->s_full);
+    bulk_load(s_zop, p.zop + static_cast<size_t>(h * 2 + p.state_slot) * kLoZop, kLoZop, &bars->s_full);
   };
 
   // the kernel behind this one may be scheduled as soon as this grid's CTAs have all started

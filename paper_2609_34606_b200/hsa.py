@@ -341,7 +341,7 @@ class HSAContext:
                                self.workspace.data_ptr(), _ptr(self.kc_pool), _ptr(self.vc_pool),
                                _ptr(e_k), _ptr(e_v))
             self.ctx = hsa_create(self.cfg, bufs, page_order)
-        self._off_S, self._off_z, self._off_ksum = hsa_state_layout(self.ctx)
+        self._off_ksum = hsa_state_layout(self.ctx)[2]
 
     # -- state views (fp32) for tests and snapshots
     def _view(self, off: int, shape) -> torch.Tensor:
@@ -352,11 +352,12 @@ class HSAContext:
 
     @property
     def S(self) -> torch.Tensor:
-        return self._view(self._off_S, (self.H, self.d, self.d))
+        # (the state lives in two slots that take turns: ask where the current one is)
+        return self._view(hsa_state_layout(self.ctx)[0], (self.H, self.d, self.d))
 
     @property
     def z(self) -> torch.Tensor:
-        return self._view(self._off_z, (self.H, self.d))
+        return self._view(hsa_state_layout(self.ctx)[1], (self.H, self.d))
 
     @property
     def ksum(self) -> torch.Tensor:

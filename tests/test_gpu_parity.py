@@ -97,6 +97,45 @@ def test_incremental_append_matches_any_chunking(cuda_device):
         assert np.abs(r[4] - res[0][4]).max() <= 4e-3
 
 
+def test_rewind_undoes_the_last_append_without_restoring_anything(cuda_device):
+    """Appending a chunk, taking it back with hsa_rewind and appending another one (here twice, and
+    with a history that ends inside a block, so that the tail block's key sum is involved) must
+    leave exactly what a context that never saw the dropped chunks holds: state, key sums, selection
+    and output bit for bit -- with no copy of the state by the caller."""
+    w = W.WORKLOADS["mid_d128"]            # chunks of 333 tokens: every chunk starts inside a block
+    ks = [W.gen_kv_chunk(w, c) for c in range(w.n_chunks + 2)]
+    q = W.gen_query(w).to(cuda_device)
+    budgets = W.gen_budgets(w).to(cuda_device)
+
+    def finish(ctx):
+        si, sc = ctx.select_blocks(q, budgets)
+        out = ctx.forward(q, si, sc)
+        assert ctx.device_status() == 0
+        return (ctx.S.clone(), ctx.z.clone(), ctx.ksum[:, :ctx.n_blocks].clone(), sc.clone(), si.clone(), out.clone())
+
+    ref_ctx = Hn.build_context(w, cuda_device, extra_pages=8)
+    for c in range(w.n_chunks):
+        ref_ctx.append_kv(ks[c][0].to(cuda_device), ks[c][1].to(cuda_device))
+    ref = finish(ref_ctx)
+
+    ctx = Hn.build_context(w, cuda_device, extra_pages=8)
+    for c in range(w.n_chunks - 1):
+        ctx.append_kv(ks[c][0].to(cuda_device), ks[c][1].to(cuda_device))
+    n0 = ctx.n_tokens
+    assert n0 % 64 != 0
+    for dropped in (w.n_chunks, w.n_chunks + 1):          # two chunks that are taken back again
+        ctx.append_kv(ks[dropped][0].to(cuda_device), ks[dropped][1].to(cuda_device))
+        assert ctx.n_tokens == n0 + w.chunk
+        ctx.rewind(n0)
+        assert ctx.n_tokens == n0
+    ctx.append_kv(ks[w.n_chunks - 1][0].to(cuda_device), ks[w.n_chunks - 1][1].to(cuda_device))
+    got = finish(ctx)
+    for a, b in zip(got, ref):
+        assert torch.equal(a, b)
+    ctx.destroy()
+    ref_ctx.destroy()
+
+
 def test_edge_cases(cuda_device):
     from paper_2609_34606_b200 import hsa
     w = W.WORKLOADS["mid_d64"]
