@@ -136,7 +136,7 @@ struct hsa_ctx {
   int cur_slot;         // state slot that holds the running state of the current history
   int64_t tail_saved_for;  // history length whose tail-block key sum sits in the saved-tail buffer (-1: none)
   int nsm;
-  CUtensorMap tm_k, tm_v, tm_state, tm_kc, tm_vc, tm_olin;
+  CUtensorMap tm_k, tm_v, tm_state, tm_kc, tm_vc, tm_olin, tm_ek, tm_ev;
   int32_t n_segs;  // Linformer: complete segments compressed so far
   std::vector<int32_t> page_table_host;  // history block -> physical page
   std::vector<uint8_t> resident;         // per history block: tiles present in the pool (tier migration)
@@ -175,6 +175,19 @@ int encode_q(CUtensorMap* tm, const void* q, int n_q, int H, int D, int64_t ts, 
   CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box,
                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HSA_OK : HSA_ERR_CUDA;
+}
+
+int encode_proj(CUtensorMap* tm, const void* e, int H, int seg_tokens, int rank) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return HSA_ERR_CUDA;
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(rank), static_cast<cuuint64_t>(seg_tokens), static_cast<cuuint64_t>(H)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(rank) * 2, static_cast<cuuint64_t>(seg_tokens) * rank * 2};
+  cuuint32_t box[3] = {64, 64, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(e), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? HSA_OK : HSA_ERR_CUDA;
 }
 
@@ -293,6 +306,9 @@ int hsa_create(hsa_ctx** out, const hsa_config* cfg, const hsa_buffers* bufs,
     const uint64_t crows = static_cast<uint64_t>(ctx->lay.n_cpages) * cfg->num_heads * kBlock;
     r = encode_2d_rows(&ctx->tm_kc, bufs->kc_pool, crows, D);
     if (r == HSA_OK) r = encode_2d_rows(&ctx->tm_vc, bufs->vc_pool, crows, D);
+    // projection weights [H][seg_tokens][rank]: boxes of 64 r x 64 tokens of one head
+    if (r == HSA_OK) r = encode_proj(&ctx->tm_ek, bufs->e_k, cfg->num_heads, cfg->lin_seg_tokens, cfg->lin_rank);
+    if (r == HSA_OK) r = encode_proj(&ctx->tm_ev, bufs->e_v, cfg->num_heads, cfg->lin_seg_tokens, cfg->lin_rank);
   }
   if (r != HSA_OK) { delete ctx; return r; }
   *out = ctx;
@@ -346,7 +362,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     return HSA_ERR_UNSUPPORTED;  // this mode appends whole segments only
   AppendMaps maps;
   const bool fused = a.D == 128 && a.lin_state;
-  if (fused) {
+  if (fused || linformer) {
     if (encode_q(&maps.kin, k, n_tokens, a.H, a.D, tok_stride, head_stride, kBlock) != HSA_OK ||
         encode_q(&maps.vin, v, n_tokens, a.H, a.D, tok_stride, head_stride, kBlock) != HSA_OK)
       return HSA_ERR_CUDA;
@@ -371,7 +387,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     la.seg_tokens = ctx->cfg.lin_seg_tokens;
     la.seg_index = ctx->n_segs;
     la.status = a.status;
-    e = launch_linformer_compress(la, static_cast<cudaStream_t>(stream));
+    e = launch_linformer_compress(la, ctx->tm_ek, ctx->tm_ev, maps.kin, maps.vin, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->n_segs += 1;
   }

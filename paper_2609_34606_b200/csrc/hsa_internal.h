@@ -172,7 +172,8 @@ struct AppendMaps {
   CUtensorMap kin, vin, kpool, vpool;
 };
 cudaError_t launch_append(const AppendArgs& a, const AppendMaps* maps, cudaStream_t st);
-cudaError_t launch_linformer_compress(const LinformerArgs& a, cudaStream_t st);
+cudaError_t launch_linformer_compress(const LinformerArgs& a, const CUtensorMap& tm_ek, const CUtensorMap& tm_ev,
+                                      const CUtensorMap& tm_kin, const CUtensorMap& tm_vin, cudaStream_t st);
 cudaError_t linformer_init();
 struct AdaptiveArgs {
   double* sorted_w;      // [H][n_groups][max_pages] softmax numerators in sorted order

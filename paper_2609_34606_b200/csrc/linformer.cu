@@ -5,8 +5,10 @@
 //
 // One CTA computes a [128 rows of r] x [128 dims] tile of K~ or V~ for one head:
 //   C (fp32 in TMEM) = sum over token blocks of  E[tokens, 128 r]^T  X[tokens, 128 d]
-// with both operands staged in shared memory in the 128-byte-swizzled MN-major layout (tcgen05,
-// K = tokens), double-buffered against the next block's loads, and writes bf16 rows to the pool.
+// One lane brings the [64 tokens x 128] tiles of E and of X into a four-stage ring by TMA (both land
+// in the 128-byte-swizzled MN-major layout the tensor cores take as they are; rows past the end of
+// the segment arrive as zeros), one lane issues four tcgen05 MMAs per block (K = tokens) and hands the
+// stage back, and at the end all warps write the bf16 rows to the compressed pool.
 #include <cuda_bf16.h>
 
 #include "hsa_internal.h"
@@ -17,14 +19,14 @@ namespace hsa {
 namespace {
 
 constexpr int kLcThreads = 512;
-constexpr int kLcRowGroups = kLcThreads / 16;
-constexpr int kLcRows = kBlock / kLcRowGroups;  // 2 token rows per thread and block
+constexpr int kLcDepth = 4;
 constexpr int kLcTile = 64 * 128 * 2;
 constexpr int kLcStage = 2 * kLcTile;  // E tile | X tile
-constexpr int kLcSmem = 2 * kLcStage + 64 + 1024;
+constexpr int kLcSmem = kLcDepth * kLcStage + 256 + 1024;
 
 struct LcBars {
-  uint64_t mma_done[2];
+  uint64_t full[kLcDepth];
+  uint64_t empty[kLcDepth];
   uint64_t all_done;
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -43,26 +45,29 @@ __device__ __forceinline__ bool lc_wait(uint64_t* bar, uint32_t parity, LcBars* 
 
 }  // namespace
 
-__global__ void __launch_bounds__(kLcThreads, 1) linformer_compress_kernel(LinformerArgs a) {
+__global__ void __launch_bounds__(kLcThreads, 1)
+linformer_compress_kernel(LinformerArgs a, const __grid_constant__ CUtensorMap tm_ek, const __grid_constant__ CUtensorMap tm_ev,
+                          const __grid_constant__ CUtensorMap tm_kin, const __grid_constant__ CUtensorMap tm_vin) {
   constexpr int D = 128;
   extern __shared__ uint8_t lc_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(lc_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  LcBars* bars = reinterpret_cast<LcBars*>(smem + 2 * kLcStage);
+  LcBars* bars = reinterpret_cast<LcBars*>(smem + kLcDepth * kLcStage);
   const int h = blockIdx.y;
   const int rtiles = a.rank / 128;
   const int which = blockIdx.x / rtiles;  // 0: keys, 1: values
   const int rt = blockIdx.x % rtiles;
-  const __nv_bfloat16* E = (which == 0 ? a.e_k : a.e_v) + static_cast<size_t>(h) * a.seg_tokens * a.rank + rt * 128;
-  const __nv_bfloat16* X = (which == 0 ? a.k : a.v) + static_cast<size_t>(h) * a.head_stride;
+  const CUtensorMap* tm_e = which == 0 ? &tm_ek : &tm_ev;  // [H][seg_tokens][rank], box 64 r x 64 tokens
+  const CUtensorMap* tm_x = which == 0 ? &tm_kin : &tm_vin;  // [tokens][H][d], box 64 d x 1 x 64 tokens
   __nv_bfloat16* pool = which == 0 ? a.kc_pool : a.vc_pool;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ch = threadIdx.x & 15, rg = threadIdx.x >> 4;
   const int nblk = (a.seg_tokens + kBlock - 1) / kBlock;
 
   if (threadIdx.x == 0) {
-    mbar_init(&bars->mma_done[0], 1);
-    mbar_init(&bars->mma_done[1], 1);
+    for (int s = 0; s < kLcDepth; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
     mbar_init(&bars->all_done, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -77,64 +82,46 @@ __global__ void __launch_bounds__(kLcThreads, 1) linformer_compress_kernel(Linfo
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
-  uint4 ereg[kLcRows], xreg[kLcRows];
-  auto load_block = [&](int bi, uint4 (&ee)[kLcRows], uint4 (&xx)[kLcRows]) {
-#pragma unroll
-    for (int i = 0; i < kLcRows; ++i) {
-      const int t = bi * kBlock + rg + kLcRowGroups * i;
-      if (t < a.seg_tokens) {
-        ee[i] = *reinterpret_cast<const uint4*>(E + static_cast<size_t>(t) * a.rank + ch * 8);
-        xx[i] = *reinterpret_cast<const uint4*>(X + static_cast<size_t>(t) * a.tok_stride + ch * 8);
-      } else {  // rows past the end of the segment contribute nothing
-        ee[i] = make_uint4(0, 0, 0, 0);
-        xx[i] = make_uint4(0, 0, 0, 0);
+  if (warp == 1) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (elect_one_sync()) {
+      for (int bi = 0; bi < nblk; ++bi) {
+        const int s = bi % kLcDepth;
+        if (bi >= kLcDepth && !lc_wait(&bars->empty[s], ((bi / kLcDepth) - 1) & 1, bars, a.status)) break;
+        uint8_t* st_e = smem + s * kLcStage;
+        uint8_t* st_x = st_e + kLcTile;
+        mbar_expect_tx(&bars->full[s], kLcStage);
+        for (int half = 0; half < 2; ++half) {
+          tma_load_3d(st_e + half * (kLcTile / 2), tm_e, &bars->full[s], rt * 128 + half * 64, bi * kBlock, h);
+          tma_load_3d(st_x + half * (kLcTile / 2), tm_x, &bars->full[s], half * 64, h, bi * kBlock);
+        }
       }
     }
-  };
-  load_block(0, ereg, xreg);
-  bool ok = true;
-#pragma unroll 1
-  for (int bi = 0; bi < nblk; ++bi) {
-    const int stage = bi & 1;
-    uint8_t* st_e = smem + stage * kLcStage;
-    uint8_t* st_x = st_e + kLcTile;
-    uint4 enext[kLcRows], xnext[kLcRows];
-    if (bi + 1 < nblk) load_block(bi + 1, enext, xnext);
-    if (bi >= 2) ok = lc_wait(&bars->mma_done[stage], ((bi >> 1) - 1) & 1, bars, a.status) && ok;
-#pragma unroll
-    for (int i = 0; i < kLcRows; ++i) {
-      const int r = rg + kLcRowGroups * i;
-      const uint32_t soff = (ch >> 3) * (kLcTile / 2) + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
-      *reinterpret_cast<uint4*>(st_e + soff) = ereg[i];
-      *reinterpret_cast<uint4*>(st_x + soff) = xreg[i];
-    }
-    fence_proxy_async_smem();
-    __syncthreads();
-    if (warp == 0) {
-      if (elect_one_sync() && ok) {
+  } else if (warp == 0) {
+    // ------------------------------------------------------------------ MMA issuer (one lane)
+    if (elect_one_sync()) {
+      constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 1, 1);
+      constexpr uint32_t hi = desc_hi_sw128(1024);
+      bool ok = true;
+      for (int bi = 0; bi < nblk && ok; ++bi) {
+        const int s = bi % kLcDepth;
+        ok = lc_wait(&bars->full[s], (bi / kLcDepth) & 1, bars, a.status);
+        if (!ok) break;
         tc_fence_after();
-        constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 1, 1);
-        constexpr uint32_t hi = desc_hi_sw128(1024);
-        const uint32_t a_lo = desc_lo_sw128(smem_u32(st_e), kLcTile / 2);
-        const uint32_t b_lo = desc_lo_sw128(smem_u32(st_x), kLcTile / 2);
+        const uint32_t a_lo = desc_lo_sw128(smem_u32(smem + s * kLcStage), kLcTile / 2);
+        const uint32_t b_lo = desc_lo_sw128(smem_u32(smem + s * kLcStage + kLcTile), kLcTile / 2);
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
           tc_mma_ss_lo(tmem, a_lo + kk * 128, b_lo + kk * 128, hi, idesc, (bi > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(&bars->mma_done[stage]);
+        tc_commit(&bars->empty[s]);
       }
-    }
-#pragma unroll
-    for (int i = 0; i < kLcRows; ++i) {
-      ereg[i] = enext[i];
-      xreg[i] = xnext[i];
+      tc_commit(&bars->all_done);
     }
   }
-  if (warp == 0) {
-    if (elect_one_sync()) tc_commit(&bars->all_done);
-  }
-  ok = lc_wait(&bars->all_done, 0, bars, a.status) && ok;
+  __syncwarp();
+  const bool ok = lc_wait(&bars->all_done, 0, bars, a.status);
   tc_fence_after();
-  {
+  if (ok) {
     const int quad = warp & 3, part = warp >> 2;
     const int rr = rt * 128 + quad * 32 + lane;  // row of the compressed segment
     uint32_t v[32];
@@ -162,9 +149,10 @@ cudaError_t linformer_init() {
                               kLcSmem);
 }
 
-cudaError_t launch_linformer_compress(const LinformerArgs& a, cudaStream_t st) {
+cudaError_t launch_linformer_compress(const LinformerArgs& a, const CUtensorMap& tm_ek, const CUtensorMap& tm_ev,
+                                      const CUtensorMap& tm_kin, const CUtensorMap& tm_vin, cudaStream_t st) {
   dim3 grid(2 * (a.rank / 128), a.H);
-  linformer_compress_kernel<<<grid, kLcThreads, kLcSmem, st>>>(a);
+  linformer_compress_kernel<<<grid, kLcThreads, kLcSmem, st>>>(a, tm_ek, tm_ev, tm_kin, tm_vin);
   return cudaGetLastError();
 }
 
