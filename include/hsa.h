@@ -140,7 +140,9 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens,
  *   sel_idx_dev      device int32[H][n_groups][max_topk], ascending block ids (output).
  *   sel_cnt_dev      device int32[H][n_groups] (output).
  * Candidates: blocks with at least one token and, if causal, first token <= last query
- * position of the group.  Counts are clamped to max_topk (flagged in the status word). */
+ * position of the group.  Counts are clamped to max_topk (flagged in the status word).
+ * The work is enqueued as one or two kernels (see HSA_CFG_GRID_BARRIER_SELECT); the lists are the
+ * same bit for bit either way. */
 int hsa_select_blocks(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride,
                       int64_t head_stride, int64_t q_pos0, int32_t causal,
                       const int32_t* budgets_dev, int32_t q_group_tokens,
