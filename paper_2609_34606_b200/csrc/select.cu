@@ -231,26 +231,50 @@ __device__ __forceinline__ void scores_item(const Blk& blk, const SelectArgs& a,
   constexpr int NB = kScoreBlocksPerCta / 8;  // candidates per warp
   constexpr int NP = MIXED ? 2 : 1;           // pages per candidate at most
   auto& kv = op.kv;
+  // this lane's part of the NB dot products (fp64), then ONE reduction for all of them: at each of
+  // the first steps a lane hands half of its values to its partner and keeps the other half
+  // (value i ends up in the lanes whose bits 4, 3 (NB = 4) spell i), the remaining steps add single
+  // values -- NB + 2 adds and 2 NB - 2 + 3 exchanges instead of 5 adds and 5 exchanges per candidate
+  static_assert(NB == 4, "the reduction below is written for four candidates per warp");
+  double dot[NB];
 #pragma unroll
   for (int i = 0; i < NB; ++i) {
-    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
-    if (c >= cg.nc) continue;  // warp-uniform
-    double dot = 0.0;
+    dot[i] = 0.0;
 #pragma unroll
     for (int e = 0; e < PER; ++e)
-      dot += qs[lane * PER + e] * (static_cast<double>(kv[i][0][e]) + (MIXED ? static_cast<double>(kv[i][NP - 1][e]) : 0.0));
+      dot[i] += qs[lane * PER + e] * (static_cast<double>(kv[i][0][e]) + (MIXED ? static_cast<double>(kv[i][NP - 1][e]) : 0.0));
+  }
+  {
+    // step 1 (partner lane ^ 16): lanes with bit 4 clear keep candidates 0, 1 and give 2, 3
+    const bool up = (lane & 16) != 0;
+    const double g0 = up ? dot[0] : dot[2], g1 = up ? dot[1] : dot[3];
+    const double k0 = up ? dot[2] : dot[0], k1 = up ? dot[3] : dot[1];
+    dot[0] = k0 + __shfl_xor_sync(0xffffffffu, g0, 16);
+    dot[1] = k1 + __shfl_xor_sync(0xffffffffu, g1, 16);
+    // step 2 (partner lane ^ 8): lanes with bit 3 clear keep the first of their two
+    const bool up2 = (lane & 8) != 0;
+    const double g = up2 ? dot[0] : dot[1], k = up2 ? dot[1] : dot[0];
+    dot[0] = k + __shfl_xor_sync(0xffffffffu, g, 8);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    if (lane == 0) {
+    for (int o = 4; o > 0; o >>= 1) dot[0] += __shfl_xor_sync(0xffffffffu, dot[0], o);
+  }
+  // lanes 0, 8, 16, 24 now hold the sums of candidates 0, 1, 2, 3 (lane bits 4, 3 = candidate: bit 4
+  // chose between {0, 1} and {2, 3}, bit 3 inside the pair)
+  if ((lane & 7) == 0) {
+    const int i = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+    const int c = chunk * kScoreBlocksPerCta + i * 8 + warp;
+    if (c < cg.nc) {
       const int64_t t0 = static_cast<int64_t>(cand_first_page<MIXED>(cg, c)) * kBlock;
       const int64_t cnt = min64(static_cast<int64_t>(cand_pages<MIXED>(cg, c)) * kBlock, a.n_tokens - t0);
-      uint32_t key = order_key(static_cast<float>(dot / static_cast<double>(cnt)));
+      // a full block's mean is an exact scaling; only a partly filled block needs the division
+      const double mean = cnt == kBlock ? dot[0] * (1.0 / kBlock) : dot[0] / static_cast<double>(cnt);
+      uint32_t key = order_key(static_cast<float>(mean));
       if (MIXED && a.kv_pages != nullptr && c < cg.ni) {
         // every page of the candidate must lie in a retrieved KV page; key 0 marks "no candidate"
         const int pf = cand_first_page<MIXED>(cg, c), pl = pf + cand_pages<MIXED>(cg, c) - 1;
         bool in_f = false, in_l = false;
-        for (int i = 0; i < a.n_kv_pages; ++i) {
-          const int kp = a.kv_pages[i];
+        for (int j = 0; j < a.n_kv_pages; ++j) {
+          const int kp = a.kv_pages[j];
           in_f |= (pf / a.kv_page_blocks == kp);
           in_l |= (pl / a.kv_page_blocks == kp);
         }
