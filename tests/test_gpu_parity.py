@@ -842,12 +842,13 @@ def test_cluster_and_grid_barrier_forms_of_the_selection_agree(name, group_token
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("n_rep,budget", [(40, 7), (300, 129), (600, 1), (600, 599)])
+@pytest.mark.parametrize("n_rep,budget", [(40, 7), (300, 129), (600, 1), (600, 599), (6400, 1000)])
 def test_selection_exact_ties_go_to_the_lower_block_index(n_rep, budget, cuda_device):
     """A history made of one 64-token block repeated n_rep times, followed by one distinct block:
     the repeated blocks have bit-identical pooled scores, so the budget cuts through a group of exact
     ties, which must go to the lower block indices (in every thread's range of the compaction, with
-    one key per thread and with several).  Checked against the oracle's selection as well."""
+    one key per thread and with several; the longest case is beyond what a thread keeps in registers
+    and takes the form that walks shared memory).  Checked against the oracle's selection as well."""
     from paper_2609_34606_b200 import hsa
     H, d = 2, 128
     gen = torch.Generator().manual_seed(1234 + n_rep)
@@ -871,10 +872,14 @@ def test_selection_exact_ties_go_to_the_lower_block_index(n_rep, budget, cuda_de
     for h in range(H):
         b = int(budgets[h])
         s = scores[h, 0]
-        assert np.all(s[:n_rep] == s[0]), "the repeated blocks must tie exactly in the oracle too"
+        # (over thousands of blocks numpy's block means differ in the last bit from block to block:
+        # there the oracle's own list is not held to the lowest indices, the GPU's is)
+        exact = bool(np.all(s[:n_rep] == s[0]))
+        assert exact or (n_rep > 1000 and np.ptp(s[:n_rep]) < 1e-12), "the repeated blocks must tie in the oracle too"
         # the distinct block either beats the ties or not; the rest of the budget is the lowest indices
         want = [n_rep] if s[n_rep] > s[0] else []
         want = sorted(list(range(b - len(want))) + want)
         assert got[h][0].tolist() == want
-        assert ref[h][0].tolist() == want
+        if exact:
+            assert ref[h][0].tolist() == want
     ctx.destroy()
