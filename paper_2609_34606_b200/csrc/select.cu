@@ -332,8 +332,10 @@ __device__ __forceinline__ void scores_item_groups(const Blk& blk, const SelectA
     const int c = c0 + 2 * (lane & 3) + t;
     const int fp = c < cg.nc ? cand_first_page<MIXED>(cg, c) : 0;
     const int np = c < cg.nc ? cand_pages<MIXED>(cg, c) : 0;
-    inv_cnt[t] = 1.0 / static_cast<double>(max64(1, min64(static_cast<int64_t>(np) * kBlock,
-                                                          a.n_tokens - static_cast<int64_t>(fp) * kBlock)));
+    // (fp64 division is a long instruction sequence on a slow pipe: a full page's count is a power
+    // of two, only a partly filled candidate needs the division)
+    const int64_t cnt = max64(1, min64(static_cast<int64_t>(np) * kBlock, a.n_tokens - static_cast<int64_t>(fp) * kBlock));
+    inv_cnt[t] = cnt == kBlock ? 1.0 / kBlock : 1.0 / static_cast<double>(cnt);
     masked[t] = false;
     if (MIXED && a.kv_pages != nullptr && c < cg.ni) {
       const int pl = fp + np - 1;
@@ -347,6 +349,7 @@ __device__ __forceinline__ void scores_item_groups(const Blk& blk, const SelectA
     }
   }
   const int tiles_per_group = gtok / kTileM;
+  const double mean_scale_full = static_cast<double>(a.scale) / static_cast<double>(gtok);  // all groups but a short last one
   for (int g0 = 0; g0 < a.n_groups; g0 += GB) {
     // mean queries of groups g0 .. g0 + 15 (tile sums added in ascending tile order, fp64)
     constexpr int NV = GB * D / 256;  // values per thread
@@ -370,7 +373,8 @@ __device__ __forceinline__ void scores_item_groups(const Blk& blk, const SelectA
       const int idx = blk.tid + 256 * v;
       const int gi = idx / D, g = g0 + gi;
       const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
-      qs[gi * PITCH + idx % D] = g < a.n_groups ? sum[v] * (static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo)) : 0.0;
+      const double ms = (q_hi - q_lo == gtok) ? mean_scale_full : static_cast<double>(a.scale) / static_cast<double>(q_hi - q_lo);
+      qs[gi * PITCH + idx % D] = g < a.n_groups ? sum[v] * ms : 0.0;
     }
     blk_sync(blk);
     const int row0 = 8 * (warp >> 2);  // this warp's eight rows of the batch
@@ -693,13 +697,15 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   const int h = static_cast<int>(blockIdx.x) / cluster_ctas;
   const int slot = (static_cast<int>(blockIdx.x) % cluster_ctas) * kSubBlocks + sub;
   const int n_slots = cluster_ctas * kSubBlocks;
-  // launched as a programmatic dependent: the kernel before this one is complete from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int n_chunks = (cand_geom<MIXED>(a).nc + kScoreBlocksPerCta - 1) / kScoreBlocksPerCta;
   // (one list per head: the launcher sends per-tile selections to the grid-barrier form)
-  // the key sums of this block's first score item are requested first
+  // The key sums of this block's first score item are requested first, ahead of the wait for the
+  // kernel before this one: that kernel (the query tile sums) writes none of them, and it has itself
+  // waited for everything before it, so they are final when any CTA of this grid runs.
   ScoreOperands<D, MIXED> op;
   if (slot < n_chunks) scores_load<D, MIXED>(blk, a, slot, h, op);
+  // launched as a programmatic dependent: the kernel before this one is complete from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
     scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot);
     blk_sync(blk);
