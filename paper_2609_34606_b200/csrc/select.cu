@@ -982,12 +982,14 @@ cudaError_t launch_pdl(const void* fn, dim3 grid, dim3 block, size_t smem, void*
 //   cluster form        query tile sums as a kernel of their own (they read the whole chunk and want
 //                       every SM), then one cluster of 8 CTAs per head for scores and lists, with one
 //                       hardware cluster barrier between them -- the default for one list per head while
-//                       a head has at most kClusterMaxChunks score items (short and medium histories)
-//   grid-barrier form   one cooperative launch over all SMs with two device barriers -- long histories
-//                       (the score stage then wants every SM too), one list per query tile (37 x H
-//                       lists want more than 24 blocks of threads per head), and on request
+//                       a head has at most kClusterMaxChunks score items (6144 blocks; measured against
+//                       the grid-barrier form: 17.1 against 20.0 us at 2194 blocks, 24.8 against 25.1 us
+//                       at 4388)
+//   grid-barrier form   one cooperative launch over all SMs with two device barriers -- histories
+//                       beyond that, one list per query tile (37 x H lists want more than 24 blocks
+//                       of threads per head), and on request
 //   three launches      for devices without cooperative launch and for callers without a barrier word
-constexpr int kClusterMaxChunks = 2 * 8 * kSubBlocks;
+constexpr int kClusterMaxChunks = 192;
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
   int nsm = 0;
