@@ -301,8 +301,10 @@ int hsa_device_status(hsa_ctx* ctx, int32_t* status_out);
 int hsa_set_wait_limit_ns(hsa_ctx* ctx, uint64_t wait_ns);
 
 /* Byte offsets inside the workspace, for tests and monitoring: the int32 status word, and the
- * two uint32 words {arrive count, generation} of the selection kernel's grid barrier (the count
- * is zero whenever no selection kernel is running; the generation advances by two per launch). */
+ * two uint32 words {arrive count, generation} of the selection kernel's grid barrier, which the
+ * kernel updates together as one 8-byte word (off_barrier is 8-byte aligned; the count is zero
+ * whenever no selection kernel is running; the generation advances by two per launch of the
+ * grid-barrier form). */
 int hsa_workspace_layout(hsa_ctx* ctx, size_t* off_status, size_t* off_barrier);
 
 /* Synchronises the device, reads and clears a counter: the number of (query tile, head) work
