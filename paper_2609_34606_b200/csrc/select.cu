@@ -190,10 +190,12 @@ __device__ __forceinline__ void scores_load(const Blk& blk, const SelectArgs& a,
 }
 
 // rebuild = false: qs[0, D) still holds the mean query of this (group, head) from the item before;
-// loaded = true: `op` already holds this item's key sums
+// loaded = true: `op` already holds this item's key sums; keys_cluster_addr != 0: where the keys go
+// instead of the workspace
 template <int D, bool MIXED>
 __device__ __forceinline__ void scores_item(const Blk& blk, const SelectArgs& a, int chunk, int g, int h, double* qs,
-                                            ScoreOperands<D, MIXED>& op, bool rebuild = true, bool loaded = false) {
+                                            ScoreOperands<D, MIXED>& op, bool rebuild = true, bool loaded = false,
+                                            uint32_t keys_cluster_addr = 0) {
   const int lane = blk.tid & 31, warp = blk.tid >> 5;
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_lo = g * gtok, q_hi = min(a.n_q, q_lo + gtok);
@@ -280,7 +282,12 @@ __device__ __forceinline__ void scores_item(const Blk& blk, const SelectArgs& a,
         }
         if (!(in_f && in_l)) key = 0u;
       }
-      keys[c] = key;
+      // cluster form: straight into the key array of the CTA that extracts the list (a
+      // shared::cluster address), else into the workspace
+      if (keys_cluster_addr)
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(keys_cluster_addr + 4u * static_cast<uint32_t>(c)), "r"(key) : "memory");
+      else
+        keys[c] = key;
     }
   }
 }
@@ -552,8 +559,10 @@ __device__ __forceinline__ int topk_range(const Blk& blk, const uint32_t* keys, 
   return total;
 }
 
+// keys_in_place: `keys` already holds the head's score keys (the cluster form writes them there)
 template <bool MIXED>
-__device__ __forceinline__ void topk_item(const Blk& blk, const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh) {
+__device__ __forceinline__ void topk_item(const Blk& blk, const SelectArgs& a, int g, int h, uint32_t* keys, TopkShared* sh,
+                                          int budget, int intra_budget, bool keys_in_place = false) {
   const CandGeom cg = cand_geom<MIXED>(a);
   const int gtok = a.group_tokens > 0 ? a.group_tokens : a.n_q;
   const int q_hi = min(a.n_q, g * gtok + gtok);
@@ -562,7 +571,8 @@ __device__ __forceinline__ void topk_item(const Blk& blk, const SelectArgs& a, i
   // last query position
   const int ncand = a.causal ? cand_visible<MIXED>(cg, p_last) : cg.nc;
   const uint32_t* gkeys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
-  for (int b = blk.tid; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
+  if (!keys_in_place)
+    for (int b = blk.tid; b < ncand; b += 256) keys[b] = __ldcg(&gkeys[b]);
   if (blk.tid == 0) {
     sh->prefix = 0;
     sh->krem = 0;
@@ -571,10 +581,9 @@ __device__ __forceinline__ void topk_item(const Blk& blk, const SelectArgs& a, i
   int32_t* out = a.sel_idx + (static_cast<size_t>(h) * a.n_groups + g) * a.kcap;
   // inter-chunk candidates against the head's budget, then intra-chunk ones against theirs
   const int n_inter = min(ncand, cg.ni);
-  int total = topk_range<MIXED>(blk, keys, n_inter, a.budgets[h], cg, 0, out, 0, a.kcap, sh, a.kv_pages != nullptr);
+  int total = topk_range<MIXED>(blk, keys, n_inter, budget, cg, 0, out, 0, a.kcap, sh, a.kv_pages != nullptr);
   if (MIXED && ncand > n_inter)
-    total += topk_range<MIXED>(blk, keys + n_inter, ncand - n_inter, a.intra_budgets ? a.intra_budgets[h] : -1, cg, cg.ni, out,
-                        total, a.kcap, sh, false);
+    total += topk_range<MIXED>(blk, keys + n_inter, ncand - n_inter, intra_budget, cg, cg.ni, out, total, a.kcap, sh, false);
   if (blk.tid == 0) {
     a.sel_cnt[static_cast<size_t>(h) * a.n_groups + g] = min(total, a.kcap);
     if (total > a.kcap) atomicCAS(a.status, 0, kDevBounds);
@@ -587,7 +596,9 @@ __global__ void __launch_bounds__(256) topk_kernel(SelectArgs a) {
   __shared__ TopkShared sh;
   asm volatile("griddepcontrol.wait;" ::: "memory");  // (see qsum_partial_kernel)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  topk_item<MIXED>(Blk{static_cast<int>(threadIdx.x), 0}, a, blockIdx.x, blockIdx.y, topk_keys, &sh);
+  const int h = blockIdx.y;
+  topk_item<MIXED>(Blk{static_cast<int>(threadIdx.x), 0}, a, blockIdx.x, h, topk_keys, &sh, a.budgets[h],
+                   (MIXED && a.intra_budgets) ? a.intra_budgets[h] : -1);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -656,7 +667,8 @@ __global__ void __launch_bounds__(256, 3) select_fused_kernel(SelectArgs a) {
   // may take their places and do its set-up meanwhile.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   for (int it = blockIdx.x; it < a.n_groups * a.H; it += gridDim.x) {
-    topk_item<MIXED>(blk, a, it % a.n_groups, it / a.n_groups, fused_keys, &sh);
+    const int h = it / a.n_groups;
+    topk_item<MIXED>(blk, a, it % a.n_groups, h, fused_keys, &sh, a.budgets[h], (MIXED && a.intra_budgets) ? a.intra_budgets[h] : -1);
     __syncthreads();
   }
 }
@@ -706,14 +718,24 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   if (slot < n_chunks) scores_load<D, MIXED>(blk, a, slot, h, op);
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the budgets are asked for now by the block that will need them, far ahead of their use
+  int budget = 0, intra_budget = -1;
+  if (slot == 0) {
+    budget = a.budgets[h];
+    if (MIXED && a.intra_budgets) intra_budget = a.intra_budgets[h];
+  }
+  // the score keys go straight into the key array of the cluster's first CTA (distributed shared
+  // memory), where the lists are extracted: no trip through global memory between the two stages
+  uint32_t keys_addr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(keys_addr) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(cl_keys))), "r"(0u));
   for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
-    scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot);
+    scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot, keys_addr);
     blk_sync(blk);
   }
-  cluster_sync_all();  // the score keys of the head are complete and visible to its cluster
+  cluster_sync_all();  // the score keys of the head are complete and visible to its first CTA
   // the kernel behind this one may take the places of the CTAs that leave now
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (slot == 0) topk_item<MIXED>(blk, a, 0, h, cl_keys, sh_all);
+  if (slot == 0) topk_item<MIXED>(blk, a, 0, h, cl_keys, sh_all, budget, intra_budget, true);
 }
 
 // ---------------------------------------------------------------------------------------
