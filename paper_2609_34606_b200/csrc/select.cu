@@ -691,7 +691,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 
 template <int D>
 struct ClusterSmem {
-  static constexpr int kScratch = (D + 256) * 8;  // mean query + its per-way partial sums, fp64
+  static constexpr int kScratch = (D + 256) * 8;  // per sub-block; together: mean query [D] + partial sums [768 / D][D], fp64
   static constexpr int kFixed = (kSubBlocks * kScratch + static_cast<int>(sizeof(TopkShared)) + 15) / 16 * 16;
 };
 
@@ -703,7 +703,6 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   constexpr int kScratch = ClusterSmem<D>::kScratch;
   const int sub = static_cast<int>(threadIdx.x) / 256;
   const Blk blk{static_cast<int>(threadIdx.x) % 256, 1 + sub};
-  unsigned char* scratch = cl_smem + sub * kScratch;
   TopkShared* sh_all = reinterpret_cast<TopkShared*>(cl_smem + kSubBlocks * kScratch);
   uint32_t* cl_keys = reinterpret_cast<uint32_t*>(cl_smem + ClusterSmem<D>::kFixed);
   const int h = static_cast<int>(blockIdx.x) / cluster_ctas;
@@ -718,6 +717,34 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   if (slot < n_chunks) scores_load<D, MIXED>(blk, a, slot, h, op);
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // The head's mean query, once per CTA: all 768 threads add up the tile sums (a column's partials
+  // split over 768 / D ways, every load of a thread in flight at once, fp64, fixed order), then one
+  // thread per column adds the ways.  The three sub-blocks share the result.
+  double* qmean = reinterpret_cast<double*>(cl_smem);  // [D], then the per-way partial sums [WAYS][D]
+  {
+    constexpr int WAYS = 256 * kSubBlocks / D;
+    constexpr int kInFlight = 8;
+    const int tid = static_cast<int>(threadIdx.x), col = tid % D, way = tid / D;
+    const int n_tiles = (a.n_q + kTileM - 1) / kTileM;
+    double sum = 0.0;
+    for (int t0 = way; t0 < n_tiles; t0 += kInFlight * WAYS) {
+      float v[kInFlight];
+#pragma unroll
+      for (int i = 0; i < kInFlight; ++i)
+        v[i] = (t0 + i * WAYS < n_tiles) ? __ldcg(&a.qpart[(static_cast<size_t>(t0 + i * WAYS) * a.H + h) * D + col]) : 0.f;
+#pragma unroll
+      for (int i = 0; i < kInFlight; ++i) sum += static_cast<double>(v[i]);
+    }
+    qmean[D + way * D + col] = sum;
+    __syncthreads();
+    if (tid < D) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < WAYS; ++w) t += qmean[D + w * D + tid];
+      qmean[tid] = t / static_cast<double>(a.n_q) * static_cast<double>(a.scale);
+    }
+    __syncthreads();
+  }
   // the budgets are asked for now by the block that will need them, far ahead of their use
   int budget = 0, intra_budget = -1;
   if (slot == 0) {
@@ -729,7 +756,7 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   uint32_t keys_addr;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(keys_addr) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(cl_keys))), "r"(0u));
   for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
-    scores_item<D, MIXED>(blk, a, chunk, 0, h, reinterpret_cast<double*>(scratch), op, chunk == slot, chunk == slot, keys_addr);
+    scores_item<D, MIXED>(blk, a, chunk, 0, h, qmean, op, false, chunk == slot, keys_addr);
     blk_sync(blk);
   }
   cluster_sync_all();  // the score keys of the head are complete and visible to its first CTA
