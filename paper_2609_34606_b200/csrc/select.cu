@@ -715,6 +715,10 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   // waited for everything before it, so they are final when any CTA of this grid runs.
   ScoreOperands<D, MIXED> op;
   if (slot < n_chunks) scores_load<D, MIXED>(blk, a, slot, h, op);
+  // A CTA's shared memory may be written by its peers only once it runs: every CTA says so here and
+  // checks, before its first such write, that all of the cluster have (the two halves of one
+  // cluster barrier; by then nobody waits).
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   // launched as a programmatic dependent: the kernel before this one is complete from here on
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // The head's mean query, once per CTA: all 768 threads add up the tile sums (a column's partials
@@ -755,6 +759,7 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   // memory), where the lists are extracted: no trip through global memory between the two stages
   uint32_t keys_addr;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(keys_addr) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(cl_keys))), "r"(0u));
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // every CTA of the cluster is running
   for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
     scores_item<D, MIXED>(blk, a, chunk, 0, h, qmean, op, false, chunk == slot, keys_addr);
     blk_sync(blk);
