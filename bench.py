@@ -457,9 +457,10 @@ def bench_ours(args, rank: int, world: int):
             "e2e": {"value": agg_e2e / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": 3 * w.Lq * w.H * w.d * 2, "d2h_bytes_per_step": w.Lq * w.H * w.d * 2},
             # per step: append_fused, state_reduce, hsa_forward and the selection -- two kernels (query
-            # sums, then one cluster per head) while a head has at most 48 score items of 32 blocks,
-            # one cooperative kernel beyond that
-            "gpu_launches": ((2 if args.lin == "linformer" else 0) + (5 if w.n_blocks <= 48 * 32 else 4)) * K,
+            # sums, then one cluster per head) for one list per head while a head has at most 192
+            # score items of 32 blocks, one cooperative kernel otherwise
+            "gpu_launches": ((2 if args.lin == "linformer" else 0) +
+                             (5 if (args.group_tokens == 0 and w.n_blocks <= 192 * 32) else 4)) * K,
             # (the Linformer form: page write + projection instead of the fused append, two forward passes)
             "device_status": status,
             "roofline": {"kernel": "hsa_forward_kernel<128, false>", "bound": "tensor", "achieved": fwd_tf,
@@ -562,8 +563,8 @@ def bench_rollout(args, rank: int, world: int):
         "rollout_ms": [r["ms_total"] for r in runs],
         "ms_per_chunk_all_layers": {"first": pc[0], "median": sorted(pc)[len(pc) // 2], "last": pc[-1]},
         "flops_per_step": fl["total"], "clocks": clocks,
-        # (the selection is two kernels while the history has at most 1536 blocks, one beyond that)
-        "gpu_launches": layers * sum(5 if (c + 1) * w.chunk <= 1536 * 64 else 4 for c in range(w.n_chunks)),
+        # (the selection is two kernels while the history has at most 6144 blocks, one beyond that)
+        "gpu_launches": layers * sum(5 if (c + 1) * w.chunk <= 6144 * 64 else 4 for c in range(w.n_chunks)),
         "device_status": status}),
         flush=True)
     for c in ctxs:
