@@ -459,9 +459,9 @@ def bench_ours(args, rank: int, world: int):
             # per step: append_fused, state_reduce, hsa_forward and the selection -- two kernels (query
             # sums, then one cluster per head) for one list per head while a head has at most 192
             # score items of 32 blocks, one cooperative kernel otherwise
-            "gpu_launches": ((2 if args.lin == "linformer" else 0) +
-                             (5 if (args.group_tokens == 0 and w.n_blocks <= 192 * 32) else 4)) * K,
-            # (the Linformer form: page write + projection instead of the fused append, two forward passes)
+            "gpu_launches": (5 if (args.group_tokens == 0 and w.n_blocks <= 192 * 32) else 4) * K,
+            # (the Linformer form has as many: page write + projection instead of the fused append and
+            # its reduction, one forward launch that walks the compressed pool before the selected pages)
             "device_status": status,
             "roofline": {"kernel": "hsa_forward_kernel<128, false>", "bound": "tensor", "achieved": fwd_tf,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tf / peaks["bf16_tflops"],

@@ -25,6 +25,12 @@
 // linear branch and the gates and stores bf16 once.
 // Every barrier wait is bounded; when one gives up the kernel records a timeout in the status
 // word and all roles drain to the common exit.
+//
+// LINF (the Linformer form of the linear branch, Sec. 3.3 Eq. 3): the loop has two segments.  The
+// first runs over every page of the compressed pool (K~, V~), the second over the selected pages;
+// each segment has its own accumulator in TMEM (O_lin | O_sp), its own exponent reference and its
+// own row sums, and the epilogue merges the two normalised results.  TMEM then holds two score
+// buffers instead of three: O_sp | O_lin | S0 | S1.
 #include <cuda_bf16.h>
 
 #include "hsa_internal.h"
@@ -56,7 +62,7 @@ struct Smem {
   static constexpr int kV = kTile + kStages * kTile;
   static constexpr int kStats = kK;  // float[2][128][4], reuses K stage 0 once the loop is over
   static constexpr int kBars = kTile + 2 * kStages * kTile;
-  static constexpr int kTotal = kBars + 1024 + 1024;  // barriers + per-row reference, + slack
+  static constexpr int kTotal = kBars + 1536 + 1024;  // barriers + per-row references, + slack
 };
 
 struct Bars {
@@ -67,15 +73,15 @@ struct Bars {
   uint64_t p_full[kSBufs];
   uint64_t pv_done;
   uint64_t o_done;
-  uint64_t mref_ready;
+  uint64_t mref_ready[2];  // per loop segment
   uint64_t lin_a_full;
   uint64_t lin_done;
   uint32_t tmem_base;
   volatile int abort_flag;
   volatile int redo;
-  float mref[128];  // per-row exponent reference (log2 domain) of the fast pass
+  float mref[2][128];  // per-row exponent reference (log2 domain) of the fast pass, per loop segment
 };
-static_assert(sizeof(Bars) <= 1024, "barrier block must fit its shared-memory slot");
+static_assert(sizeof(Bars) <= 1536, "barrier block must fit its shared-memory slot");
 
 constexpr int kExpLag = 8;  // columns between scale-and-shift, exponential and row sum in the softmax pipeline
 
@@ -141,7 +147,7 @@ __device__ __forceinline__ void init_barriers(Bars* bars) {
   }
   mbar_init(&bars->pv_done, 1);
   mbar_init(&bars->o_done, 1);
-  mbar_init(&bars->mref_ready, 128);  // group 0 publishes the per-row reference
+  for (int i = 0; i < 2; ++i) mbar_init(&bars->mref_ready[i], 128);  // one group publishes the per-row reference
   mbar_init(&bars->lin_a_full, 256);
   mbar_init(&bars->lin_done, 1);
   bars->redo = 0;
@@ -151,12 +157,18 @@ __device__ __forceinline__ void init_barriers(Bars* bars) {
 }  // namespace
 
 // SPLIT: compiled with the split-tile path (grid z > 1); the plain kernel carries none of it
-template <int D, bool SPLIT>
+// LINF: compiled with the compressed-pool segment in front of the selected pages (tm_kc, tm_vc)
+template <int D, bool SPLIT, bool LINF>
 __global__ void __launch_bounds__(kThreads, 1)
 hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ CUtensorMap tm_state,
-                   const __grid_constant__ CUtensorMap tm_out, const FwdParams p) {
+                   const __grid_constant__ CUtensorMap tm_out, const __grid_constant__ CUtensorMap tm_kc,
+                   const __grid_constant__ CUtensorMap tm_vc, const FwdParams p) {
+  static_assert(!(SPLIT && LINF), "split lists and the compressed segment are not combined");
+  constexpr int NSB = LINF ? 2 : kSBufs;                 // score buffers in use
+  constexpr uint32_t kColSb = LINF ? 256 : kColS;        // first score buffer
+  constexpr uint32_t kColLn = LINF ? 128 : kColLin;      // linear-branch accumulator
   using L = Smem<D>;
   constexpr int DH = D / 64;  // 64-element (128-byte) slabs per row
   extern __shared__ uint8_t smem_raw[];
@@ -256,7 +268,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
   }
   const int slot = (tile * p.H + h) * p.max_splits + part;  // this CTA's partial-result slot
-  const int nsteps = (cnt + 1) / 2;
+  // steps of the compressed segment (LINF), then of the selected pages
+  const int lf_pages = LINF ? p.lf_pages : 0;
+  const int nA = (lf_pages + 1) / 2;
+  const int nsteps = nA + (cnt + 1) / 2;
+  // pages of step j (1 or 2) and whether it belongs to the compressed segment
+  auto in_a = [&](int j) -> bool { return LINF && j < nA; };
+  auto pages_of = [&](int j) -> int { return in_a(j) ? min(2, lf_pages - 2 * j) : min(2, cnt - 2 * (j - nA)); };
 
   if (SPLIT) setup();
   const uint32_t tmem = bars->tmem_base;
@@ -309,13 +327,16 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         auto load_kv = [&](int j, bool is_k) -> bool {
           const int s = j % kStages;
           const uint32_t ph = (j / kStages) & 1;
-          const int npg = min(2, cnt - 2 * j);
+          const int npg = pages_of(j);
+          const bool seg_a = in_a(j);
           uint64_t* full = is_k ? &bars->k_full[s] : &bars->v_full[s];
           uint64_t* empty = is_k ? &bars->k_empty[s] : &bars->v_empty[s];
           uint8_t* dst = smem + (is_k ? L::kK : L::kV) + s * L::kTile;
-          const void* tm = is_k ? static_cast<const void*>(&tm_k) : static_cast<const void*>(&tm_v);
+          const void* tm = seg_a ? (is_k ? static_cast<const void*>(&tm_kc) : static_cast<const void*>(&tm_vc))
+                                 : (is_k ? static_cast<const void*>(&tm_k) : static_cast<const void*>(&tm_v));
           int32_t y[2] = {0, 0};
-          for (int pg = 0; pg < npg; ++pg) y[pg] = page_row(2 * j + pg);
+          for (int pg = 0; pg < npg; ++pg)
+            y[pg] = seg_a ? (p.lf_table[2 * j + pg] * p.H + h) * kBlock : page_row(2 * (j - nA) + pg);
           if (!wait_bar(empty, ph ^ 1, bars, p.status)) return false;
           mbar_expect_tx(full, npg * kBlock * D * 2);
           for (int pg = 0; pg < npg; ++pg)
@@ -328,13 +349,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           return true;
         };
         // K runs three steps ahead of V: the scores of step j+3 are issued right after P V of j
-        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = load_kv(j, true);
+        for (int j = 0; j < min(NSB, nsteps) && ok; ++j) ok = load_kv(j, true);
 #pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
           ok = load_kv(j, false);
-          if (ok && j + kSBufs < nsteps) ok = load_kv(j + kSBufs, true);
+          if (ok && j + NSB < nsteps) ok = load_kv(j + NSB, true);
         }
-        if (ok && p.do_linear) {
+        if (ok && p.do_linear && !LINF) {
           // hi and lo halves of the D x D state ride the V ring as two more "steps"
           for (int hl = 0; hl < 2 && ok; ++hl) {
             const int j = nsteps + hl;
@@ -391,8 +412,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (!wait_bar(&bars->k_full[s], (j / kStages) & 1, bars, p.status)) return false;
           tc_fence_after();
           const uint32_t k_lo = desc_lo_sw128(smem_u32(smem + L::kK + s * L::kTile), 16);
-          const uint32_t d_tmem = tmem + kColS + 128 * (j % kSBufs);
-          if (cnt - 2 * j >= 2) {
+          const uint32_t d_tmem = tmem + kColSb + 128 * (j % NSB);
+          if (pages_of(j) >= 2) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, 128, 0, 0);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
@@ -408,28 +429,28 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
           }
           tc_commit(&bars->k_empty[s]);
-          tc_commit(&bars->s_full[j % kSBufs]);
+          tc_commit(&bars->s_full[j % NSB]);
           return true;
         };
-        for (int j = 0; j < min(kSBufs, nsteps) && ok; ++j) ok = issue_qk(j);
+        for (int j = 0; j < min(NSB, nsteps) && ok; ++j) ok = issue_qk(j);
 #pragma unroll 1
         for (int j = 0; j < nsteps && ok; ++j) {
           const int s = j % kStages;
-          const int b = j % kSBufs;
-          ok = wait_bar(&bars->p_full[b], (j / kSBufs) & 1, bars, p.status);
+          const int b = j % NSB;
+          ok = wait_bar(&bars->p_full[b], (j / NSB) & 1, bars, p.status);
           if (!ok) break;
           ok = wait_bar(&bars->v_full[s], (j / kStages) & 1, bars, p.status);
           if (!ok) break;
           tc_fence_after();
           constexpr uint32_t idesc = idesc_bf16_f32(128, D, 0, 1);
           const uint32_t v_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
-          const uint32_t o_acc = tmem + kColO;
-          const uint32_t p_op = tmem + kColS + 128 * b;
-          const uint32_t acc0 = j > 0 ? 1u : 0u;
+          const uint32_t o_acc = tmem + (in_a(j) ? kColLn : kColO);  // each segment has its accumulator
+          const uint32_t p_op = tmem + kColSb + 128 * b;
+          const uint32_t acc0 = (j > 0 && !(LINF && j == nA)) ? 1u : 0u;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, kk > 0 ? 1u : acc0);
-          if (cnt - 2 * j >= 2) {
+          if (pages_of(j) >= 2) {
 #pragma unroll
             for (int kk = 4; kk < 8; ++kk)
               tc_mma_ts_lo(o_acc, p_op + kk * 8, v_lo + kk * 128, kHiSw, idesc, 1u);
@@ -438,10 +459,10 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           tc_commit(&bars->pv_done);
           // the scores of step j+3 overwrite the P just consumed: issued after the P V above,
           // the tensor pipe runs them in order
-          if (j + kSBufs < nsteps) ok = issue_qk(j + kSBufs);
+          if (j + NSB < nsteps) ok = issue_qk(j + NSB);
         }
         if (ok) tc_commit(&bars->o_done);
-        if (ok && p.do_linear) {
+        if (ok && p.do_linear && !LINF) {
           ok = wait_bar(&bars->lin_a_full, 0, bars, p.status);
           for (int hl = 0; hl < 2 && ok; ++hl) {
             const int j = nsteps + hl;
@@ -453,7 +474,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t b_lo = desc_lo_sw128(smem_u32(smem + L::kV + s * L::kTile), L::kHalf);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk)
-              tc_mma_ts_lo(tmem + kColLin, tmem + kColPhi + kk * 8, b_lo + kk * 128, kHiSw, idesc,
+              tc_mma_ts_lo(tmem + kColLn, tmem + kColPhi + kk * 8, b_lo + kk * 128, kHiSw, idesc,
                            (hl > 0 || kk > 0) ? 1u : 0u);
             tc_commit(&bars->v_empty[s]);
           }
@@ -486,6 +507,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       float t_ref = 0.f;
       float m_used = -INFINITY;
       float l = 0.f;
+      float l_a = 0.f;    // LINF: row sum of the compressed segment (l then counts the selected pages)
+      bool in_b = false;  // LINF: this thread has entered the second segment
+      const int64_t lf_tokens = static_cast<int64_t>(lf_pages) * kBlock;
       bool ok = true;
       const int first = safe ? (grp == 0 ? 0 : nsteps) : grp;
       const int stride = safe ? 1 : kGroups;
@@ -496,7 +520,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       const int cbase = (grp & 1) * HC;
       float den_part = 0.f, den_part2 = 0.f;
       uint32_t fr[HC / 2];
-      if (ok && p.do_linear && epi) {
+      if (ok && p.do_linear && epi && !LINF) {
         // phi(q) of this thread's row for its half of the dims (bf16 A operand of the linear
         // MMA) and the partial denominator phi(q) . z -- computed up front, while the first scores are on their way,
         // and kept in registers until the epilogue
@@ -524,42 +548,62 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
 
       // block ids of the next step are fetched one step ahead, off the critical path
+      // (compressed segment: its pages in order; selected pages: the list)
+      auto blocks_of = [&](int j, int& b0, int& b1) {
+        if (in_a(j)) {
+          b0 = 2 * j;
+          b1 = 2 * j + 1;
+        } else {
+          const int e = 2 * (j - nA);
+          b0 = sel[e];
+          b1 = (e + 1 < cnt) ? sel[e + 1] : 0;
+        }
+      };
       int nb0 = 0, nb1 = 0;
-      if (first < nsteps) {
-        nb0 = sel[2 * first];
-        nb1 = (2 * first + 1 < cnt) ? sel[2 * first + 1] : 0;
-      }
+      if (first < nsteps) blocks_of(first, nb0, nb1);
 #pragma unroll 1
       for (int j = first; j < nsteps; j += stride) {
         int blk0 = nb0, blk1 = nb1;
-        if (j + stride < nsteps) {
-          nb0 = sel[2 * (j + stride)];
-          nb1 = (2 * (j + stride) + 1 < cnt) ? sel[2 * (j + stride) + 1] : 0;
+        if (j + stride < nsteps) blocks_of(j + stride, nb0, nb1);
+        // segment of this step: the compressed rows are all visible and have their own reference
+        const bool seg_a = in_a(j);
+        if (LINF && !seg_a && !in_b) {
+          in_b = true;
+          l_a = l;
+          l = 0.f;
+          m_used = -INFINITY;
         }
-        const int b = j % kSBufs;
-        const uint32_t s_tmem = tmem + lane_off + kColS + 128 * b;
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], (j / kSBufs) & 1, bars, p.status));
+        const int jj = j - (seg_a ? 0 : nA);      // step inside its segment
+        const int seg = (LINF && !seg_a) ? 1 : 0;  // which reference array / barrier
+        const bool seg_first = jj == 0;
+        const int seg_blocks = seg_a ? lf_pages : p.n_blocks;
+        const int64_t seg_vis = seg_a ? lf_tokens : vis_end;
+        const int64_t seg_tile_vis = seg_a ? lf_tokens : tile_vis_end;
+        const uint32_t o_seg = seg_a ? tmem + lane_off + kColLn : o_tmem;
+        const int b = j % NSB;
+        const uint32_t s_tmem = tmem + lane_off + kColSb + 128 * b;
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[b], (j / NSB) & 1, bars, p.status));
         if (!ok) break;
         tc_fence_after();
         uint32_t cbuf[2][32];  // two 32-column chunks of the score row in flight
         // the first chunk is requested at once: its latency runs under the bookkeeping below
         // (the steps that look for the row maximum first issue their own loads)
-        const bool early_ld = !(safe || j == 0);
+        const bool early_ld = !(safe || seg_first);
         if (early_ld) tmem_ld32(s_tmem, cbuf[0]);
-        const int npg = min(2, cnt - 2 * j);
+        const int npg = pages_of(j);
         const int n = npg * kBlock;
-        if (blk0 < 0 || blk0 >= p.n_blocks) blk0 = 0;
-        if (blk1 < 0 || blk1 >= p.n_blocks) blk1 = 0;
+        if (blk0 < 0 || blk0 >= seg_blocks) blk0 = 0;
+        if (blk1 < 0 || blk1 >= seg_blocks) blk1 = 0;
         const int64_t last_blk = blk0 > blk1 ? blk0 : blk1;
-        const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > tile_vis_end);
+        const bool need_mask = (n != 128) || (last_blk * kBlock + kBlock > seg_tile_vis);
         // visible keys per page: columns [0, lim) of the page's 64
         int lim0 = kBlock, lim1 = kBlock;
         if (need_mask) {
-          lim0 = static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk0) * kBlock)));
-          lim1 = npg > 1 ? static_cast<int>(max64(0, min64(kBlock, vis_end - static_cast<int64_t>(blk1) * kBlock))) : 0;
+          lim0 = static_cast<int>(max64(0, min64(kBlock, seg_vis - static_cast<int64_t>(blk0) * kBlock)));
+          lim1 = npg > 1 ? static_cast<int>(max64(0, min64(kBlock, seg_vis - static_cast<int64_t>(blk1) * kBlock))) : 0;
         }
         const int nchunks = n / 32;
-        if (safe || j == 0) {
+        if (safe || seg_first) {
           // the reference needs the row maximum first: a pass over the score row in chunks
           float mxa = -INFINITY, mxb = -INFINITY;
           // (the fixed reference of the fast pass only has to be near the row maximum: an unmasked
@@ -589,8 +633,8 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           if (!safe) {
             // fix the row's reference for the whole tile and hand it to the other group
             t_ref = (m_new == -INFINITY) ? 0.f : fmaf(m_new, sl2, kHeadroom);
-            bars->mref[r] = t_ref;
-            mbar_arrive(&bars->mref_ready);
+            bars->mref[seg][r] = t_ref;
+            mbar_arrive(&bars->mref_ready[seg]);
           } else {
             // lazy rescale: move the reference only when it would grow by more than 2^8
             float factor = 1.f;
@@ -603,6 +647,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             }
             if (j > 0) {
               // O must be quiescent: the previous P V has to be complete before it is rescaled
+              // (at the first step of the second segment nothing is rescaled: factor is 1)
               ok = __all_sync(0xffffffffu, wait_bar(&bars->pv_done, (j - 1) & 1, bars, p.status));
               if (!ok) break;
               tc_fence_after();
@@ -610,22 +655,23 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll 1
                 for (int c0 = 0; c0 < D; c0 += 32) {
                   uint32_t o[32];
-                  tmem_ld32(o_tmem + c0, o);
+                  tmem_ld32(o_seg + c0, o);
                   tc_wait_ld();
 #pragma unroll
                   for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                  tmem_st32(o_tmem + c0, o);
+                  tmem_st32(o_seg + c0, o);
                 }
                 tc_wait_st();
               }
             }
             t_ref = (m_used == -INFINITY) ? 0.f : m_used * sl2;
           }
-        } else if (j < kGroups) {
-          // first step of group 1 in the fast pass: take the reference group 0 fixed
-          ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready, 0, bars, p.status));
+        } else if (jj < kGroups) {
+          // first step of the other group in this segment (fast pass): take the reference the
+          // segment's first step fixed
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->mref_ready[seg], 0, bars, p.status));
           if (!ok) break;
-          t_ref = bars->mref[r];
+          t_ref = bars->mref[seg][r];
         }
         // exponentials in four chunks of 32 columns: the load of the next chunk and the store of
         // the previous P chunk run under the arithmetic of the current one
@@ -708,7 +754,11 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         ok = __all_sync(0xffffffffu, wait_bar(&bars->o_done, 0, bars, p.status));
         tc_fence_after();
       }
-      if (ok && p.do_linear && epi) {
+      if (LINF && !in_b) {  // a thread that saw no step of the second segment
+        l_a = l;
+        l = 0.f;
+      }
+      if (ok && p.do_linear && epi && !LINF) {
         if constexpr (D == 128) {
           tmem_st32(tmem + lane_off + kColPhi + grp * 32, reinterpret_cast<uint32_t(&)[32]>(fr[0]));
         } else {
@@ -720,7 +770,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       // publish this group's partial row sum and denominator, then read the other group's
       stats[(grp * 128 + r) * 4 + 0] = l;
-      stats[(grp * 128 + r) * 4 + 1] = den_part;
+      stats[(grp * 128 + r) * 4 + 1] = LINF ? l_a : den_part;  // LINF: the denominator is the compressed segment's row sum
       named_bar_sync(1, 128 * kGroups);
       float lsum = 0.f, den = 0.f;
 #pragma unroll
@@ -728,8 +778,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         lsum += stats[(gg * 128 + r) * 4 + 0];
         den += stats[(gg * 128 + r) * 4 + 1];
       }
-      float inv_l = (nsteps > 0 && lsum > 0.f) ? 1.f / lsum : 0.f;
-      const bool has_o = nsteps > 0;
+      float inv_l = (nsteps > nA && lsum > 0.f) ? 1.f / lsum : 0.f;
+      const bool has_o = nsteps > nA;                       // the selected pages wrote an accumulator
+      const bool has_lin = LINF ? nA > 0 : p.do_linear != 0;  // the linear branch wrote one
       // Split tile: every part dumps its unnormalised accumulator with the row sums and the
       // exponent references, then takes a ticket; the part that draws the last ticket merges all of
       // them (its own included) in the epilogue below, the others write no output.  Only the attempt
@@ -789,13 +840,13 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           inv_l = ltot > 0.f ? 1.f / ltot : 0.f;
         }
       }
-      if (ok && p.do_linear && epi) {
+      if (ok && p.do_linear && epi && !LINF) {
         ok = __all_sync(0xffffffffu, wait_bar(&bars->lin_done, 0, bars, p.status));
         tc_fence_after();
       }
       // The output tile is staged in the Q tile's shared memory.  A tile with no step and no linear
       // branch has not looked at Q at all: its TMA load may still be in flight and must land first.
-      if (ok && epi && nsteps == 0 && !p.do_linear)
+      if (ok && epi && nsteps == 0 && (!p.do_linear || LINF))
         ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
       if (ok && epi && do_output) {  // warp-uniform: the TMEM loads below are warp-collective
         const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
@@ -820,14 +871,14 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                            !(SPLIT && nsplit > 1);
         if (plain) {
           // no gates, no causal partials, no external linear output, no merge: 32 columns per trip
-          const float il = has_o ? inv_l : 0.f, id = p.do_linear ? inv_den : 0.f;
+          const float il = has_o ? inv_l : 0.f, id = has_lin ? inv_den : 0.f;
 #pragma unroll 1
           for (int c0 = cbase; c0 < cbase + HC; c0 += 32) {
             uint32_t oa[32], ln[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) oa[i] = ln[i] = 0u;
             if (has_o) tmem_ld32(o_tmem + c0, oa);
-            if (p.do_linear) tmem_ld32(tmem + lane_off + kColLin + c0, ln);
+            if (has_lin) tmem_ld32(tmem + lane_off + kColLn + c0, ln);
             tc_wait_ld();
             uint32_t pk[16];
 #pragma unroll
@@ -872,7 +923,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           } else if (has_o) {
             tmem_ld16(o_tmem + c0, oa);
           }
-          if (p.do_linear) tmem_ld16(tmem + lane_off + kColLin + c0, ln);
+          if (has_lin) tmem_ld16(tmem + lane_off + kColLn + c0, ln);
           tc_wait_ld();
           uint32_t packed[8];
           {
@@ -923,7 +974,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               const float osp = has_o ? __uint_as_float(oa[i + e]) * inv_l : 0.f;
-              const float olin = p.do_linear ? (__uint_as_float(ln[i + e]) + ladd[i + e]) * inv_den
+              const float olin = has_lin ? (__uint_as_float(ln[i + e]) + ladd[i + e]) * inv_den
                                              : ladd[i + e];  // 0 unless an external linear output is given
               res[e] = fmaf(wl[i + e], olin, ws[i + e] * osp);
             }
@@ -966,27 +1017,32 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
 
 cudaError_t forward_init() {
-  cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128, false>,
+  cudaError_t e = cudaFuncSetAttribute(hsa_forward_kernel<128, false, false>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kTotal);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(hsa_forward_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(hsa_forward_kernel<128, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Smem<128>::kTotal);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(hsa_forward_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(hsa_forward_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Smem<128>::kTotal);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(hsa_forward_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Smem<64>::kTotal);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(hsa_forward_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(hsa_forward_kernel<64, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Smem<64>::kTotal);
   return e;
 }
 
 cudaError_t launch_forward(const FwdParams& p_in, int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                            const CUtensorMap& tm_v, const CUtensorMap& tm_state, const CUtensorMap& tm_out,
-                           cudaStream_t st) {
+                           cudaStream_t st, const CUtensorMap* tm_kc, const CUtensorMap* tm_vc) {
   const int n_tiles = (p_in.n_q + kTileM - 1) / kTileM;
   FwdParams p = p_in;
   p.n_tiles = n_tiles;
   const bool split = p.max_splits > 1;
+  const bool linf = p.lf_table != nullptr;
+  if (linf && (split || D != 128 || !tm_kc || !tm_vc)) return cudaErrorInvalidValue;
   // One list per head and few heads: the split kernel ranks the heads itself and walks a
   // one-dimensional grid longest lists first; its balance rule makes at most nsm + H * n_tiles parts.
   p.remap = split && p.n_groups == 1 && p.H <= 32;
@@ -1002,12 +1058,16 @@ cudaError_t launch_forward(const FwdParams& p_in, int D, const CUtensorMap& tm_q
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  // (kernels without the compressed segment never look at the last two maps)
+  const CUtensorMap& kc = linf ? *tm_kc : tm_k;
+  const CUtensorMap& vc = linf ? *tm_vc : tm_v;
   if (D == 128) {
-    if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, true>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
-    return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, false>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
+    if (linf) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, false, true>, tm_q, tm_k, tm_v, tm_state, tm_out, kc, vc, p);
+    if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, true, false>, tm_q, tm_k, tm_v, tm_state, tm_out, kc, vc, p);
+    return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<128, false, false>, tm_q, tm_k, tm_v, tm_state, tm_out, kc, vc, p);
   }
-  if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, true>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
-  return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, false>, tm_q, tm_k, tm_v, tm_state, tm_out, p);
+  if (split) return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, true, false>, tm_q, tm_k, tm_v, tm_state, tm_out, kc, vc, p);
+  return cudaLaunchKernelEx(&cfg, hsa_forward_kernel<64, false, false>, tm_q, tm_k, tm_v, tm_state, tm_out, kc, vc, p);
 }
 
 }  // namespace hsa

@@ -611,9 +611,19 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     p.lin_num = c.lin_num;
     p.lin_den = c.lin_den;
   }
+  if (do_linformer && p.max_splits == 1 && D == 128) {
+    // one launch: the kernel's loop runs over the compressed pool first (its own accumulator,
+    // exponent reference and row sums), then over the selected pages, and merges in its epilogue
+    p.lf_table = reinterpret_cast<const int32_t*>(ws + ctx->lay.ctable);
+    p.lf_pages = static_cast<int>(static_cast<int64_t>(ctx->n_segs) * ctx->cfg.lin_rank / kBlock);
+    p.do_linear = 1;  // the compressed segment is this launch's linear branch
+    cudaError_t ef = launch_forward(p, D, tm_q, ctx->tm_k, ctx->tm_v, ctx->tm_state, tm_out, st, &ctx->tm_kc, &ctx->tm_vc);
+    if (ef != cudaSuccess) return cuda_fail(ctx, ef);
+    return HSA_OK;
+  }
   if (do_linformer) {
-    // pass 1: plain softmax attention of the chunk over every compressed row -> O_lin (bf16) in the
-    // workspace; pass 2 below picks it up in its epilogue
+    // long lists split over CTAs: two launches.  Pass 1: plain softmax attention of the chunk over
+    // every compressed row -> O_lin (bf16) in the workspace; pass 2 below picks it up in its epilogue
     uint8_t* olin = ws + ctx->lay.olin;
     CUtensorMap tm_olin;
     r = encode_q(&tm_olin, olin, n_q, H, D, static_cast<int64_t>(H) * D, D);

@@ -123,6 +123,10 @@ struct FwdParams {
   const float* lin_num;  // causal intra-chunk partials [n_q][H][D] (or null)
   const float* lin_den;  // [n_q][H]
   const __nv_bfloat16* ext_lin;  // linear-branch output computed elsewhere, [n_q][H][D] (or null)
+  // Linformer form inside the kernel: the loop first runs over the lf_pages pages of the compressed
+  // pool (page ids through lf_table), with an accumulator and row sums of their own (null: none)
+  const int32_t* lf_table;
+  int lf_pages;
   // split tiles: a (tile, head) with more than split_blocks selected blocks runs as several CTAs
   // (grid z = max_splits); each dumps its unnormalised O, row sums and exponent references, the last
   // one to take a ticket merges them and writes the output
@@ -188,9 +192,11 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
 cudaError_t launch_qsum(const SelectArgs& a, cudaStream_t st);  // stage 1 alone: query tile sums
 cudaError_t launch_retrieve(const RetrieveArgs& a, int n_pages, cudaStream_t st);
 cudaError_t launch_select_adaptive(const SelectArgs& a, const AdaptiveArgs& ad, cudaStream_t st);
+// tm_kc / tm_vc: maps of the compressed pools, used when p.lf_table is set (else null)
 cudaError_t launch_forward(const FwdParams& p, int D, const CUtensorMap& tm_q,
                            const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                           const CUtensorMap& tm_state, const CUtensorMap& tm_out, cudaStream_t st);
+                           const CUtensorMap& tm_state, const CUtensorMap& tm_out, cudaStream_t st,
+                           const CUtensorMap* tm_kc = nullptr, const CUtensorMap* tm_vc = nullptr);
 cudaError_t launch_causal_linear(const CausalLinArgs& a, cudaStream_t st);
 // linear branch alone (head_dim 128): lean HBM-bound kernel, nsm = SMs of the device
 cudaError_t launch_linear_only(const FwdParams& p, int nsm, const CUtensorMap& tm_q, const CUtensorMap& tm_state,

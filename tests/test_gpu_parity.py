@@ -500,6 +500,69 @@ def test_linformer_linear_branch(cuda_device):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("n_segs,k_scale,split_blocks,gates", [
+    (1, None, 0, None),          # one compressed step: both softmax groups start in different segments
+    (2, None, 0, "head"),        # gated merge of the two segments' results
+    (4, (0.05, 12.0), 0, None),  # later segments / blocks dominate: both segments overflow the fixed reference
+    (4, None, 4, None),          # long lists split over CTAs: the two-launch form
+])
+def test_linformer_segments_inside_the_forward_kernel(n_segs, k_scale, split_blocks, gates, cuda_device):
+    """The Linformer form runs as one launch whose loop walks the compressed pool first and the
+    selected pages second, each with its own accumulator, exponent reference and row sums.  Cases:
+    a single compressed step, gates, a history whose later parts outweigh the first step by far more
+    than the fixed reference allows (the tile is redone with running maxima in both segments), and
+    the split-list configuration, which keeps the form with two launches."""
+    from paper_2609_34606_b200 import hsa
+    base = W.WORKLOADS["mid_linformer"]
+    w = W.Workload("linf_case", H=base.H, d=128, Lq=300, chunk=base.chunk, n_chunks=n_segs, topk=6, seed=90 + n_segs)
+    rank, seg = 128, w.chunk
+    ek, ev = W.gen_linformer_weights(w, rank, seg)
+    ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk), max_topk=w.n_blocks,
+                         lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=rank, lin_seg_tokens=seg,
+                         e_k=ek.to(cuda_device), e_v=ev.to(cuda_device), device=cuda_device,
+                         split_blocks=split_blocks)
+    for pool in (ctx.k_pool, ctx.v_pool, ctx.kc_pool, ctx.vc_pool):
+        pool.fill_(0xFF)
+    K, V = W.gen_history(w)
+    if k_scale is not None:
+        K = K.float()
+        K[:seg] *= k_scale[0]     # the first segment (and the first blocks) barely score
+        K[seg:] *= k_scale[1]     # everything later scores far higher
+        K = K.to(torch.bfloat16)
+    for c in range(n_segs):
+        ctx.append_kv(K[c * seg:(c + 1) * seg].to(cuda_device), V[c * seg:(c + 1) * seg].to(cuda_device))
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    allsel = [[np.arange(w.n_blocks, dtype=np.int32)] for _ in range(w.H)]
+    si, sc = Hn.selection_to_device(allsel, ctx.max_topk, cuda_device)
+    g_lin = g_sp = None
+    wl = ws = 1.0
+    if gates:
+        g_lin, g_sp = W.gen_gates(w, per_dim=False)
+        wl, ws = Hn.f64(g_lin)[..., None], Hn.f64(g_sp)[..., None]
+        g_lin, g_sp = g_lin.to(cuda_device), g_sp.to(cuda_device)
+    Kt, Vt = O.linformer_compress(Kn, Vn, Hn.f32(ek), Hn.f32(ev), seg)
+    if k_scale is not None:
+        # logits of a few hundred: the bf16 rounding of the stored compressed rows (0.4 % of a logit)
+        # is no longer small against 1, so this case takes the rows as the pool holds them
+        Kt = Hn.f64(torch.from_numpy(Kt).to(torch.bfloat16))
+        Vt = Hn.f64(torch.from_numpy(Vt).to(torch.bfloat16))
+    o_lin_ref = O.linformer_branch(qn, Kt, Vt)
+    o_sp_ref = O.dense_attention(qn, Kn, Vn, w.N, False)   # every block selected
+    assert ctx.safe_pass_tiles() == 0
+    out = Hn.f64(ctx.forward(qd, si, sc, g_lin=g_lin, g_sp=g_sp))
+    o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
+    assert ctx.device_status() == 0
+    redone = ctx.safe_pass_tiles()
+    assert (redone > 0) == (k_scale is not None)
+    tol = dict(rel_fro=1e-2, max_abs=4e-2 if k_scale is not None else 2e-2)
+    for got, ref, what in ((o_lin, o_lin_ref, "O_lin"), (out, wl * o_lin_ref + ws * o_sp_ref, "out")):
+        e = Hn.err_stats(got, ref)
+        assert e["rel_fro"] <= tol["rel_fro"] and e["max_abs"] <= tol["max_abs"], (what, e)
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("name,group_tokens", [("mid_mix", 0), ("mid_d128", 0), ("mid_d128", 128), ("cfg1_sharp", 0)])
 def test_head_adaptive_selection(name, group_tokens, cuda_device):
     """Cumulative-mass selection with the Gini threshold map (tau_max = 1.00, tau_min = 0.35, the
