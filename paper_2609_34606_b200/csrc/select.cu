@@ -225,8 +225,9 @@ __device__ __forceinline__ void scores_item(const Blk& blk, const SelectArgs& a,
       for (int w = 0; w < WAYS; ++w) t += part[w * D + blk.tid];
       qs[blk.tid] = t / static_cast<double>(q_hi - q_lo) * static_cast<double>(a.scale);
     }
+    blk_sync(blk);  // (a mean query that was not rebuilt here is complete already: no barrier, the
+                    // warps walk through their candidates independently)
   }
-  blk_sync(blk);
   constexpr int PER = D / 32;
   uint32_t* keys = a.keys + (static_cast<size_t>(h) * a.n_groups + g) * a.max_pages;
   const CandGeom cg = cand_geom<MIXED>(a);
@@ -760,10 +761,8 @@ __global__ void __launch_bounds__(256 * kSubBlocks, 1) select_cluster_kernel(Sel
   uint32_t keys_addr;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(keys_addr) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(cl_keys))), "r"(0u));
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // every CTA of the cluster is running
-  for (int chunk = slot; chunk < n_chunks; chunk += n_slots) {
+  for (int chunk = slot; chunk < n_chunks; chunk += n_slots)
     scores_item<D, MIXED>(blk, a, chunk, 0, h, qmean, op, false, chunk == slot, keys_addr);
-    blk_sync(blk);
-  }
   cluster_sync_all();  // the score keys of the head are complete and visible to its first CTA
   // the kernel behind this one may take the places of the CTAs that leave now
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
