@@ -563,6 +563,35 @@ def test_linformer_segments_inside_the_forward_kernel(n_segs, k_scale, split_blo
     ctx.destroy()
 
 
+def test_linformer_form_with_one_selection_per_query_tile(cuda_device):
+    """The compressed segment in front of per-tile lists: every query tile walks the same compressed
+    pool, then its own selection."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["mid_linformer"]
+    rank, seg, gtok = 128, w.chunk, 128
+    ek, ev = W.gen_linformer_weights(w, rank, seg)
+    ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk), max_topk=w.n_blocks,
+                         lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=rank, lin_seg_tokens=seg,
+                         e_k=ek.to(cuda_device), e_v=ev.to(cuda_device), device=cuda_device)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w)
+    qd = q.to(cuda_device)
+    budgets = W.gen_budgets(w)
+    qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
+    si, sc = ctx.select_blocks(qd, budgets.to(cuda_device), group_tokens=gtok)
+    sel_gpu = Hn.selection_lists(si, sc)
+    sel_ref, scores = O.select_blocks(qn, Kn, w.N, False, budgets.tolist(), gtok)
+    Hn.check_selection(sel_gpu, sel_ref, scores)
+    assert len(sel_gpu[0]) == (w.Lq + gtok - 1) // gtok and any(
+        list(sel_gpu[0][0]) != list(sel_gpu[0][g]) for g in range(1, len(sel_gpu[0]))), "the tiles' lists should differ"
+    Kt, Vt = O.linformer_compress(Kn, Vn, Hn.f32(ek), Hn.f32(ev), seg)
+    ref = O.linformer_branch(qn, Kt, Vt) + O.sparse_branch(qn, Kn, Vn, sel_gpu, w.N, False, gtok)
+    out = Hn.f64(ctx.forward(qd, si, sc, group_tokens=gtok))
+    assert ctx.device_status() == 0
+    Hn.assert_close(out, ref, "out")
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("name,group_tokens", [("mid_mix", 0), ("mid_d128", 0), ("mid_d128", 128), ("cfg1_sharp", 0)])
 def test_head_adaptive_selection(name, group_tokens, cuda_device):
     """Cumulative-mass selection with the Gini threshold map (tau_max = 1.00, tau_min = 0.35, the
