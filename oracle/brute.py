@@ -70,18 +70,21 @@ def topk_blocks(scores, cand, budget):
     return sorted(idx[:budget])
 
 
-def _phi(x):
+def _phi(x, relu=False):
     x = float(x)
+    if relu:
+        return x if x > 0 else 0.0
     return x + 1.0 if x > 0 else math.exp(x)
 
 
-def linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal):
-    """sum_j phi(q).phi(k_j) v_j / sum_j phi(q).phi(k_j) over visible j."""
+def linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal, relu=False):
+    """sum_j phi(q).phi(k_j) v_j / sum_j phi(q).phi(k_j) over visible j (relu: the sum of weights
+    plus 1e-6 in the denominator)."""
     out = [[[0.0] * d for _ in range(H)] for _ in range(Lq)]
     for h in range(H):
-        fk = [[_phi(K[j][h][c]) for c in range(d)] for j in range(N)]
+        fk = [[_phi(K[j][h][c], relu) for c in range(d)] for j in range(N)]
         for i in range(Lq):
-            fq = [_phi(q[i][h][c]) for c in range(d)]
+            fq = [_phi(q[i][h][c], relu) for c in range(d)]
             p = q_pos0 + i
             num = [0.0] * d
             den = 0.0
@@ -92,6 +95,8 @@ def linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal):
                 den += w
                 for c in range(d):
                     num[c] += w * float(V[j][h][c])
-            if den > 0:
+            if relu:
+                out[i][h] = [x / (den + 1e-6) for x in num]
+            elif den > 0:
                 out[i][h] = [x / den for x in num]
     return out

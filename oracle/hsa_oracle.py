@@ -327,14 +327,31 @@ def sparse_branch(q, K, V, sel, q_pos0: int, causal: bool, group_tokens: int = 0
 #   O_lin[i] = sum_{j vis} (phi(q_i).phi(k_j)) v_j / sum_{j vis} phi(q_i).phi(k_j)
 # This is the "fixed-size hidden state" linear attention the Linear Branch
 # appendix contrasts with Linformer; it is the form the measured path uses.
-# phi is not given by the paper: phi(x) = elu(x) + 1.   (parity unpinned)
+# phi is not given by the paper: phi(x) = elu(x) + 1 ("elu1", the default), or
+# phi(x) = max(x, 0) ("relu").  With relu a query can have weight zero on every
+# visible key, so that form divides by (sum of weights + 1e-6): a row without
+# any weight is 0 / 1e-6 = 0.   (parity unpinned)
 # --------------------------------------------------------------------------
-def phi(x):
+RELU_EPS = 1e-6
+
+
+def phi(x, fmap: str = "elu1"):
     x = _f64(x)
+    if fmap == "relu":
+        return np.maximum(x, 0.0)
+    if fmap != "elu1":
+        raise ValueError("fmap must be 'elu1' or 'relu'")
     return np.where(x > 0, x + 1.0, np.exp(np.minimum(x, 0.0)))
 
 
-def linear_parallel(q, K, V, q_pos0: int, causal: bool, rows=None):
+def _normalise(num, den, fmap: str):
+    """num / den per row; elu1: rows without a visible key (den = 0) are 0; relu: num / (den + eps)."""
+    if fmap == "relu":
+        return num / (den + RELU_EPS)
+    return np.divide(num, den, out=np.zeros_like(num), where=den > 0)
+
+
+def linear_parallel(q, K, V, q_pos0: int, causal: bool, rows=None, fmap: str = "elu1"):
     """The definition written out: explicit [rows x N] weight matrix,
     masked, row-normalised."""
     Lq, H, d = q.shape
@@ -343,33 +360,33 @@ def linear_parallel(q, K, V, q_pos0: int, causal: bool, rows=None):
     r_all = np.arange(Lq) if rows is None else np.asarray(rows)
     step = max(1, int(2.5e7 // max(1, N)))
     for h in range(H):
-        fk = phi(K[:, h, :])
+        fk = phi(K[:, h, :], fmap)
         for c0 in range(0, r_all.size, step):
             rr = r_all[c0:c0 + step]
-            W = phi(q[rr, h, :]) @ fk.T                       # [rows, N], all > 0
+            W = phi(q[rr, h, :], fmap) @ fk.T                 # [rows, N], all >= 0
             if causal:
                 vis = np.arange(N)[None, :] <= (q_pos0 + rr)[:, None]
                 W = np.where(vis, W, 0.0)
             den = W.sum(axis=1, keepdims=True)
             num = W @ _f64(V[:, h, :])
-            out[rr, h, :] = np.divide(num, den, out=np.zeros_like(num), where=den > 0)
+            out[rr, h, :] = _normalise(num, den, fmap)
     return out
 
 
-def linear_state(K, V, upto: int | None = None):
+def linear_state(K, V, upto: int | None = None, fmap: str = "elu1"):
     """S[h] = sum_j phi(k_j)^T v_j  (d x d),  z[h] = sum_j phi(k_j), over tokens j < upto."""
     N, H, d = K.shape
     n = N if upto is None else max(0, min(N, upto))
     S = np.zeros((H, d, d))
     z = np.zeros((H, d))
     for h in range(H):
-        fk = phi(K[:n, h, :])
+        fk = phi(K[:n, h, :], fmap)
         S[h] = fk.T @ _f64(V[:n, h, :])
         z[h] = fk.sum(axis=0)
     return S, z
 
 
-def linear_recurrent(q, K, V, q_pos0: int, causal: bool):
+def linear_recurrent(q, K, V, q_pos0: int, causal: bool, fmap: str = "elu1"):
     """Token-by-token recurrence S_t = S_{t-1} + phi(k_t)^T v_t, z_t likewise.
     Query i reads the state after token min(p_i, N-1) if causal, else after the
     last token."""
@@ -381,33 +398,33 @@ def linear_recurrent(q, K, V, q_pos0: int, causal: bool):
     for h in range(H):
         S = np.zeros((d, d))
         z = np.zeros(d)
-        fq = phi(q[:, h, :])
+        fq = phi(q[:, h, :], fmap)
         order = np.argsort(need, kind="stable")
         t = 0
         for i in order:
             while t < need[i]:
-                fk = phi(K[t, h, :])
+                fk = phi(K[t, h, :], fmap)
                 S += np.outer(fk, _f64(V[t, h, :]))
                 z += fk
                 t += 1
             den = fq[i] @ z
             if need[i] > 0:
-                out[i, h, :] = (fq[i] @ S) / den
+                out[i, h, :] = (fq[i] @ S) / (den + RELU_EPS if fmap == "relu" else den)
     return out
 
 
-def linear_chunked(q, K, V, q_pos0: int, causal: bool, boundary: int):
+def linear_chunked(q, K, V, q_pos0: int, causal: bool, boundary: int, fmap: str = "elu1"):
     """State of the tokens before `boundary` plus the explicitly masked part over
     tokens >= boundary: the split the GPU uses (state at a chunk boundary +
     intra-chunk part)."""
     Lq, H, d = q.shape
     N = K.shape[0]
-    S0, z0 = linear_state(K, V, upto=boundary)
+    S0, z0 = linear_state(K, V, upto=boundary, fmap=fmap)
     out = np.zeros((Lq, H, d))
     p = q_pos0 + np.arange(Lq)
     jj = np.arange(boundary, N)
     for h in range(H):
-        fq = phi(q[:, h, :])
+        fq = phi(q[:, h, :], fmap)
         num = np.zeros((Lq, d))
         den = np.zeros(Lq)
         # the boundary state holds tokens < boundary; a causal query before the
@@ -417,25 +434,24 @@ def linear_chunked(q, K, V, q_pos0: int, causal: bool, boundary: int):
         num += fq @ S0[h]
         den += fq @ z0[h]
         if jj.size:
-            W = fq @ phi(K[boundary:, h, :]).T
+            W = fq @ phi(K[boundary:, h, :], fmap).T
             if causal:
                 W = np.where(jj[None, :] <= p[:, None], W, 0.0)
             num += W @ _f64(V[boundary:, h, :])
             den += W.sum(axis=1)
-        out[:, h, :] = np.divide(num, den[:, None], out=np.zeros_like(num),
-                                 where=den[:, None] > 0)
+        out[:, h, :] = _normalise(num, den[:, None], fmap)
     return out
 
 
-def linear_from_state(q, S, z):
+def linear_from_state(q, S, z, fmap: str = "elu1"):
     """phi(q) S / (phi(q) z): applying a given state to the chunk's queries."""
     Lq, H, d = q.shape
     out = np.zeros((Lq, H, d))
     for h in range(H):
-        fq = phi(q[:, h, :])
+        fq = phi(q[:, h, :], fmap)
         den = (fq @ z[h])[:, None]
         num = fq @ S[h]
-        out[:, h, :] = np.divide(num, den, out=np.zeros_like(num), where=den > 0)
+        out[:, h, :] = _normalise(num, den, fmap)
     return out
 
 
@@ -489,7 +505,7 @@ def merge(O_lin, O_sp, g_lin=None, g_sp=None, gate_act: int = 0):
 def hsa_forward(q, K, V, q_pos0: int, causal: bool, sel, group_tokens: int = 0,
                 g_lin=None, g_sp=None, gate_act: int = 0, scale: float | None = None,
                 no_linear: bool = False, no_sparse: bool = False, rows=None,
-                linear_form: str = "parallel"):
+                linear_form: str = "parallel", fmap: str = "elu1"):
     """out = gate(g_lin) * O_lin + gate(g_sp) * O_sp with a disabled branch
     contributing exactly 0.  linear_form: "parallel" (definition) or "state"
     (phi(q) S / phi(q) z, non-causal only; equal up to rounding order and used
@@ -501,10 +517,10 @@ def hsa_forward(q, K, V, q_pos0: int, causal: bool, sel, group_tokens: int = 0,
         O_sp = sparse_branch(q, K, V, sel, q_pos0, causal, group_tokens, scale, rows)
     if not no_linear:
         if linear_form == "state" and not causal:
-            S, z = linear_state(K, V)
-            O_lin = linear_from_state(q, S, z)
+            S, z = linear_state(K, V, fmap=fmap)
+            O_lin = linear_from_state(q, S, z, fmap)
         else:
-            O_lin = linear_parallel(q, K, V, q_pos0, causal, rows)
+            O_lin = linear_parallel(q, K, V, q_pos0, causal, rows, fmap)
         if rows is not None:
             keep = np.zeros(Lq, bool)
             keep[np.asarray(rows)] = True

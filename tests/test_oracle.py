@@ -116,6 +116,72 @@ def test_phi_is_elu_plus_one():
     assert (O.phi(x) > 0).all()
 
 
+# ---------------------------------------------------------------- the relu feature map
+def test_relu_feature_map_is_torch_relu():
+    x = np.array([-30.0, -1.0, -1e-9, 0.0, 1e-9, 2.5])
+    assert np.array_equal(O.phi(x, "relu"), torch.relu(torch.from_numpy(x)).numpy())
+    with pytest.raises(ValueError):
+        O.phi(x, "gelu")
+
+
+@pytest.mark.parametrize("causal,q_pos0", [(False, 300), (True, 300 - 37), (True, 5)])
+def test_relu_recurrent_equals_parallel_equals_chunked(causal, q_pos0):
+    """The algebraic identities of the running-state form hold for any feature map."""
+    H, d, Lq, N = 2, 16, 37, 300
+    q, K, V = rnd((Lq, H, d), 7), rnd((N, H, d), 8), rnd((N, H, d), 9)
+    a = O.linear_parallel(q, K, V, q_pos0, causal, fmap="relu")
+    b = O.linear_recurrent(q, K, V, q_pos0, causal, fmap="relu")
+    assert np.abs(a - b).max() <= 1e-10 * max(1.0, np.abs(a).max())
+    if q_pos0 >= N - Lq - 1:
+        c = O.linear_chunked(q, K, V, q_pos0, causal, boundary=N - Lq, fmap="relu")
+        assert np.abs(a - c).max() <= 1e-10
+    if not causal:
+        S, z = O.linear_state(K, V, fmap="relu")
+        assert np.abs(a - O.linear_from_state(q, S, z, "relu")).max() <= 1e-10
+    # and the map matters: the two forms differ on the same inputs
+    assert np.abs(a - O.linear_parallel(q, K, V, q_pos0, causal)).max() > 1e-3
+
+
+def test_relu_brute_force_and_closed_forms():
+    H, d, Lq, N = 2, 4, 6, 70
+    q, K, V = rnd((Lq, H, d), 13), rnd((N, H, d), 14), rnd((N, H, d), 15)
+    for causal, q_pos0 in [(False, N), (True, N - Lq), (True, 3)]:
+        a = O.linear_parallel(q, K, V, q_pos0, causal, fmap="relu")
+        b = np.array(brute.linear_rows(q, K, V, N, H, d, Lq, q_pos0, causal, relu=True))
+        assert np.abs(a - b).max() < 1e-12
+    # keys without a positive component carry no weight: the state is zero and the branch is 0 / eps = 0
+    Kn = -np.abs(K)
+    S, z = O.linear_state(Kn, V, fmap="relu")
+    assert not S.any() and not z.any()
+    assert not O.linear_parallel(q, Kn, V, N, False, fmap="relu").any()
+    # one key e_0, queries with a positive first component w: weight w, so O_lin = w v / (w + eps)
+    K1 = np.zeros((1, H, d)); K1[0, :, 0] = 1.0
+    q1 = np.abs(q) + 0.5
+    out = O.linear_parallel(q1, K1, V[:1], 1, False, fmap="relu")
+    w = q1[:, :, :1]
+    assert np.allclose(out, w * V[0][None] / (w + O.RELU_EPS), atol=1e-14)
+    # V = 1 everywhere: every row with weight returns 1 up to eps / (den + eps)
+    ones = np.ones_like(V)
+    o1 = O.linear_parallel(q, np.abs(K) + 0.1, ones, N, False, fmap="relu")
+    den = (O.phi(q, "relu").reshape(Lq, H, 1, d) * (np.abs(K) + 0.1).transpose(1, 0, 2)[None]).sum(axis=(2, 3))
+    has = den > 0
+    assert np.allclose(o1[has], (den / (den + O.RELU_EPS))[has][:, None] * np.ones(d), atol=1e-14)
+    assert not o1[~has].any()
+
+
+def test_forward_with_relu_uses_it_in_the_linear_branch_only():
+    H, d, Lq, N = 2, 8, 16, 192
+    q, K, V = rnd((Lq, H, d), 31), rnd((N, H, d), 32), rnd((N, H, d), 33)
+    sel = O.select_blocks(q, K, N, False, [2] * H)[0]
+    a = O.hsa_forward(q, K, V, N, False, sel, fmap="relu")
+    b = O.hsa_forward(q, K, V, N, False, sel)
+    assert np.array_equal(a["O_sp"], b["O_sp"])
+    assert np.allclose(a["O_lin"], O.linear_parallel(q, K, V, N, False, fmap="relu"), atol=0)
+    assert np.allclose(a["out"], a["O_lin"] + a["O_sp"], atol=1e-15)
+    s = O.hsa_forward(q, K, V, N, False, sel, fmap="relu", linear_form="state")
+    assert np.abs(s["O_lin"] - a["O_lin"]).max() <= 1e-10
+
+
 def test_single_token_history():
     H, d, Lq = 2, 8, 5
     q, K, V = rnd((Lq, H, d), 16), rnd((1, H, d), 17), rnd((1, H, d), 18)
