@@ -54,10 +54,16 @@ typedef enum {
 
 /* lin_mode */
 #define HSA_LIN_NONE 0
-#define HSA_LIN_STATE 1      /* running state S = sum phi(k)^T v, z = sum phi(k); phi = elu + 1 */
+#define HSA_LIN_STATE 1      /* running state S = sum phi(k)^T v, z = sum phi(k); phi: feature_map */
 #define HSA_LIN_LINFORMER 2  /* Section 3.3 "Linear branch" (Eq. 3) and Appendix G: per segment of
                                 lin_seg_tokens tokens K~ = E_K^T K, V~ = E_V^T V (lin_rank rows each),
                                 concatenated; O_lin = Softmax(Q K~^T / sqrt(d)) V~.  head_dim 128 only */
+
+/* feature_map of the running-state linear branch (the paper defines none for this form):
+ * phi(x) = elu(x) + 1, the default, or phi(x) = max(x, 0).  With relu a query can have weight zero
+ * on every key, so that form divides by (phi(q) . z + 1e-6). */
+#define HSA_PHI_ELU1 0
+#define HSA_PHI_RELU 1
 
 /* hsa_config.flags: reserve workspace for causal forwards with the linear branch on */
 #define HSA_CFG_CAUSAL 1u
@@ -91,6 +97,7 @@ typedef struct {
   int32_t split_blocks;   /* a (query tile, head) with more selected blocks than this is split over
                              several CTAs whose partial results the last one to finish merges
                              (0 -> 256; only matters when max_topk exceeds it)                     */
+  int32_t feature_map;    /* HSA_LIN_STATE: HSA_PHI_ELU1 (0) or HSA_PHI_RELU                           */
 } hsa_config;
 
 typedef struct {

@@ -118,8 +118,8 @@ __global__ void __launch_bounds__(256) state_partial_kernel(AppendArgs a) {
         for (int i = 0; i < 4; ++i) {
           const float2 f = __bfloat1622float2(k2[i]);
           const float2 g = __bfloat1622float2(v2[i]);
-          kf[2 * i] = phi_elu1(f.x);
-          kf[2 * i + 1] = phi_elu1(f.y);
+          kf[2 * i] = a.relu ? fmaxf(f.x, 0.f) : phi_elu1(f.x);
+          kf[2 * i + 1] = a.relu ? fmaxf(f.y, 0.f) : phi_elu1(f.y);
           vf[2 * i] = g.x;
           vf[2 * i + 1] = g.y;
         }
@@ -285,6 +285,9 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, const void* smem_
 
 }  // namespace
 
+// RELU: the feature map is max(x, 0) instead of elu(x) + 1 (an instance of its own: the map sits in
+// the innermost loop of the worker warps)
+template <bool RELU>
 __global__ void __launch_bounds__(kAfThreads, 1)
 append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CUtensorMap tm_kin,
                     const __grid_constant__ CUtensorMap tm_vin, const __grid_constant__ CUtensorMap tm_kpool,
@@ -494,8 +497,9 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
         uint32_t hw[4], lw[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float p0 = phi_fast(__uint_as_float(kw[e] << 16));
-          const float p1 = phi_fast(__uint_as_float(kw[e] & 0xffff0000u));
+          const float x0 = __uint_as_float(kw[e] << 16), x1 = __uint_as_float(kw[e] & 0xffff0000u);
+          const float p0 = RELU ? fmaxf(x0, 0.f) : phi_fast(x0);
+          const float p1 = RELU ? fmaxf(x1, 0.f) : phi_fast(x1);
           hw[e] = pack_bf16(p0, p1);
           lw[e] = pack_bf16(p0 - __uint_as_float(hw[e] << 16), p1 - __uint_as_float(hw[e] & 0xffff0000u));
         }
@@ -563,7 +567,10 @@ append_fused_kernel(AppendArgs a, int blocks_per_cta, const __grid_constant__ CU
 }
 
 cudaError_t append_init() {
-  return cudaFuncSetAttribute(append_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);
+  cudaError_t e = cudaFuncSetAttribute(append_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(append_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAfSmem);
+  return e;
 }
 
 cudaError_t launch_append(const AppendArgs& a_in, const AppendMaps* maps, cudaStream_t st) {
@@ -586,7 +593,10 @@ cudaError_t launch_append(const AppendArgs& a_in, const AppendMaps* maps, cudaSt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, append_fused_kernel, a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
+    if (a.relu)
+      e = cudaLaunchKernelEx(&cfg, append_fused_kernel<true>, a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
+    else
+      e = cudaLaunchKernelEx(&cfg, append_fused_kernel<false>, a, per, maps->kin, maps->vin, maps->kpool, maps->vpool);
     if (e != cudaSuccess) return e;
   } else {
     dim3 gridA(static_cast<unsigned>(b1 - b0 + 1), a.H);

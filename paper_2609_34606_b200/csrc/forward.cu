@@ -120,9 +120,9 @@ __device__ __forceinline__ float ex2v(float x) {
   asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// phi(x) = elu(x) + 1 = max(x, 0) + exp(min(x, 0))
-__device__ __forceinline__ float phi_elu1(float x) {
-  return fmaxf(x, 0.f) + ex2(fminf(x, 0.f) * 1.4426950408889634f);
+// either feature map without a branch: max(x, 0) + w * exp(min(x, 0)) with w = 1 (elu + 1) or 0 (relu)
+__device__ __forceinline__ float phi_q(float x, float w) {
+  return fmaf(w, ex2(fminf(x, 0.f) * 1.4426950408889634f), fmaxf(x, 0.f));
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float m;
@@ -526,6 +526,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         // and kept in registers until the epilogue
         ok = __all_sync(0xffffffffu, wait_bar(&bars->q_full, 0, bars, p.status));
         const uint8_t* qrow = smem + L::kQ + r * 128;
+        const float exp_part = p.relu ? 0.f : 1.f;  // relu drops the exponential part of the map
         const float4* z4 = reinterpret_cast<const float4*>(p.z + static_cast<size_t>(h) * D + cbase);
 #pragma unroll
         for (int c16 = 0; c16 < HC / 8; ++c16) {
@@ -537,7 +538,7 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const uint32_t pk = pack_bf16(phi_elu1(__uint_as_float(qw[i] << 16)), phi_elu1(__uint_as_float(qw[i] & 0xffff0000u)));
+            const uint32_t pk = pack_bf16(phi_q(__uint_as_float(qw[i] << 16), exp_part), phi_q(__uint_as_float(qw[i] & 0xffff0000u), exp_part));
             fr[c16 * 4 + i] = pk;
             // the denominator uses the rounded values the MMA will see
             den_part = fmaf(__uint_as_float(pk << 16), z[2 * i], den_part);
@@ -856,7 +857,9 @@ hsa_forward_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D;
           lin_den += p.lin_den[static_cast<size_t>(row) * p.H + h];
         }
-        const float inv_den = (p.do_linear && lin_den > 0.f) ? 1.f / lin_den : 0.f;
+        // (relu: a row may have no weight at all, hence 1e-6 in its denominator; 0 / 1e-6 = 0)
+        const float den_eps = lin_den + ((!LINF && p.relu) ? 1e-6f : 0.f);
+        const float inv_den = (p.do_linear && den_eps > 0.f) ? 1.f / den_eps : 0.f;
         const __nv_bfloat16* gl =
             (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
         const __nv_bfloat16* gs =

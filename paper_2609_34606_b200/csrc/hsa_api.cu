@@ -62,6 +62,7 @@ bool config_ok(const hsa_config* c) {
   if (c->gate_act != 0 && c->gate_act != 1) return false;
   if (!(c->softmax_scale >= 0.f)) return false;
   if (c->split_blocks < 0) return false;
+  if (c->feature_map != HSA_PHI_ELU1 && c->feature_map != HSA_PHI_RELU) return false;
   if ((c->flags & HSA_CFG_ADAPTIVE) && c->max_pages > 8192) return false;
   return true;
 }
@@ -356,6 +357,7 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
   if (nsplit > by_tokens) nsplit = by_tokens;
   a.nsplit = nsplit;
   a.lin_state = ctx->cfg.lin_mode == HSA_LIN_STATE;
+  a.relu = ctx->cfg.feature_map == HSA_PHI_RELU;
   a.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   const bool linformer = ctx->cfg.lin_mode == HSA_LIN_LINFORMER;
   if (linformer && (n_tokens != ctx->cfg.lin_seg_tokens || ctx->n_tokens != static_cast<int64_t>(ctx->n_segs) * n_tokens))
@@ -577,6 +579,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.flags = flags;
   p.do_linear = do_linear;
+  p.relu = ctx->cfg.feature_map == HSA_PHI_RELU;
   p.do_sparse = do_sparse;
   p.status = reinterpret_cast<int32_t*>(ws + ctx->lay.status);
   p.max_splits = 1;
@@ -604,6 +607,7 @@ int hsa_forward(hsa_ctx* ctx, const void* q, int32_t n_q, int64_t tok_stride, in
     c.n_tokens = ctx->n_tokens;
     c.H = H;
     c.D = D;
+    c.relu = p.relu;
     c.lin_num = reinterpret_cast<float*>(ws + ctx->lay.lin_num);
     c.lin_den = reinterpret_cast<float*>(ws + ctx->lay.lin_den);
     cudaError_t e = launch_causal_linear(c, st);

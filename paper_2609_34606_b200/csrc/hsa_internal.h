@@ -50,6 +50,7 @@ struct AppendArgs {
   float* spart;         // [H][nsplit][D*D + D] scratch
   int nsplit;
   int lin_state;  // update the linear state?
+  int relu;       // feature map of the state: 0 elu(x) + 1, 1 max(x, 0)
   int32_t* status;  // device status word
 };
 
@@ -127,6 +128,7 @@ struct FwdParams {
   // pool (page ids through lf_table), with an accumulator and row sums of their own (null: none)
   const int32_t* lf_table;
   int lf_pages;
+  int relu;  // feature map of the state form: 0 elu(x) + 1, 1 max(x, 0) with 1e-6 added to the denominator
   // split tiles: a (tile, head) with more than split_blocks selected blocks runs as several CTAs
   // (grid z = max_splits); each dumps its unnormalised O, row sums and exponent references, the last
   // one to take a ticket merges them and writes the output
@@ -153,6 +155,7 @@ struct CausalLinArgs {
   int64_t q_pos0;   // first query position == first token of the intra-chunk part
   int64_t n_tokens;
   int H, D;
+  int relu;  // feature map: 0 elu(x) + 1, 1 max(x, 0)
   float* lin_num;
   float* lin_den;
 };

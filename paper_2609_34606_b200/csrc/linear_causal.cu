@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(256) causal_linear_kernel(CausalLinArgs a) {
 #pragma unroll
   for (int e = 0; e < PER; ++e) {
     const float x = __bfloat162float(qrow[e]);
-    fq[e] = x > 0.f ? x + 1.f : expf(x);
+    fq[e] = a.relu ? fmaxf(x, 0.f) : (x > 0.f ? x + 1.f : expf(x));
     num[e] = 0.f;
   }
   float den = 0.f;
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) causal_linear_kernel(CausalLinArgs a) {
 #pragma unroll
     for (int e = 0; e < PER; ++e) {
       const float x = __bfloat162float(kr[e]);
-      w = fmaf(fq[e], x > 0.f ? x + 1.f : expf(x), w);
+      w = fmaf(fq[e], a.relu ? fmaxf(x, 0.f) : (x > 0.f ? x + 1.f : expf(x)), w);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);

@@ -86,6 +86,9 @@ __device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t& r0, uint32_t&
 }
 }  // namespace
 
+// RELU: feature map max(x, 0) instead of elu(x) + 1, and 1e-6 in the denominator (an instance of its
+// own: the map sits in the worker warps' innermost loop)
+template <bool RELU>
 __global__ void __launch_bounds__(kLoThreads, 1)
 hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtensorMap tm_q,
                        const __grid_constant__ CUtensorMap tm_state, const __grid_constant__ CUtensorMap tm_out) {
@@ -252,8 +255,10 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
         for (int i = 0; i < 4; ++i) {
           const uint32_t* qw = reinterpret_cast<const uint32_t*>(&raw[i]);
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            o[4 * i + e] = pack_bf16(lo_phi(__uint_as_float(qw[e] << 16)), lo_phi(__uint_as_float(qw[e] & 0xffff0000u)));
+          for (int e = 0; e < 4; ++e) {
+            const float x0 = __uint_as_float(qw[e] << 16), x1 = __uint_as_float(qw[e] & 0xffff0000u);
+            o[4 * i + e] = RELU ? pack_bf16(fmaxf(x0, 0.f), fmaxf(x1, 0.f)) : pack_bf16(lo_phi(x0), lo_phi(x1));
+          }
         }
         // this thread's 32 values of phi(q) are 16 columns of its TMEM lane
         tmem_st16(tmem + lane_off + kLoSlotCols * (it % kLoSlots) + kLoColA + cq * 16, o);
@@ -284,7 +289,7 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
         const bool wr = row < p.n_q;  // rows past the end of the chunk compute but never store
         uint32_t packed[16];
         if (plain) {
-          const float inv_den = den > 0.f ? 1.f / den : 0.f;
+          const float inv_den = RELU ? 1.f / (den + 1e-6f) : (den > 0.f ? 1.f / den : 0.f);
 #pragma unroll
           for (int i = 0; i < 32; i += 2)
             packed[i >> 1] = pack_bf16(__uint_as_float(v[i]) * inv_den, __uint_as_float(v[i + 1]) * inv_den);
@@ -294,7 +299,7 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
             lnum = p.lin_num + (static_cast<size_t>(row) * p.H + h) * D + cq * 32;
             den += p.lin_den[static_cast<size_t>(row) * p.H + h];
           }
-          const float inv_den = den > 0.f ? 1.f / den : 0.f;
+          const float inv_den = RELU ? 1.f / (den + 1e-6f) : (den > 0.f ? 1.f / den : 0.f);
           const __nv_bfloat16* gl =
               (wr && p.g_lin) ? p.g_lin + static_cast<size_t>(row) * p.g_ts + static_cast<size_t>(h) * p.g_hs : nullptr;
           const int g_ds = static_cast<int>(p.g_ds);
@@ -334,7 +339,10 @@ hsa_linear_only_kernel(FwdParams p, int n_items, const __grid_constant__ CUtenso
 }
 
 cudaError_t linear_only_init() {
-  return cudaFuncSetAttribute(hsa_linear_only_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLoSmem);
+  cudaError_t e = cudaFuncSetAttribute(hsa_linear_only_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLoSmem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(hsa_linear_only_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLoSmem);
+  return e;
 }
 
 cudaError_t launch_linear_only(const FwdParams& p, int nsm, const CUtensorMap& tm_q, const CUtensorMap& tm_state,
@@ -352,7 +360,8 @@ cudaError_t launch_linear_only(const FwdParams& p, int nsm, const CUtensorMap& t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, hsa_linear_only_kernel, p, n_items, tm_q, tm_state, tm_out);
+  if (p.relu) return cudaLaunchKernelEx(&cfg, hsa_linear_only_kernel<true>, p, n_items, tm_q, tm_state, tm_out);
+  return cudaLaunchKernelEx(&cfg, hsa_linear_only_kernel<false>, p, n_items, tm_q, tm_state, tm_out);
 }
 
 }  // namespace hsa

@@ -29,6 +29,7 @@ HSA_ERR_CUDA = -4
 HSA_ERR_DEVICE_TIMEOUT = -5
 HSA_ERR_DEVICE_BOUNDS = -6
 HSA_LIN_NONE, HSA_LIN_STATE, HSA_LIN_LINFORMER = 0, 1, 2
+HSA_PHI_ELU1, HSA_PHI_RELU = 0, 1
 HSA_CFG_CAUSAL = 1
 HSA_CFG_ADAPTIVE = 2
 HSA_CFG_GRID_BARRIER_SELECT = 4
@@ -54,7 +55,7 @@ class hsa_config(C.Structure):
                 ("max_pages", C.c_int32), ("max_q_tokens", C.c_int32), ("max_topk", C.c_int32),
                 ("lin_mode", C.c_int32), ("gate_act", C.c_int32), ("softmax_scale", C.c_float),
                 ("flags", C.c_uint32), ("lin_rank", C.c_int32), ("lin_seg_tokens", C.c_int32),
-                ("split_blocks", C.c_int32)]
+                ("split_blocks", C.c_int32), ("feature_map", C.c_int32)]
 
 
 class hsa_select_opts(C.Structure):
@@ -321,14 +322,14 @@ class HSAContext:
                  causal: bool = False, page_order: Optional[torch.Tensor] = None,
                  device: str | torch.device = "cuda:0", adaptive: bool = False, lin_rank: int = 0, lin_seg_tokens: int = 0,
                  e_k: Optional[torch.Tensor] = None, e_v: Optional[torch.Tensor] = None, split_blocks: int = 0,
-                 grid_barrier_select: bool = False):
+                 grid_barrier_select: bool = False, feature_map: int = 0):
         self.device = torch.device(device)
         self.H, self.d = H, d
         self.max_pages, self.max_q_tokens, self.max_topk = max_pages, max_q_tokens, max_topk
         self.cfg = hsa_config(H, d, PAGE_TOKENS, max_pages, max_q_tokens, max_topk, lin_mode, gate_act,
                               softmax_scale, (HSA_CFG_CAUSAL if causal else 0) | (HSA_CFG_ADAPTIVE if adaptive else 0) |
                               (HSA_CFG_GRID_BARRIER_SELECT if grid_barrier_select else 0),
-                              lin_rank, lin_seg_tokens, split_blocks)
+                              lin_rank, lin_seg_tokens, split_blocks, feature_map)
         self.sizes = hsa_query_sizes(self.cfg)
         with torch.cuda.device(self.device):
             mk = lambda n: torch.empty(max(n, 16), dtype=torch.uint8, device=self.device)

@@ -24,7 +24,7 @@ def f32(t: torch.Tensor) -> np.ndarray:
 
 
 def build_context(w: W.Workload, device, max_topk=None, causal=None, extra_pages=0, lin_mode=1,
-                  gate_act=0, split_blocks=0, grid_barrier_select=False):
+                  gate_act=0, split_blocks=0, grid_barrier_select=False, feature_map=0):
     from paper_2609_34606_b200 import hsa
     max_pages = w.n_blocks + extra_pages
     order = W.gen_page_order(w, max_pages)
@@ -32,7 +32,7 @@ def build_context(w: W.Workload, device, max_topk=None, causal=None, extra_pages
                          max_topk=max_topk or max(w.n_blocks, 1), lin_mode=lin_mode,
                          gate_act=gate_act, causal=w.causal if causal is None else causal,
                          page_order=order, device=device, split_blocks=split_blocks,
-                         grid_barrier_select=grid_barrier_select)
+                         grid_barrier_select=grid_barrier_select, feature_map=feature_map)
     # poison the pools (0xFFFF is a bf16 NaN): anything read but never written shows up
     ctx.k_pool.fill_(0xFF)
     ctx.v_pool.fill_(0xFF)
@@ -102,10 +102,10 @@ def oracle_inputs(w: W.Workload, K: torch.Tensor, V: torch.Tensor, q: torch.Tens
     return f32(q), f32(K), f32(V)
 
 
-def run_case(w: W.Workload, device, group_tokens=0, gates=None, gate_act=0, check_state=True):
+def run_case(w: W.Workload, device, group_tokens=0, gates=None, gate_act=0, check_state=True, fmap="elu1"):
     """Full path on the GPU and in the oracle; returns a dict of error statistics."""
     from paper_2609_34606_b200 import hsa
-    ctx = build_context(w, device, gate_act=gate_act)
+    ctx = build_context(w, device, gate_act=gate_act, feature_map=1 if fmap == "relu" else 0)
     K, V = append_history(ctx, w, device)
     q = W.gen_query(w)
     qd = q.to(device)
@@ -113,7 +113,7 @@ def run_case(w: W.Workload, device, group_tokens=0, gates=None, gate_act=0, chec
     qn, Kn, Vn = oracle_inputs(w, K, V, q)
     res = {}
     if check_state:
-        S_ref, z_ref = O.linear_state(Kn, Vn)
+        S_ref, z_ref = O.linear_state(Kn, Vn, fmap=fmap)
         kbar = O.block_key_means(Kn)
         cnts = np.array([O.block_count(b, w.N) for b in range(w.n_blocks)])
         ksum_ref = (kbar * cnts[:, None, None]).transpose(1, 0, 2)
@@ -134,7 +134,7 @@ def run_case(w: W.Workload, device, group_tokens=0, gates=None, gate_act=0, chec
         gl_n, gs_n = f64(g_lin), f64(g_sp)
         g_lin, g_sp = g_lin.to(device), g_sp.to(device)
     # the oracle evaluates the GPU's own selection (identical up to forgiven ties)
-    ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, w.causal, sel_gpu, group_tokens, gl_n, gs_n, gate_act)
+    ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, w.causal, sel_gpu, group_tokens, gl_n, gs_n, gate_act, fmap=fmap)
     out = ctx.forward(qd, sel_idx, sel_cnt, q_pos0=w.q_pos0, causal=w.causal, group_tokens=group_tokens,
                       g_lin=g_lin, g_sp=g_sp)
     o_sp = ctx.forward(qd, sel_idx, sel_cnt, q_pos0=w.q_pos0, causal=w.causal,

@@ -42,9 +42,10 @@ def test_query_sizes_and_config_validation():
     big = hsa.hsa_query_sizes(hsa.hsa_config(12, 128, 64, 732, 4680, 64, 1, 0, 0.0, hsa.HSA_CFG_CAUSAL))
     assert big.workspace >= s.workspace + 4680 * 12 * 128 * 4
     for bad in [dict(head_dim=96), dict(page_tokens=32), dict(num_heads=0), dict(max_pages=0),
-                dict(lin_mode=2), dict(gate_act=3), dict(max_topk=0)]:
+                dict(lin_mode=2), dict(gate_act=3), dict(max_topk=0), dict(feature_map=2)]:
         kw = dict(num_heads=12, head_dim=128, page_tokens=64, max_pages=8, max_q_tokens=128, max_topk=4,
-                  lin_mode=1, gate_act=0, softmax_scale=0.0, flags=0)
+                  lin_mode=1, gate_act=0, softmax_scale=0.0, flags=0, lin_rank=0, lin_seg_tokens=0,
+                  split_blocks=0, feature_map=0)
         kw.update(bad)
         with pytest.raises(hsa.HSAError) as e:
             hsa.hsa_query_sizes(hsa.hsa_config(*kw.values()))

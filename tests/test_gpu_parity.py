@@ -18,6 +18,40 @@ def test_small_workloads_full_parity(name, cuda_device):
     Hn.run_case(W.WORKLOADS[name], cuda_device)
 
 
+@pytest.mark.parametrize("name", ["mid_d128", "mid_mix", "mid_causal", "mid_d64", "cfg1b"])
+def test_relu_feature_map(name, cuda_device):
+    """phi(x) = max(x, 0) in every kernel that applies the feature map (fused and SIMT append, the
+    forward epilogue, the stand-alone linear kernel, the causal intra-chunk part), with 1e-6 in the
+    denominator: state, both branches and the merged output against the oracle's relu form."""
+    res = Hn.run_case(W.WORKLOADS[name], cuda_device, fmap="relu")
+    assert res["S_rel"] <= 1e-5 and res["z_rel"] <= 1e-5
+
+
+def test_relu_rows_without_any_weight_are_zero(cuda_device):
+    """Queries with no positive component have weight zero on every key: the linear branch of those
+    rows is 0 / 1e-6 = 0 (no division by zero, no NaN), in the fused epilogue and in the stand-alone
+    linear kernel; the other rows match the oracle."""
+    from paper_2609_34606_b200 import hsa
+    w = W.WORKLOADS["mid_d128"]
+    ctx = Hn.build_context(w, cuda_device, feature_map=1)
+    K, V = Hn.append_history(ctx, w, cuda_device)
+    q = W.gen_query(w).float()
+    q[::3] = -q[::3].abs()            # every third row: all components negative
+    q = q.to(torch.bfloat16)
+    qd = q.to(cuda_device)
+    si, sc = ctx.select_blocks(qd, W.gen_budgets(w).to(cuda_device))
+    o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
+    out = Hn.f64(ctx.forward(qd, si, sc))
+    o_sp = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_LINEAR))
+    assert ctx.device_status() == 0
+    assert np.isfinite(o_lin).all() and np.isfinite(out).all()
+    assert not o_lin[::3].any()
+    assert np.abs(out[::3] - o_sp[::3]).max() == 0.0
+    ref = O.linear_parallel(Hn.f32(q), Hn.f32(K), Hn.f32(V), w.q_pos0, False, fmap="relu")
+    Hn.assert_close(o_lin, ref, "O_lin (relu)")
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("gates,act", [("head", 0), ("dim", 1), ("head", 1)])
 def test_gated_merge(gates, act, cuda_device):
     Hn.run_case(W.WORKLOADS["mid_d128"], cuda_device, gates=gates, gate_act=act, check_state=False)
