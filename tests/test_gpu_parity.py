@@ -262,20 +262,20 @@ def test_selection_kcap_clamp_and_large_candidate_sets(cuda_device):
     ctx.destroy()
 
 
-@pytest.mark.parametrize("name", ["cfg2"])
-def test_full_size_sampled_parity(name, cuda_device):
-    """Full-size workload in the launch configuration the benchmark times: selection checked in full,
-    outputs on the first and last query tile plus seeded random rows (rows are independent given the
-    selection), state and key sums in full."""
+@pytest.mark.parametrize("name,fmap", [("cfg2", "elu1"), ("cfg2", "relu")])
+def test_full_size_sampled_parity(name, fmap, cuda_device):
+    """Full-size workload in the launch configuration the benchmark times (and the same with the relu
+    feature map): selection checked in full, outputs on the first and last query tile plus seeded
+    random rows (rows are independent given the selection), state and key sums in full."""
     from paper_2609_34606_b200 import hsa
     w = W.WORKLOADS[name]
-    ctx = Hn.build_context(w, cuda_device, max_topk=max(w.topk, 1))
+    ctx = Hn.build_context(w, cuda_device, max_topk=max(w.topk, 1), feature_map=1 if fmap == "relu" else 0)
     K, V = Hn.append_history(ctx, w, cuda_device)
     q = W.gen_query(w)
     qd = q.to(cuda_device)
     budgets = W.gen_budgets(w)
     qn, Kn, Vn = Hn.f32(q), Hn.f32(K), Hn.f32(V)
-    S_ref, z_ref = O.linear_state(Kn, Vn)
+    S_ref, z_ref = O.linear_state(Kn, Vn, fmap=fmap)
     assert np.linalg.norm(Hn.f64(ctx.S) - S_ref) <= 1e-5 * np.linalg.norm(S_ref)
     assert np.linalg.norm(Hn.f64(ctx.z) - z_ref) <= 1e-5 * np.linalg.norm(z_ref)
     si, sc = ctx.select_blocks(qd, budgets.to(cuda_device))
@@ -283,7 +283,7 @@ def test_full_size_sampled_parity(name, cuda_device):
     sel_ref, scores = O.select_blocks(qn, Kn, w.q_pos0, w.causal, budgets.tolist())
     Hn.check_selection(sel_gpu, sel_ref, scores)
     rows = W.sample_rows(w, n_random=256).numpy()
-    ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, w.causal, sel_gpu, rows=rows, linear_form="state")
+    ref = O.hsa_forward(qn, Kn, Vn, w.q_pos0, w.causal, sel_gpu, rows=rows, linear_form="state", fmap=fmap)
     out = Hn.f64(ctx.forward(qd, si, sc))
     o_sp = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_LINEAR))
     o_lin = Hn.f64(ctx.forward(qd, si, sc, flags=hsa.HSA_FWD_NO_SPARSE))
