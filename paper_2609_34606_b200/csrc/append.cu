@@ -73,6 +73,10 @@ __global__ void __launch_bounds__(256) append_pool_ksum_kernel(AppendArgs a) {
     }
     *dst = old + s;
   }
+  // Launched as a programmatic dependent (Linformer form: behind the compression kernel, whose
+  // outputs it does not touch) this grid runs beside that kernel and waits for it only here, so
+  // that its own end implies that kernel's.  Launched normally this is a no-op.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------
@@ -600,11 +604,20 @@ cudaError_t launch_append(const AppendArgs& a_in, const AppendMaps* maps, cudaSt
     if (e != cudaSuccess) return e;
   } else {
     dim3 gridA(static_cast<unsigned>(b1 - b0 + 1), a.H);
+    cudaLaunchConfig_t cfgA{};
+    cfgA.gridDim = gridA;
+    cfgA.blockDim = dim3(256);
+    cfgA.stream = st;
+    cudaLaunchAttribute attrA[1];
+    attrA[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrA[0].val.programmaticStreamSerializationAllowed = 1;
+    cfgA.attrs = attrA;
+    cfgA.numAttrs = a.beside_prior ? 1 : 0;  // (only behind a kernel whose outputs this one leaves alone)
     if (a.D == 128)
-      append_pool_ksum_kernel<128><<<gridA, 256, 0, st>>>(a);
+      e = cudaLaunchKernelEx(&cfgA, append_pool_ksum_kernel<128>, a);
     else
-      append_pool_ksum_kernel<64><<<gridA, 256, 0, st>>>(a);
-    e = cudaGetLastError();
+      e = cudaLaunchKernelEx(&cfgA, append_pool_ksum_kernel<64>, a);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess || !a.lin_state) return e;
     dim3 gridB(a.nsplit, a.H);
     if (a.D == 128)

@@ -371,8 +371,11 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     maps.kpool = ctx->tm_k;
     maps.vpool = ctx->tm_v;
   }
-  cudaError_t e = launch_append(a, fused ? &maps : nullptr, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  cudaError_t e = cudaSuccess;
+  if (!linformer) {
+    e = launch_append(a, fused ? &maps : nullptr, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+  }
   if (linformer) {
     LinformerArgs la{};
     la.k = a.k;
@@ -390,6 +393,11 @@ int hsa_append_kv(hsa_ctx* ctx, const void* k, const void* v, int32_t n_tokens, 
     la.seg_index = ctx->n_segs;
     la.status = a.status;
     e = launch_linformer_compress(la, ctx->tm_ek, ctx->tm_ev, maps.kin, maps.vin, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    // pages and key sums of the chunk: launched behind the compression kernel, runs beside it (the
+    // two write nothing in common) and ends after it
+    a.beside_prior = 1;
+    e = launch_append(a, nullptr, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->n_segs += 1;
   }

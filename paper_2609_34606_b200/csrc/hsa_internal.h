@@ -50,6 +50,7 @@ struct AppendArgs {
   float* spart;         // [H][nsplit][D*D + D] scratch
   int nsplit;
   int lin_state;  // update the linear state?
+  int beside_prior;  // SIMT page write: may run beside the kernel launched just before it (see launch_append)
   int relu;       // feature map of the state: 0 elu(x) + 1, 1 max(x, 0)
   int32_t* status;  // device status word
 };

@@ -62,6 +62,9 @@ linformer_compress_kernel(LinformerArgs a, const __grid_constant__ CUtensorMap t
   __nv_bfloat16* pool = which == 0 ? a.kc_pool : a.vc_pool;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nblk = (a.seg_tokens + kBlock - 1) / kBlock;
+  // the page-write kernel of the same append is launched behind this one as a programmatic
+  // dependent and may run beside it (it touches none of this kernel's outputs)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kLcDepth; ++s) {
