@@ -92,7 +92,7 @@ typedef struct {
   int32_t gate_act;       /* 0: gates used as given; 1: sigmoid(gate) (Section 3.3, Eq. 5)     */
   float softmax_scale;    /* 0 -> 1/sqrt(head_dim)                                             */
   uint32_t flags;         /* HSA_CFG_* bits                                                    */
-  int32_t lin_rank;       /* HSA_LIN_LINFORMER: projection rank r, a multiple of 128 (else 0)         */
+  int32_t lin_rank;       /* HSA_LIN_LINFORMER: projection rank r, a multiple of 64, 64..2048 (else 0) */
   int32_t lin_seg_tokens; /* HSA_LIN_LINFORMER: segment length L; every append must be exactly L      */
   int32_t split_blocks;   /* a (query tile, head) with more selected blocks than this is split over
                              several CTAs whose partial results the last one to finish merges

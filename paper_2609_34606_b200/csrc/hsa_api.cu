@@ -56,7 +56,7 @@ bool config_ok(const hsa_config* c) {
     return false;
   if (c->lin_mode == HSA_LIN_LINFORMER) {
     if (c->head_dim != 128) return false;
-    if (c->lin_rank < 128 || c->lin_rank > 2048 || (c->lin_rank % 128) != 0) return false;
+    if (c->lin_rank < kBlock || c->lin_rank > 2048 || (c->lin_rank % kBlock) != 0) return false;  // whole compressed pages
     if (c->lin_seg_tokens < 1 || c->lin_seg_tokens > c->max_q_tokens) return false;
   }
   if (c->gate_act != 0 && c->gate_act != 1) return false;

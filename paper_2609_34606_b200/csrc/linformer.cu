@@ -54,7 +54,7 @@ linformer_compress_kernel(LinformerArgs a, const __grid_constant__ CUtensorMap t
                                              ~static_cast<uintptr_t>(1023));
   LcBars* bars = reinterpret_cast<LcBars*>(smem + kLcDepth * kLcStage);
   const int h = blockIdx.y;
-  const int rtiles = a.rank / 128;
+  const int rtiles = (a.rank + 127) / 128;  // (the last tile may hold 64 rows only: E reads as zeros beyond the rank)
   const int which = blockIdx.x / rtiles;  // 0: keys, 1: values
   const int rt = blockIdx.x % rtiles;
   const CUtensorMap* tm_e = which == 0 ? &tm_ek : &tm_ev;  // [H][seg_tokens][rank], box 64 r x 64 tokens
@@ -124,9 +124,9 @@ linformer_compress_kernel(LinformerArgs a, const __grid_constant__ CUtensorMap t
   __syncwarp();
   const bool ok = lc_wait(&bars->all_done, 0, bars, a.status);
   tc_fence_after();
-  if (ok) {
+  const int rr = rt * 128 + (warp & 3) * 32 + lane;  // row of the compressed segment
+  if (ok && rr < a.rank) {                            // (warp-uniform: the rank is a multiple of 64)
     const int quad = warp & 3, part = warp >> 2;
-    const int rr = rt * 128 + quad * 32 + lane;  // row of the compressed segment
     uint32_t v[32];
     tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + part * 32, v);
     tc_wait_ld();
@@ -154,7 +154,7 @@ cudaError_t linformer_init() {
 
 cudaError_t launch_linformer_compress(const LinformerArgs& a, const CUtensorMap& tm_ek, const CUtensorMap& tm_ev,
                                       const CUtensorMap& tm_kin, const CUtensorMap& tm_vin, cudaStream_t st) {
-  dim3 grid(2 * (a.rank / 128), a.H);
+  dim3 grid(2 * ((a.rank + 127) / 128), a.H);
   linformer_compress_kernel<<<grid, kLcThreads, kLcSmem, st>>>(a, tm_ek, tm_ev, tm_kin, tm_vin);
   return cudaGetLastError();
 }

@@ -534,22 +534,25 @@ def test_linformer_linear_branch(cuda_device):
     ctx.destroy()
 
 
-@pytest.mark.parametrize("n_segs,k_scale,split_blocks,gates", [
-    (1, None, 0, None),          # one compressed step: both softmax groups start in different segments
-    (2, None, 0, "head"),        # gated merge of the two segments' results
-    (4, (0.05, 12.0), 0, None),  # later segments / blocks dominate: both segments overflow the fixed reference
-    (4, None, 4, None),          # long lists split over CTAs: the two-launch form
+@pytest.mark.parametrize("n_segs,k_scale,split_blocks,gates,rank", [
+    (1, None, 0, None, 128),          # one compressed step: both softmax groups start in different segments
+    (2, None, 0, "head", 128),        # gated merge of the two segments' results
+    (4, (0.05, 12.0), 0, None, 128),  # later segments / blocks dominate: both segments overflow the fixed reference
+    (4, None, 4, None, 128),          # long lists split over CTAs: the two-launch form
+    (3, None, 0, None, 192),          # three compressed pages per segment: an odd page count, a half-filled tile
+    (1, None, 0, None, 64),           # the smallest rank: one compressed page in all
 ])
-def test_linformer_segments_inside_the_forward_kernel(n_segs, k_scale, split_blocks, gates, cuda_device):
+def test_linformer_segments_inside_the_forward_kernel(n_segs, k_scale, split_blocks, gates, rank, cuda_device):
     """The Linformer form runs as one launch whose loop walks the compressed pool first and the
     selected pages second, each with its own accumulator, exponent reference and row sums.  Cases:
     a single compressed step, gates, a history whose later parts outweigh the first step by far more
-    than the fixed reference allows (the tile is redone with running maxima in both segments), and
-    the split-list configuration, which keeps the form with two launches."""
+    than the fixed reference allows (the tile is redone with running maxima in both segments), the
+    split-list configuration, which keeps the form with two launches, and ranks that are not a
+    multiple of the compression kernel's 128-row tile."""
     from paper_2609_34606_b200 import hsa
     base = W.WORKLOADS["mid_linformer"]
     w = W.Workload("linf_case", H=base.H, d=128, Lq=300, chunk=base.chunk, n_chunks=n_segs, topk=6, seed=90 + n_segs)
-    rank, seg = 128, w.chunk
+    seg = w.chunk
     ek, ev = W.gen_linformer_weights(w, rank, seg)
     ctx = hsa.HSAContext(w.H, w.d, max_pages=w.n_blocks, max_q_tokens=max(w.Lq, w.chunk), max_topk=w.n_blocks,
                          lin_mode=hsa.HSA_LIN_LINFORMER, lin_rank=rank, lin_seg_tokens=seg,
