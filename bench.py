@@ -658,6 +658,53 @@ def bench_reference(args, rank: int, world: int):
         "gpu_launches": 0}), flush=True)
 
 
+# ----------------------------------------------------------------------------- context (third party)
+def context_library_attention(args):
+    """Context only -- neither the product nor the oracle: library attention kernels (torch SDPA back
+    ends, flash_attn, flashinfer, whichever the image has) on dense, contiguous K and V of the size
+    the workload's sparse branch selects (top-k blocks per head), i.e. the same FLOPs as the sparse
+    branch without the page gather.  One JSON line."""
+    w = W.WORKLOADS[args.workload]
+    dev = torch.device("cuda:0")
+    T = min(w.topk * W.BLOCK, w.N)
+    gen = torch.Generator(device="cpu").manual_seed(1234)
+    q, k, v = (torch.randn(1, w.H, n, w.d, generator=gen).to(torch.bfloat16).to(dev) for n in (w.Lq, T, T))
+    flops = 4.0 * w.Lq * T * w.d * w.H
+
+    def timeit(fn, n=50):
+        for _ in range(5):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    res = {}
+    from torch.nn.attention import SDPBackend, sdpa_kernel
+    for name, be in (("torch_sdpa_cudnn", SDPBackend.CUDNN_ATTENTION), ("torch_sdpa_flash", SDPBackend.FLASH_ATTENTION)):
+        try:
+            with sdpa_kernel(be):
+                ms = timeit(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v))
+            res[name] = {"ms": ms, "tflops": flops / ms / 1e9}
+        except Exception as e:  # a back end the build does not have
+            res[name] = {"unavailable": type(e).__name__}
+    try:
+        from flash_attn import flash_attn_func
+        q2, k2, v2 = (t.transpose(1, 2).contiguous() for t in (q, k, v))
+        ms = timeit(lambda: flash_attn_func(q2, k2, v2))
+        res["flash_attn"] = {"ms": ms, "tflops": flops / ms / 1e9}
+    except Exception as e:
+        res["flash_attn"] = {"unavailable": type(e).__name__}
+    print(json.dumps({"context": "third-party attention kernels on dense contiguous K, V of the selected size "
+                                 "(same FLOPs as the sparse branch, no page gather); not the product, not the oracle",
+                      "workload": f"{w.name}: H={w.H} d={w.d} Lq={w.Lq} keys={T}", "flops": flops, "results": res}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -682,6 +729,9 @@ def main():
     ap.add_argument("--profile", action="store_true",
                     help="profiling run: set-up, warm-up and the K timed steps only (no clock probe loop, "
                          "no end-to-end loop, no CPU baseline), for use under ncu")
+    ap.add_argument("--context", action="store_true",
+                    help="context only: time library attention kernels (third party) on dense K, V of the "
+                         "selected size and exit")
     ap.add_argument("--rank-check", action="store_true",
                     help="start the ranks, let them meet over gloo and report the aggregation of stand-in "
                          "numbers, then exit before any GPU is touched (checks the launcher on a CPU box)")
@@ -697,6 +747,9 @@ def main():
         sys.exit(f"bench: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if args.rank_check:
         rank_check(rank, world)
+    elif args.context:
+        if rank == 0:
+            context_library_attention(args)
     elif args.impl == "reference":
         bench_reference(args, rank, world)
     elif W.WORKLOADS[args.workload].layers > 1:
